@@ -1,0 +1,174 @@
+/*
+ * dqrm.h - C ABI of the B200 (sm_100a) library for the embedding half of a DQRM
+ * training step: quantisation-aware training of DLRM embedding tables
+ * ("DQRM: Deep Quantized Recommendation Models", arXiv 2410.20046).
+ *
+ * The calls follow the paper's statement of the problem:
+ *   - Section 3.1 / Figure 2(b): run the embedding lookup first, then quantise only
+ *     the rows the batch uses                                   -> dqrm_emb_fwd
+ *   - Section 3.2: the per-table scale is found by traversing the whole table and is
+ *     refreshed only every P iterations                         -> dqrm_scale_refresh
+ *   - Section 4.3 / Appendix B.1: the embedding gradient is a sparse (indices, values)
+ *     tensor over the touched rows, duplicates coalesced        -> dqrm_emb_bwd
+ *   - Appendix B.1: only the values are quantised to INT8, with a scale fixed by the
+ *     bit width and the tensor's distribution                   -> dqrm_grad_quant_int8
+ *   - Appendix B.1: the local step uses the dequantised gradient; Section 3.1: the FP32
+ *     master copy is what is updated                            -> dqrm_row_update
+ *
+ * Quantiser (the paper prints no formula; Section 4.1 fixes "one scale per table",
+ * Appendix A "uniform mapping" and "static min-max clipping range"):
+ *     n(b) = 2^(b-1) - 1
+ *     scale(absmax, b) = max(absmax, 1e-8f) / (float)n(b)                 one FP32 divide
+ *     Q(x; s, b) = clamp(round_half_even(x / s), -2^(b-1), 2^(b-1) - 1)   one FP32 divide
+ *     DQ(q; s)   = (float)q * s                                           one FP32 multiply
+ * Every FP32 operation is a single IEEE round-to-nearest operation (no reciprocal
+ * shortcuts, no fused multiply-add where two roundings are specified).
+ *
+ * Conventions
+ *   - All array arguments are DEVICE pointers unless the name starts with h_ (host).
+ *     The caller owns every buffer.  After dqrm_create the library allocates nothing;
+ *     scratch comes from a caller-provided workspace (see dqrm_workspace_bytes).
+ *   - `stream` is a cudaStream_t passed as void*; calls are asynchronous on it.  Calls
+ *     that share a context or a workspace must be ordered on one stream.
+ *   - Tables live in one arena [sum_t R_t, D] float32, row-major, base aligned to 16
+ *     bytes; row_off[t] is the first arena row of table t.  D is a multiple of 4,
+ *     4 <= D <= 1024.  sum_t R_t < 2^31.
+ *   - indices[L] int32: row numbers within their table, 0 <= idx < R_t, table-major
+ *     (all lookups of table 0 in sample order, then table 1, ...).
+ *   - offsets[T*B + 1] int32, non-decreasing, offsets[0] = 0, offsets[T*B] = L:
+ *     bag g = t*B + i owns indices[offsets[g] .. offsets[g+1]).  Empty bags are allowed.
+ *   - out and grad_out are [B, T, D] float32 (sample-major).  T*B < 2^31.
+ *   - bits[T] int32, each in 2..16.  scales[T] float32.
+ *   - Return value: DQRM_OK or a negative error.  Invalid arguments are detected on the
+ *     host before anything is launched.  Conditions only the device can see (an index
+ *     outside its table, offsets that decrease or leave [0, L]) never trap: the
+ *     offending value is clamped into range, an error code is recorded in the context's
+ *     device status word, and dqrm_check_status reports it.
+ */
+#ifndef DQRM_H_
+#define DQRM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DQRM_OK                 0
+#define DQRM_ERR_INVALID_ARG   (-1)  /* null pointer, bad T/D/B/L, bits outside 2..16 */
+#define DQRM_ERR_WORKSPACE     (-2)  /* workspace null, misaligned (256 B) or too small */
+#define DQRM_ERR_CUDA          (-3)  /* a CUDA runtime call failed; see dqrm_last_cuda_error */
+#define DQRM_ERR_INDEX_RANGE   (-4)  /* device saw an index outside [0, R_t) or a bad offset */
+#define DQRM_ERR_TIMEOUT       (-5)  /* reserved: a bounded device-side wait ran out */
+
+typedef struct dqrm_ctx dqrm_ctx;
+
+/* Creates a context for T tables of feature size D on the current device.
+ * h_row_off: HOST array [T+1], h_row_off[0] = 0, strictly increasing.
+ * Allocates a few KB of device memory (row offsets, status word).  Not stream-ordered:
+ * synchronises the device. */
+int dqrm_create(dqrm_ctx **ctx, int T, int D, const int64_t *h_row_off);
+
+/* Frees what dqrm_create allocated.  The caller must have synchronised its streams. */
+int dqrm_destroy(dqrm_ctx *ctx);
+
+/* Bytes of scratch the calls below need for at most max_lookups lookups and max_bags
+ * bags per call.  The workspace must be 256-byte aligned.  Contents need not be
+ * preserved between calls and need no initialisation. */
+size_t dqrm_workspace_bytes(const dqrm_ctx *ctx, int64_t max_lookups, int64_t max_bags);
+
+/* Synchronises `stream`, returns DQRM_OK or the first device-detected error since the
+ * last check, and clears the status word. */
+int dqrm_check_status(dqrm_ctx *ctx, void *stream);
+
+/* The cudaError_t (as int) of the last failed runtime call on this context, 0 if none. */
+int dqrm_last_cuda_error(const dqrm_ctx *ctx);
+
+/* Static text for a DQRM_* code. */
+const char *dqrm_status_string(int status);
+
+/* Scale refresh (Section 3.2): for every table, min and max over all R_t*D elements,
+ * a = max(|min|, |max|), scales[t] = scale(a, bits[t]).
+ *   tables  in   [sum R_t, D]
+ *   bits    in   [T]
+ *   scales  out  [T]
+ *   minmax  out  [T][2] (min, max), may be NULL
+ * Reads the arena once.  Bit-exact: min/max do not depend on the order of evaluation. */
+int dqrm_scale_refresh(dqrm_ctx *ctx, const float *tables, const int32_t *bits,
+                       float *scales, float *minmax,
+                       void *workspace, size_t workspace_bytes, void *stream);
+
+/* Forward (Section 3.1, Figure 2(b)): for every bag, gather its rows from the FP32
+ * master table, fake-quantise each gathered row with its table's stored scale and bit
+ * width, and sum over the bag (in bag order, FP64 accumulator, rounded once):
+ *   out[i][t][:] = sum_{j in bag (t,i)} DQ(Q(W_t[indices[j]][:]; scales[t], bits[t]); scales[t])
+ *   codes_out    out [L][D] int8, the integer codes of every gathered row; may be NULL;
+ *                only meaningful when every bits[t] <= 8.
+ * The table is not modified and no low-precision copy of it is ever made. */
+int dqrm_emb_fwd(dqrm_ctx *ctx, const float *tables, const int32_t *indices,
+                 const int32_t *offsets, const float *scales, const int32_t *bits,
+                 float *out, int8_t *codes_out, int B, int64_t L, void *stream);
+
+/* Backward (Section 4.3, Appendix B.1): sum pooling and a straight-through quantiser
+ * hand every lookup its bag's upstream gradient unchanged; lookups of the same
+ * (table, row) are summed (FP64 accumulator, rounded once to FP32).
+ *   grad_out     in   [B][T][D]
+ *   unique_rows  out  [>= L] int32: per table ascending distinct row numbers, table-major
+ *   uniq_off     out  [T+1] int32: table t owns unique_rows[uniq_off[t] .. uniq_off[t+1])
+ *   grad_rows    out  [>= L][D] float32: summed gradient of each unique row
+ * Takes neither tables nor scales: the pass-through backward needs neither.
+ * Entries of unique_rows / grad_rows at and beyond uniq_off[T] are left untouched.
+ * Deterministic: the same inputs give the same bits on every run. */
+int dqrm_emb_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices,
+                 const int32_t *offsets, int32_t *unique_rows, int32_t *uniq_off,
+                 float *grad_rows, int B, int64_t L,
+                 void *workspace, size_t workspace_bytes, void *stream);
+
+/* INT8 gradient quantiser (Appendix B.1): per table t over its U_t*D summed gradients,
+ *   grad_scales[t] = scale(max |grad_rows|, 8);  codes = Q(grad_rows; grad_scales[t], 8).
+ * A table that touched no row gets scale(0, 8) and no codes.
+ *   grad_rows in [U][D], uniq_off in [T+1], codes out [U][D] int8, grad_scales out [T]. */
+int dqrm_grad_quant_int8(dqrm_ctx *ctx, const float *grad_rows, const int32_t *uniq_off,
+                         int8_t *codes, float *grad_scales,
+                         void *workspace, size_t workspace_bytes, void *stream);
+
+/* Touched-row SGD update (Appendix B.1, Section 3.1): for every unique row u of table t,
+ *   g = (float)codes[u][d] * grad_scales[t];  step = lr * g;  W[row][d] = W[row][d] - step
+ * (three separately rounded FP32 operations).  Rows not listed are not read or written.
+ * Rows are distinct, so the update is free of conflicts. */
+int dqrm_row_update(dqrm_ctx *ctx, float *tables, const int32_t *unique_rows,
+                    const int32_t *uniq_off, const int8_t *codes, const float *grad_scales,
+                    float lr, void *stream);
+
+/* One training iteration of the embedding path in the order the paper's loop takes it:
+ * forward, backward, INT8 gradient quantisation, touched-row update.  Results equal
+ * those of the four separate calls; the gradient abs-max is folded into the backward
+ * and the quantiser is fused with the update, which saves launches and one read of
+ * grad_rows.  grad_out is an input (in training it comes from the dense layers). */
+int dqrm_train_step(dqrm_ctx *ctx, float *tables, const int32_t *indices,
+                    const int32_t *offsets, const float *grad_out,
+                    const float *scales, const int32_t *bits,
+                    float *out, int32_t *unique_rows, int32_t *uniq_off, float *grad_rows,
+                    int8_t *codes, float *grad_scales, float lr, int B, int64_t L,
+                    void *workspace, size_t workspace_bytes, void *stream);
+
+/* Bytes of workspace dqrm_train_step_host needs (device staging for the host buffers,
+ * the step's intermediate outputs and the scratch of dqrm_train_step). */
+size_t dqrm_host_step_workspace_bytes(const dqrm_ctx *ctx, int64_t max_lookups, int64_t max_bags);
+
+/* dqrm_train_step for callers whose batch lives in HOST memory: copies h_indices [L],
+ * h_offsets [T*B+1] and h_grad_out [B][T][D] to the device, runs the step, and copies
+ * the pooled output back to h_out [B][T][D]; all on `stream`, asynchronously when the
+ * host buffers are pinned.  tables, scales and bits stay on the device.  The sparse
+ * gradient (unique rows, codes, scales) stays in the workspace. */
+int dqrm_train_step_host(dqrm_ctx *ctx, float *tables, const int32_t *h_indices,
+                         const int32_t *h_offsets, const float *h_grad_out,
+                         const float *scales, const int32_t *bits, float *h_out,
+                         float lr, int B, int64_t L,
+                         void *workspace, size_t workspace_bytes, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DQRM_H_ */
