@@ -1,0 +1,207 @@
+"""ctypes binding of ``libdqrm_b200.so``: argument marshalling only."""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libdqrm_b200.so")
+
+OK = 0
+ERR_INVALID_ARG = -1
+ERR_WORKSPACE = -2
+ERR_CUDA = -3
+ERR_INDEX_RANGE = -4
+ERR_TIMEOUT = -5
+
+_vp = ctypes.c_void_p
+_i = ctypes.c_int
+_i64 = ctypes.c_int64
+_sz = ctypes.c_size_t
+_f = ctypes.c_float
+
+# name -> (restype, argtypes); mirrors include/dqrm.h
+SIGNATURES = {
+    "dqrm_create": (_i, [ctypes.POINTER(_vp), _i, _i, ctypes.POINTER(_i64)]),
+    "dqrm_destroy": (_i, [_vp]),
+    "dqrm_workspace_bytes": (_sz, [_vp, _i64, _i64]),
+    "dqrm_check_status": (_i, [_vp, _vp]),
+    "dqrm_last_cuda_error": (_i, [_vp]),
+    "dqrm_status_string": (ctypes.c_char_p, [_i]),
+    "dqrm_scale_refresh": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "dqrm_emb_fwd": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i64, _vp]),
+    "dqrm_emb_bwd": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i64, _vp, _sz, _vp]),
+    "dqrm_grad_quant_int8": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "dqrm_row_update": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _f, _vp]),
+    "dqrm_train_step": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _f, _i, _i64,
+                             _vp, _sz, _vp]),
+    "dqrm_host_step_workspace_bytes": (_sz, [_vp, _i64, _i64]),
+    "dqrm_train_step_host": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _f, _i, _i64, _vp, _sz, _vp]),
+}
+
+_lib = None
+
+
+class DqrmError(RuntimeError):
+    def __init__(self, call: str, status: int, text: str, cuda_error: int = 0):
+        extra = f" (cudaError {cuda_error})" if cuda_error else ""
+        super().__init__(f"{call} failed: {status} {text}{extra}")
+        self.status = status
+        self.cuda_error = cuda_error
+
+
+def load_library(path: Optional[str] = None):
+    """Loads the CUDA library.  Raises if it has not been built: there is no fallback."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or LIB_PATH
+    if not os.path.exists(p):
+        raise ImportError(
+            f"{p} is missing: build it with `python -m paper_2410_20046_b200.build` "
+            "(nvcc, sm_100a).  This package has no CPU or PyTorch fallback.")
+    lib = ctypes.CDLL(p)
+    for name, (res, args) in SIGNATURES.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def _ptr(t, dtype=None, device="cuda"):
+    """Device (or host) pointer of a contiguous torch tensor; None -> NULL."""
+    if t is None:
+        return None
+    import torch
+
+    assert isinstance(t, torch.Tensor), "expected a torch tensor"
+    assert t.is_contiguous(), "tensor must be contiguous"
+    if dtype is not None:
+        assert t.dtype == dtype, f"expected {dtype}, got {t.dtype}"
+    if device == "cuda":
+        assert t.is_cuda, "expected a CUDA tensor"
+    else:
+        assert not t.is_cuda, "expected a host tensor"
+    return t.data_ptr()
+
+
+def _stream(stream=None):
+    import torch
+
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+class Context:
+    """One ``dqrm_ctx`` plus a torch-allocated workspace.  Method names and argument
+    order are those of the C ABI; tensors stand in for the pointers."""
+
+    def __init__(self, row_off, D: int, max_lookups: int, max_bags: int, host_step: bool = False):
+        import torch
+
+        self.lib = load_library()
+        self.T = len(row_off) - 1
+        self.D = int(D)
+        arr = (_i64 * (self.T + 1))(*[int(x) for x in row_off])
+        h = _vp()
+        rc = self.lib.dqrm_create(ctypes.byref(h), self.T, self.D, arr)
+        self._h = h if rc == OK else None
+        self._check("dqrm_create", rc)
+        self.max_lookups = int(max_lookups)
+        self.max_bags = int(max_bags)
+        self.workspace_bytes = int(self.lib.dqrm_workspace_bytes(self._h, self.max_lookups, self.max_bags))
+        self.workspace = torch.empty(self.workspace_bytes + 256, dtype=torch.uint8, device="cuda")
+        self._ws_ptr = (self.workspace.data_ptr() + 255) // 256 * 256
+        self.host_workspace = None
+        if host_step:
+            self.host_workspace_bytes = int(
+                self.lib.dqrm_host_step_workspace_bytes(self._h, self.max_lookups, self.max_bags))
+            self.host_workspace = torch.empty(self.host_workspace_bytes + 256, dtype=torch.uint8, device="cuda")
+            self._hws_ptr = (self.host_workspace.data_ptr() + 255) // 256 * 256
+
+    # ---- plumbing ----
+    def _check(self, call: str, rc: int):
+        if rc != OK:
+            text = self.lib.dqrm_status_string(rc).decode()
+            ce = self.lib.dqrm_last_cuda_error(self._h) if self._h else 0
+            raise DqrmError(call, rc, text, ce)
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self.lib.dqrm_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def check_status(self, stream=None) -> int:
+        return int(self.lib.dqrm_check_status(self._h, _stream(stream)))
+
+    def raise_on_device_error(self, stream=None):
+        self._check("dqrm_check_status", self.check_status(stream))
+
+    # ---- the calls of include/dqrm.h ----
+    def scale_refresh(self, tables, bits, scales, minmax=None, stream=None):
+        import torch
+
+        self._check("dqrm_scale_refresh", self.lib.dqrm_scale_refresh(
+            self._h, _ptr(tables, torch.float32), _ptr(bits, torch.int32), _ptr(scales, torch.float32),
+            _ptr(minmax, torch.float32), self._ws_ptr, self.workspace_bytes, _stream(stream)))
+
+    def emb_fwd(self, tables, indices, offsets, scales, bits, out, codes_out=None, *, B, L, stream=None):
+        import torch
+
+        self._check("dqrm_emb_fwd", self.lib.dqrm_emb_fwd(
+            self._h, _ptr(tables, torch.float32), _ptr(indices, torch.int32), _ptr(offsets, torch.int32),
+            _ptr(scales, torch.float32), _ptr(bits, torch.int32), _ptr(out, torch.float32),
+            _ptr(codes_out, torch.int8), int(B), int(L), _stream(stream)))
+
+    def emb_bwd(self, grad_out, indices, offsets, unique_rows, uniq_off, grad_rows, *, B, L, stream=None):
+        import torch
+
+        self._check("dqrm_emb_bwd", self.lib.dqrm_emb_bwd(
+            self._h, _ptr(grad_out, torch.float32), _ptr(indices, torch.int32), _ptr(offsets, torch.int32),
+            _ptr(unique_rows, torch.int32), _ptr(uniq_off, torch.int32), _ptr(grad_rows, torch.float32),
+            int(B), int(L), self._ws_ptr, self.workspace_bytes, _stream(stream)))
+
+    def grad_quant_int8(self, grad_rows, uniq_off, codes, grad_scales, stream=None):
+        import torch
+
+        self._check("dqrm_grad_quant_int8", self.lib.dqrm_grad_quant_int8(
+            self._h, _ptr(grad_rows, torch.float32), _ptr(uniq_off, torch.int32), _ptr(codes, torch.int8),
+            _ptr(grad_scales, torch.float32), self._ws_ptr, self.workspace_bytes, _stream(stream)))
+
+    def row_update(self, tables, unique_rows, uniq_off, codes, grad_scales, lr, stream=None):
+        import torch
+
+        self._check("dqrm_row_update", self.lib.dqrm_row_update(
+            self._h, _ptr(tables, torch.float32), _ptr(unique_rows, torch.int32), _ptr(uniq_off, torch.int32),
+            _ptr(codes, torch.int8), _ptr(grad_scales, torch.float32), float(lr), _stream(stream)))
+
+    def train_step(self, tables, indices, offsets, grad_out, scales, bits, out, unique_rows, uniq_off,
+                   grad_rows, codes, grad_scales, lr, *, B, L, stream=None):
+        import torch
+
+        self._check("dqrm_train_step", self.lib.dqrm_train_step(
+            self._h, _ptr(tables, torch.float32), _ptr(indices, torch.int32), _ptr(offsets, torch.int32),
+            _ptr(grad_out, torch.float32), _ptr(scales, torch.float32), _ptr(bits, torch.int32),
+            _ptr(out, torch.float32), _ptr(unique_rows, torch.int32), _ptr(uniq_off, torch.int32),
+            _ptr(grad_rows, torch.float32), _ptr(codes, torch.int8), _ptr(grad_scales, torch.float32),
+            float(lr), int(B), int(L), self._ws_ptr, self.workspace_bytes, _stream(stream)))
+
+    def train_step_host(self, tables, h_indices, h_offsets, h_grad_out, scales, bits, h_out, lr, *, B, L,
+                        stream=None):
+        import torch
+
+        assert self.host_workspace is not None, "create the Context with host_step=True"
+        self._check("dqrm_train_step_host", self.lib.dqrm_train_step_host(
+            self._h, _ptr(tables, torch.float32), _ptr(h_indices, torch.int32, "cpu"),
+            _ptr(h_offsets, torch.int32, "cpu"), _ptr(h_grad_out, torch.float32, "cpu"),
+            _ptr(scales, torch.float32), _ptr(bits, torch.int32), _ptr(h_out, torch.float32, "cpu"),
+            float(lr), int(B), int(L), self._hws_ptr, self.host_workspace_bytes, _stream(stream)))

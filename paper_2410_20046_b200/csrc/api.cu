@@ -1,0 +1,241 @@
+// C ABI of the DQRM embedding-path library: context, argument checks, workspace carving
+// and the order of kernel launches.  No arithmetic of the method lives here.
+#include <new>
+#include <string.h>
+#include "common.cuh"
+
+namespace {
+
+inline cudaStream_t as_stream(void *s) { return reinterpret_cast<cudaStream_t>(s); }
+
+inline bool ws_ok(const void *ws, size_t have, size_t need)
+{
+    return ws != nullptr && (reinterpret_cast<uintptr_t>(ws) % 256u) == 0 && have >= need;
+}
+
+inline bool batch_ok(const dqrm_ctx *ctx, int B, int64_t L)
+{
+    return ctx && B > 0 && L >= 0 && L < (int64_t)1 << 31 && (int64_t)ctx->T * B < ((int64_t)1 << 31) - 1;
+}
+
+struct HostStepLayout {
+    size_t indices, offsets, grad_out, out, unique_rows, uniq_off, grad_rows, codes, grad_scales, step_ws, total;
+};
+
+HostStepLayout host_layout(const dqrm_ctx *ctx, int64_t L, int64_t G)
+{
+    HostStepLayout y;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+    const int64_t Lc = L < 1 ? 1 : L;
+    y.indices = take(sizeof(int32_t) * Lc);
+    y.offsets = take(sizeof(int32_t) * (G + 1));
+    y.grad_out = take(sizeof(float) * G * ctx->D);
+    y.out = take(sizeof(float) * G * ctx->D);
+    y.unique_rows = take(sizeof(int32_t) * Lc);
+    y.uniq_off = take(sizeof(int32_t) * (ctx->T + 1));
+    y.grad_rows = take(sizeof(float) * Lc * ctx->D);
+    y.codes = take((size_t)Lc * ctx->D);
+    y.grad_scales = take(sizeof(float) * ctx->T);
+    y.step_ws = o;
+    y.total = o + dqrm_workspace_bytes(ctx, L, G);
+    return y;
+}
+
+}  // namespace
+
+extern "C" {
+
+int dqrm_create(dqrm_ctx **out, int T, int D, const int64_t *h_row_off)
+{
+    if (!out) return DQRM_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!h_row_off || T <= 0 || T > 2048 || D < 4 || D > 1024 || (D % 4) != 0) return DQRM_ERR_INVALID_ARG;
+    if (h_row_off[0] != 0) return DQRM_ERR_INVALID_ARG;
+    for (int t = 0; t < T; ++t)
+        if (h_row_off[t + 1] <= h_row_off[t]) return DQRM_ERR_INVALID_ARG;
+    if (h_row_off[T] >= ((int64_t)1 << 31)) return DQRM_ERR_INVALID_ARG;
+
+    dqrm_ctx *ctx = new (std::nothrow) dqrm_ctx();
+    if (!ctx) return DQRM_ERR_INVALID_ARG;
+    ctx->T = T;
+    ctx->D = D;
+    ctx->total_rows = h_row_off[T];
+    ctx->key_bits = 1;
+    while (((int64_t)1 << ctx->key_bits) < ctx->total_rows) ctx->key_bits++;
+    ctx->h_row_off = new (std::nothrow) int64_t[T + 1];
+    if (!ctx->h_row_off) { delete ctx; return DQRM_ERR_INVALID_ARG; }
+    memcpy(ctx->h_row_off, h_row_off, sizeof(int64_t) * (T + 1));
+
+    cudaError_t e = cudaGetDevice(&ctx->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, ctx->device);
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_row_off, sizeof(int64_t) * (T + 1));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, sizeof(int));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_done, sizeof(u32));
+    if (e == cudaSuccess) e = cudaMallocHost(&ctx->h_status_pinned, sizeof(int));
+    if (e == cudaSuccess) e = cudaMemcpy(ctx->d_row_off, h_row_off, sizeof(int64_t) * (T + 1), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(ctx->d_done, 0, sizeof(u32));
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        dqrm_destroy(ctx);
+        return DQRM_ERR_CUDA;
+    }
+    *out = ctx;
+    return DQRM_OK;
+}
+
+int dqrm_destroy(dqrm_ctx *ctx)
+{
+    if (!ctx) return DQRM_OK;
+    if (ctx->d_row_off) cudaFree(ctx->d_row_off);
+    if (ctx->d_status) cudaFree(ctx->d_status);
+    if (ctx->d_done) cudaFree(ctx->d_done);
+    if (ctx->h_status_pinned) cudaFreeHost(ctx->h_status_pinned);
+    delete[] ctx->h_row_off;
+    delete ctx;
+    return DQRM_OK;
+}
+
+size_t dqrm_workspace_bytes(const dqrm_ctx *ctx, int64_t max_lookups, int64_t max_bags)
+{
+    if (!ctx || max_lookups < 0 || max_bags < 0) return 0;
+    size_t a = dq_refresh_ws_bytes(ctx);
+    size_t b = dq_bwd_ws_bytes(ctx, max_lookups, max_bags);
+    size_t c = dq_quant_ws_bytes(ctx);
+    size_t m = a > b ? a : b;
+    return m > c ? m : c;
+}
+
+int dqrm_check_status(dqrm_ctx *ctx, void *stream)
+{
+    if (!ctx) return DQRM_ERR_INVALID_ARG;
+    cudaStream_t st = as_stream(stream);
+    DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->h_status_pinned, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
+    DQRM_CUDA_TRY(ctx, cudaStreamSynchronize(st));
+    int s = *ctx->h_status_pinned;
+    if (s != 0) {
+        DQRM_CUDA_TRY(ctx, cudaMemsetAsync(ctx->d_status, 0, sizeof(int), st));
+        DQRM_CUDA_TRY(ctx, cudaStreamSynchronize(st));
+    }
+    return s;
+}
+
+int dqrm_last_cuda_error(const dqrm_ctx *ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+const char *dqrm_status_string(int status)
+{
+    switch (status) {
+    case DQRM_OK: return "ok";
+    case DQRM_ERR_INVALID_ARG: return "invalid argument";
+    case DQRM_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case DQRM_ERR_CUDA: return "CUDA runtime error";
+    case DQRM_ERR_INDEX_RANGE: return "index or offset out of range (detected on the device)";
+    case DQRM_ERR_TIMEOUT: return "bounded device-side wait ran out";
+    default: return "unknown status";
+    }
+}
+
+int dqrm_scale_refresh(dqrm_ctx *ctx, const float *tables, const int32_t *bits, float *scales, float *minmax,
+                       void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!ctx || !tables || !bits || !scales) return DQRM_ERR_INVALID_ARG;
+    if (!ws_ok(workspace, workspace_bytes, dq_refresh_ws_bytes(ctx))) return DQRM_ERR_WORKSPACE;
+    return dq_launch_refresh(ctx, tables, bits, scales, minmax, workspace, workspace_bytes, as_stream(stream));
+}
+
+int dqrm_emb_fwd(dqrm_ctx *ctx, const float *tables, const int32_t *indices, const int32_t *offsets,
+                 const float *scales, const int32_t *bits, float *out, int8_t *codes_out, int B, int64_t L,
+                 void *stream)
+{
+    if (!batch_ok(ctx, B, L) || !tables || !offsets || !scales || !bits || !out) return DQRM_ERR_INVALID_ARG;
+    if (L > 0 && !indices) return DQRM_ERR_INVALID_ARG;
+    return dq_launch_fwd(ctx, tables, indices, offsets, scales, bits, out, codes_out, B, L, as_stream(stream));
+}
+
+int dqrm_emb_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, const int32_t *offsets,
+                 int32_t *unique_rows, int32_t *uniq_off, float *grad_rows, int B, int64_t L,
+                 void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!batch_ok(ctx, B, L) || !grad_out || !offsets || !uniq_off) return DQRM_ERR_INVALID_ARG;
+    if (L > 0 && (!indices || !unique_rows || !grad_rows)) return DQRM_ERR_INVALID_ARG;
+    if (!ws_ok(workspace, workspace_bytes, dq_bwd_ws_bytes(ctx, L, (int64_t)ctx->T * B))) return DQRM_ERR_WORKSPACE;
+    return dq_launch_bwd(ctx, grad_out, indices, offsets, unique_rows, uniq_off, grad_rows, B, L, workspace,
+                         workspace_bytes, as_stream(stream), nullptr);
+}
+
+int dqrm_grad_quant_int8(dqrm_ctx *ctx, const float *grad_rows, const int32_t *uniq_off, int8_t *codes,
+                         float *grad_scales, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!ctx || !grad_rows || !uniq_off || !codes || !grad_scales) return DQRM_ERR_INVALID_ARG;
+    if (!ws_ok(workspace, workspace_bytes, dq_quant_ws_bytes(ctx))) return DQRM_ERR_WORKSPACE;
+    return dq_launch_grad_quant(ctx, grad_rows, uniq_off, codes, grad_scales, workspace, workspace_bytes,
+                                as_stream(stream));
+}
+
+int dqrm_row_update(dqrm_ctx *ctx, float *tables, const int32_t *unique_rows, const int32_t *uniq_off,
+                    const int8_t *codes, const float *grad_scales, float lr, void *stream)
+{
+    if (!ctx || !tables || !unique_rows || !uniq_off || !codes || !grad_scales) return DQRM_ERR_INVALID_ARG;
+    return dq_launch_row_update(ctx, tables, unique_rows, uniq_off, codes, grad_scales, lr, as_stream(stream));
+}
+
+int dqrm_train_step(dqrm_ctx *ctx, float *tables, const int32_t *indices, const int32_t *offsets,
+                    const float *grad_out, const float *scales, const int32_t *bits, float *out,
+                    int32_t *unique_rows, int32_t *uniq_off, float *grad_rows, int8_t *codes, float *grad_scales,
+                    float lr, int B, int64_t L, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!batch_ok(ctx, B, L) || !tables || !offsets || !grad_out || !scales || !bits || !out || !uniq_off ||
+        !grad_scales)
+        return DQRM_ERR_INVALID_ARG;
+    if (L > 0 && (!indices || !unique_rows || !grad_rows || !codes)) return DQRM_ERR_INVALID_ARG;
+    if (!ws_ok(workspace, workspace_bytes, dq_bwd_ws_bytes(ctx, L, (int64_t)ctx->T * B))) return DQRM_ERR_WORKSPACE;
+    cudaStream_t st = as_stream(stream);
+    int rc = dq_launch_fwd(ctx, tables, indices, offsets, scales, bits, out, nullptr, B, L, st);
+    if (rc != DQRM_OK) return rc;
+    const u32 *absmax = nullptr;
+    rc = dq_launch_bwd(ctx, grad_out, indices, offsets, unique_rows, uniq_off, grad_rows, B, L, workspace,
+                       workspace_bytes, st, &absmax);
+    if (rc != DQRM_OK) return rc;
+    return dq_launch_quant_update(ctx, tables, unique_rows, uniq_off, grad_rows, absmax, codes, grad_scales, lr, st);
+}
+
+size_t dqrm_host_step_workspace_bytes(const dqrm_ctx *ctx, int64_t max_lookups, int64_t max_bags)
+{
+    if (!ctx || max_lookups < 0 || max_bags < 0) return 0;
+    return host_layout(ctx, max_lookups, max_bags).total;
+}
+
+int dqrm_train_step_host(dqrm_ctx *ctx, float *tables, const int32_t *h_indices, const int32_t *h_offsets,
+                         const float *h_grad_out, const float *scales, const int32_t *bits, float *h_out,
+                         float lr, int B, int64_t L, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!batch_ok(ctx, B, L) || !tables || !h_offsets || !h_grad_out || !scales || !bits || !h_out)
+        return DQRM_ERR_INVALID_ARG;
+    if (L > 0 && !h_indices) return DQRM_ERR_INVALID_ARG;
+    const int64_t G = (int64_t)ctx->T * B;
+    const HostStepLayout y = host_layout(ctx, L, G);
+    if (!ws_ok(workspace, workspace_bytes, y.total)) return DQRM_ERR_WORKSPACE;
+    char *ws = reinterpret_cast<char *>(workspace);
+    cudaStream_t st = as_stream(stream);
+    int32_t *d_idx = reinterpret_cast<int32_t *>(ws + y.indices);
+    int32_t *d_off = reinterpret_cast<int32_t *>(ws + y.offsets);
+    float *d_go = reinterpret_cast<float *>(ws + y.grad_out);
+    float *d_out = reinterpret_cast<float *>(ws + y.out);
+    if (L > 0) DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(d_idx, h_indices, sizeof(int32_t) * L, cudaMemcpyHostToDevice, st));
+    DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(d_off, h_offsets, sizeof(int32_t) * (G + 1), cudaMemcpyHostToDevice, st));
+    DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(d_go, h_grad_out, sizeof(float) * G * ctx->D, cudaMemcpyHostToDevice, st));
+    int rc = dqrm_train_step(ctx, tables, d_idx, d_off, d_go, scales, bits, d_out,
+                             reinterpret_cast<int32_t *>(ws + y.unique_rows),
+                             reinterpret_cast<int32_t *>(ws + y.uniq_off),
+                             reinterpret_cast<float *>(ws + y.grad_rows),
+                             reinterpret_cast<int8_t *>(ws + y.codes),
+                             reinterpret_cast<float *>(ws + y.grad_scales), lr, B, L,
+                             ws + y.step_ws, workspace_bytes - y.step_ws, stream);
+    if (rc != DQRM_OK) return rc;
+    DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(h_out, d_out, sizeof(float) * G * ctx->D, cudaMemcpyDeviceToHost, st));
+    return DQRM_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,653 @@
+// Backward of the embedding lookup (paper Section 4.3 and Appendix B.1): the gradient of
+// an embedding table is a sparse (indices, values) tensor over the rows the batch
+// touched; lookups that hit the same row are coalesced.  Sum pooling and the
+// straight-through quantiser hand every lookup its bag's upstream gradient unchanged.
+//
+// Pipeline (all on one stream, no inter-block waits anywhere):
+//   prepare      one thread per bag: arena-row key + gradient-row payload per lookup,
+//                digit histograms of every radix pass, first pass's per-tile histogram
+//   per pass     scan   : per-digit exclusive scan of the tile histograms (+ digit base)
+//                scatter: stable least-significant-digit scatter of (key, payload);
+//                         counts the next pass's tile histogram on the way
+//   seg_count / seg_emit  head flags of the sorted keys -> unique_rows, uniq_off,
+//                         segment starts, first segment of every 32-entry chunk
+//   seg_reduce   one lane group per 32-entry chunk of the sorted order: gathers the
+//                upstream gradient rows (128-bit loads), sums runs in FP64; runs that are
+//                whole segments are rounded and written, runs cut by a chunk boundary
+//                leave an FP64 partial
+//   seg_fixup    one warp per cut segment: adds its partials in a fixed order
+// The sort is stable and every sum has a fixed shape, so results are reproducible bit
+// for bit.  The per-table abs-max of the summed gradient (needed by the INT8 gradient
+// quantiser) is folded into the last two kernels.
+#include "common.cuh"
+
+namespace {
+
+constexpr int ST_THREADS = 256;
+constexpr int ST_ITEMS = 8;
+constexpr int ST_TILE = ST_THREADS * ST_ITEMS;   // 2048 entries per tile
+constexpr int ST_WARPS = ST_THREADS / 32;
+constexpr int NB_MAX = 512;                      // bins per pass (<= 9 bit digits)
+constexpr int MAX_PASSES = 4;
+constexpr int SEG_CHUNK = 32;                    // sorted entries per reduce work item
+
+struct Layout {
+    int passes, digit_bits, nb;
+    int64_t num_tiles, num_chunks;
+    size_t ghist, absmax, counters, tilehist_a, zero_bytes;   // zeroed at call start: [0, zero_bytes)
+    size_t tilehist_b, keys_a, keys_b, vals_a, vals_b, tile_heads, seg_start, chunk_first, long_list, partials;
+    size_t total;
+};
+
+Layout make_layout(const dqrm_ctx *ctx, int64_t L)
+{
+    Layout y;
+    y.passes = (ctx->key_bits + 8) / 9;
+    if (y.passes < 1) y.passes = 1;
+    y.digit_bits = (ctx->key_bits + y.passes - 1) / y.passes;
+    y.nb = 1 << y.digit_bits;
+    int64_t Lc = L < 1 ? 1 : L;
+    y.num_tiles = (Lc + ST_TILE - 1) / ST_TILE;
+    y.num_chunks = (Lc + SEG_CHUNK - 1) / SEG_CHUNK;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+    y.ghist = take(sizeof(u32) * MAX_PASSES * NB_MAX);
+    y.absmax = take(sizeof(u32) * ctx->T);
+    y.counters = take(sizeof(u32) * 8);
+    y.tilehist_a = take(sizeof(u32) * y.nb * y.num_tiles);
+    y.zero_bytes = o;
+    y.tilehist_b = take(sizeof(u32) * y.nb * y.num_tiles);
+    y.keys_a = take(sizeof(u32) * Lc);
+    y.keys_b = take(sizeof(u32) * Lc);
+    y.vals_a = take(sizeof(u32) * Lc);
+    y.vals_b = take(sizeof(u32) * Lc);
+    y.tile_heads = take(sizeof(u32) * y.num_tiles);
+    y.seg_start = take(sizeof(u32) * (Lc + 1));
+    y.chunk_first = take(sizeof(u32) * y.num_chunks);
+    y.long_list = take(sizeof(u32) * y.num_chunks);
+    y.partials = take(sizeof(double) * y.num_chunks * 2 * ctx->D);
+    y.total = o;
+    return y;
+}
+
+// counters[]: 0 = number of cut segments, 1 = U
+enum { CNT_LONG = 0, CNT_U = 1 };
+
+// ---------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+prepare_kernel(const int32_t *__restrict__ indices, const int32_t *__restrict__ offsets,
+               const int64_t *__restrict__ row_off, int T, int B, int64_t G, int64_t L,
+               u32 *__restrict__ keys, u32 *__restrict__ vals, u32 *__restrict__ ghist,
+               u32 *__restrict__ tilehist0, int64_t num_tiles, int passes, int digit_bits,
+               int *__restrict__ status)
+{
+    __shared__ u32 sh[MAX_PASSES * NB_MAX];
+    for (int i = threadIdx.x; i < MAX_PASSES * NB_MAX; i += blockDim.x) sh[i] = 0;
+    __syncthreads();
+    const u32 mask = (1u << digit_bits) - 1u;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        if (__ldg(offsets) != 0 || (int64_t)__ldg(offsets + G) != L) dq_report(status, DQRM_ERR_INDEX_RANGE);
+    }
+    for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < G; g += (int64_t)gridDim.x * blockDim.x) {
+        int32_t a = __ldg(offsets + g), e = __ldg(offsets + g + 1);
+        if (a < 0 || e < a || (int64_t)e > L) { dq_report(status, DQRM_ERR_INDEX_RANGE); continue; }
+        const int t = (int)(g / B);
+        const u32 payload = (u32)((g - (int64_t)t * B) * T + t);      // row of grad_out [B][T][D]
+        const int64_t r0 = __ldg(row_off + t);
+        const int64_t nrows = __ldg(row_off + t + 1) - r0;
+        for (int32_t j = a; j < e; ++j) {
+            int32_t idx = __ldg(indices + j);
+            if (idx < 0 || idx >= nrows) {
+                dq_report(status, DQRM_ERR_INDEX_RANGE);
+                idx = idx < 0 ? 0 : (int32_t)(nrows - 1);
+            }
+            const u32 key = (u32)(r0 + idx);
+            keys[j] = key;
+            vals[j] = payload;
+            for (int p = 0; p < passes; ++p) atomicAdd(&sh[p * NB_MAX + ((key >> (p * digit_bits)) & mask)], 1u);
+            atomicAdd(&tilehist0[(size_t)(key & mask) * num_tiles + j / ST_TILE], 1u);
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < MAX_PASSES * NB_MAX; i += blockDim.x)
+        if (sh[i]) atomicAdd(&ghist[i], sh[i]);
+}
+
+// one warp per digit: exclusive scan over tiles, plus the digit's global base
+__global__ void __launch_bounds__(256)
+sort_scan_kernel(u32 *__restrict__ tilehist, const u32 *__restrict__ ghist_p, int nb, int64_t num_tiles,
+                 u32 *__restrict__ next_tilehist, int64_t next_count)
+{
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = tid; i < next_count; i += nthreads) next_tilehist[i] = 0u;
+    const int b = (int)(tid >> 5);
+    const int lane = threadIdx.x & 31;
+    if (b >= nb) return;
+    u32 sum = 0;
+    for (int bb = lane; bb < b; bb += 32) sum += ghist_p[bb];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    u32 carry = sum;
+    u32 *row = tilehist + (size_t)b * num_tiles;
+    for (int64_t t0 = 0; t0 < num_tiles; t0 += 32) {
+        int64_t i = t0 + lane;
+        u32 c = i < num_tiles ? row[i] : 0u;
+        u32 incl = c;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            u32 n = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += n;
+        }
+        if (i < num_tiles) row[i] = carry + incl - c;
+        carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+}
+
+// stable scatter of one tile by one digit
+__global__ void __launch_bounds__(ST_THREADS)
+sort_scatter_kernel(const u32 *__restrict__ keys_in, const u32 *__restrict__ vals_in,
+                    u32 *__restrict__ keys_out, u32 *__restrict__ vals_out,
+                    const u32 *__restrict__ tile_offsets, u32 *__restrict__ next_tilehist,
+                    int64_t L, int shift, int nb, int next_shift, int64_t num_tiles, int *__restrict__ status)
+{
+    __shared__ u32 cnt[ST_WARPS][NB_MAX];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t tile = blockIdx.x;
+    const u32 mask = (u32)nb - 1u;
+    for (int i = threadIdx.x; i < ST_WARPS * NB_MAX; i += ST_THREADS) (&cnt[0][0])[i] = 0u;
+    __syncthreads();
+
+    u32 key[ST_ITEMS], val[ST_ITEMS], rank[ST_ITEMS];
+    const int64_t base = tile * ST_TILE + (int64_t)warp * (32 * ST_ITEMS) + lane;
+#pragma unroll
+    for (int k = 0; k < ST_ITEMS; ++k) {
+        int64_t i = base + k * 32;
+        bool valid = i < L;
+        key[k] = valid ? keys_in[i] : 0u;
+        val[k] = valid ? vals_in[i] : 0u;
+    }
+    const u32 lt = (1u << lane) - 1u;
+#pragma unroll
+    for (int k = 0; k < ST_ITEMS; ++k) {
+        bool valid = (base + k * 32) < L;
+        u32 digit = valid ? ((key[k] >> shift) & mask) : (u32)nb;      // nb = "no item"
+        u32 peers = __match_any_sync(0xffffffffu, digit);
+        int leader = __ffs(peers) - 1;
+        u32 pre = 0;
+        if (lane == leader && valid) {
+            pre = cnt[warp][digit];
+            cnt[warp][digit] = pre + __popc(peers);
+        }
+        pre = __shfl_sync(0xffffffffu, pre, leader);
+        rank[k] = pre + __popc(peers & lt);
+        __syncwarp();
+    }
+    __syncthreads();
+    // per digit: running offset over warps, starting at this tile's global offset
+    for (int b = threadIdx.x; b < nb; b += ST_THREADS) {
+        u32 run = tile_offsets[(size_t)b * num_tiles + tile];
+#pragma unroll
+        for (int w = 0; w < ST_WARPS; ++w) {
+            u32 c = cnt[w][b];
+            cnt[w][b] = run;
+            run += c;
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < ST_ITEMS; ++k) {
+        if ((base + k * 32) < L) {
+            u32 digit = (key[k] >> shift) & mask;
+            u32 pos = cnt[warp][digit] + rank[k];
+            if ((int64_t)pos < L) {
+                keys_out[pos] = key[k];
+                vals_out[pos] = val[k];
+                if (next_tilehist)
+                    atomicAdd(&next_tilehist[(size_t)((key[k] >> next_shift) & mask) * num_tiles + pos / ST_TILE], 1u);
+            } else {
+                dq_report(status, DQRM_ERR_INDEX_RANGE);   // only reachable with inconsistent offsets
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------
+// heads of the sorted key array
+__device__ __forceinline__ void load_tile_keys(const u32 *__restrict__ keys, int64_t L, int64_t i0,
+                                               u32 (&k)[ST_ITEMS], u32 &prev, int &n)
+{
+    n = (int)max((int64_t)0, min((int64_t)ST_ITEMS, L - i0));
+    prev = (i0 > 0 && i0 <= L) ? keys[i0 - 1] : 0xFFFFFFFFu;
+#pragma unroll
+    for (int e = 0; e < ST_ITEMS; ++e) k[e] = (e < n) ? keys[i0 + e] : 0u;
+}
+
+__global__ void __launch_bounds__(ST_THREADS)
+seg_count_kernel(const u32 *__restrict__ keys, int64_t L, u32 *__restrict__ tile_heads)
+{
+    __shared__ u32 wsum[ST_WARPS];
+    const int64_t i0 = (int64_t)blockIdx.x * ST_TILE + (int64_t)threadIdx.x * ST_ITEMS;
+    u32 k[ST_ITEMS], prev; int n;
+    load_tile_keys(keys, L, i0, k, prev, n);
+    u32 c = 0;
+#pragma unroll
+    for (int e = 0; e < ST_ITEMS; ++e) {
+        if (e < n) c += (i0 + e == 0 || k[e] != prev) ? 1u : 0u;
+        prev = k[e];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+    if ((threadIdx.x & 31) == 0) wsum[threadIdx.x >> 5] = c;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        u32 s = 0;
+        for (int w = 0; w < ST_WARPS; ++w) s += wsum[w];
+        tile_heads[blockIdx.x] = s;
+    }
+}
+
+__global__ void __launch_bounds__(ST_THREADS)
+seg_emit_kernel(const u32 *__restrict__ keys, int64_t L, const u32 *__restrict__ tile_heads,
+                const int64_t *__restrict__ row_off, int T,
+                u32 *__restrict__ seg_start, u32 *__restrict__ chunk_first,
+                int32_t *__restrict__ unique_rows, int32_t *__restrict__ uniq_off, u32 *__restrict__ counters)
+{
+    extern __shared__ unsigned char smem_raw[];
+    int64_t *s_off = reinterpret_cast<int64_t *>(smem_raw);   // [T+1]
+    __shared__ u32 wsum[ST_WARPS];
+    __shared__ u32 s_prefix;
+    for (int t = threadIdx.x; t <= T; t += ST_THREADS) s_off[t] = row_off[t];
+    // heads in all earlier tiles
+    u32 p = 0;
+    for (int64_t i = threadIdx.x; i < blockIdx.x; i += ST_THREADS) p += tile_heads[i];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) p += __shfl_xor_sync(0xffffffffu, p, o);
+    if ((threadIdx.x & 31) == 0) wsum[threadIdx.x >> 5] = p;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        u32 s = 0;
+        for (int w = 0; w < ST_WARPS; ++w) s += wsum[w];
+        s_prefix = s;
+    }
+    __syncthreads();
+    const u32 tile_prefix = s_prefix;
+    __syncthreads();
+
+    const int64_t i0 = (int64_t)blockIdx.x * ST_TILE + (int64_t)threadIdx.x * ST_ITEMS;
+    u32 k[ST_ITEMS], prev0; int n;
+    load_tile_keys(keys, L, i0, k, prev0, n);
+    u32 c = 0;
+    {
+        u32 prev = prev0;
+#pragma unroll
+        for (int e = 0; e < ST_ITEMS; ++e) {
+            if (e < n) c += (i0 + e == 0 || k[e] != prev) ? 1u : 0u;
+            prev = k[e];
+        }
+    }
+    // block exclusive scan of c
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    u32 incl = c;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        u32 v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    if (lane == 31) wsum[warp] = incl;
+    __syncthreads();
+    u32 woff = 0;
+    for (int w = 0; w < warp; ++w) woff += wsum[w];
+    u32 heads_before = tile_prefix + woff + incl - c;   // heads strictly before entry i0
+
+    u32 prev = prev0;
+#pragma unroll
+    for (int e = 0; e < ST_ITEMS; ++e) {
+        if (e < n) {
+            const int64_t i = i0 + e;
+            const bool head = (i == 0 || k[e] != prev);
+            if (head) {
+                const u32 u = heads_before;
+                heads_before += 1;
+                seg_start[u] = (u32)i;
+                const int t = dq_table_of(s_off, T, (int64_t)k[e]);
+                unique_rows[u] = (int32_t)((int64_t)k[e] - s_off[t]);
+                const int t_prev = (i == 0) ? -1 : dq_table_of(s_off, T, (int64_t)prev);
+                for (int tt = t_prev + 1; tt <= t; ++tt) uniq_off[tt] = (int32_t)u;
+            }
+            const u32 u_of_i = heads_before - 1;
+            if ((i % SEG_CHUNK) == 0) chunk_first[i / SEG_CHUNK] = u_of_i;
+            if (i == L - 1) {
+                const u32 U = u_of_i + 1;
+                seg_start[U] = (u32)L;
+                const int t = dq_table_of(s_off, T, (int64_t)k[e]);
+                for (int tt = t + 1; tt <= T; ++tt) uniq_off[tt] = (int32_t)U;
+                counters[CNT_U] = U;
+            }
+        }
+        prev = k[e];
+    }
+}
+
+// ---------------------------------------------------------------------------------
+template <int LPR>
+__device__ __forceinline__ u32 group_mask()
+{
+    if constexpr (LPR >= 32) {
+        return 0xffffffffu;
+    } else {
+        const int lane = threadIdx.x & 31;
+        return ((1u << LPR) - 1u) << (lane / LPR * LPR);
+    }
+}
+
+template <int LPR>
+__device__ __forceinline__ float group_max(float m)
+{
+    const u32 gm = group_mask<LPR>();
+#pragma unroll
+    for (int o = LPR / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(gm, m, o));
+    return m;
+}
+
+// per-thread tracker of the abs-max of one table at a time
+struct AbsmaxTracker {
+    int t = -1;
+    int64_t t_end = -1;
+    float m = 0.f;
+};
+
+template <int LPR>
+__device__ __forceinline__ void absmax_push(AbsmaxTracker &tr, u32 *absmax)
+{
+    // called group-uniformly
+    float m = group_max<LPR>(tr.m);
+    if ((threadIdx.x % LPR) == 0 && tr.t >= 0 && m > 0.f) atomicMax(&absmax[tr.t], __float_as_uint(m));
+    tr.m = 0.f;
+}
+
+template <int LPR>
+__device__ __forceinline__ void absmax_note(AbsmaxTracker &tr, u32 key, float m, const int64_t *s_off, int T,
+                                            u32 *absmax)
+{
+    if ((int64_t)key >= tr.t_end) {      // keys only ascend along a group's work
+        absmax_push<LPR>(tr, absmax);
+        tr.t = dq_table_of(s_off, T, (int64_t)key);
+        tr.t_end = s_off[tr.t + 1];
+    }
+    tr.m = fmaxf(tr.m, m);
+}
+
+template <int LPR, int CH>
+__global__ void __launch_bounds__(256)
+seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
+                  const u32 *__restrict__ seg_start, const u32 *__restrict__ chunk_first,
+                  const float *__restrict__ grad_out, float *__restrict__ grad_rows,
+                  double *__restrict__ partials, u32 *__restrict__ long_list, u32 *__restrict__ counters,
+                  u32 *__restrict__ absmax, const int64_t *__restrict__ row_off, int T, int D,
+                  int64_t L, int64_t G, int64_t num_chunks, int *__restrict__ status)
+{
+    extern __shared__ unsigned char smem_raw[];
+    int64_t *s_off = reinterpret_cast<int64_t *>(smem_raw);
+    for (int t = threadIdx.x; t <= T; t += blockDim.x) s_off[t] = row_off[t];
+    __syncthreads();
+
+    constexpr int BATCH = 8;
+    const int d4 = D >> 2;
+    const int lane = threadIdx.x % LPR;
+    const int64_t group = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / LPR;
+    const int64_t n_groups = (int64_t)gridDim.x * blockDim.x / LPR;
+    AbsmaxTracker tr;
+
+    for (int64_t c = group; c < num_chunks; c += n_groups) {
+        const int64_t i0 = c * SEG_CHUNK;
+        const int64_t i1 = min(i0 + (int64_t)SEG_CHUNK, L);
+        u32 u = chunk_first[c];
+        u32 cur_key = keys[i0];
+        int64_t run_start = i0;
+        double acc[CH][4];
+#pragma unroll
+        for (int ch = 0; ch < CH; ++ch) acc[ch][0] = acc[ch][1] = acc[ch][2] = acc[ch][3] = 0.0;
+
+        auto flush = [&](int64_t a, int64_t b) {
+            // run [a, b) of segment u; interior runs are whole segments by construction
+            bool begins = true, ends = true;
+            if (a == i0) begins = (seg_start[u] == (u32)a);
+            if (b == i1) ends = (seg_start[u + 1] == (u32)b);
+            if (begins && ends) {
+                float m = 0.f;
+#pragma unroll
+                for (int ch = 0; ch < CH; ++ch) {
+                    int c4 = ch * LPR + lane;
+                    if (c4 < d4) {
+                        float4 r = make_float4((float)acc[ch][0], (float)acc[ch][1], (float)acc[ch][2], (float)acc[ch][3]);
+                        *reinterpret_cast<float4 *>(grad_rows + (int64_t)u * D + 4 * c4) = r;
+                        m = fmaxf(fmaxf(m, fmaxf(fabsf(r.x), fabsf(r.y))), fmaxf(fabsf(r.z), fabsf(r.w)));
+                    }
+                }
+                absmax_note<LPR>(tr, cur_key, m, s_off, T, absmax);
+            } else {
+                const int slot = begins ? 1 : 0;
+                double *p = partials + ((size_t)c * 2 + slot) * D;
+#pragma unroll
+                for (int ch = 0; ch < CH; ++ch) {
+                    int c4 = ch * LPR + lane;
+                    if (c4 < d4) {
+                        *reinterpret_cast<double2 *>(p + 4 * c4) = make_double2(acc[ch][0], acc[ch][1]);
+                        *reinterpret_cast<double2 *>(p + 4 * c4 + 2) = make_double2(acc[ch][2], acc[ch][3]);
+                    }
+                }
+                if (begins && lane == 0) long_list[atomicAdd(&counters[CNT_LONG], 1u)] = u;
+            }
+        };
+
+        for (int64_t ib = i0; ib < i1; ib += BATCH) {
+            u32 k8[BATCH], v8[BATCH];
+#pragma unroll
+            for (int e = 0; e < BATCH; ++e) {
+                bool ok = ib + e < i1;
+                k8[e] = ok ? keys[ib + e] : 0u;
+                v8[e] = ok ? vals[ib + e] : 0u;
+                if (ok && (int64_t)v8[e] >= G) { dq_report(status, DQRM_ERR_INDEX_RANGE); v8[e] = 0u; }
+            }
+            float4 r[BATCH][CH];
+#pragma unroll
+            for (int e = 0; e < BATCH; ++e) {
+                if (ib + e < i1) {
+                    const float4 *src = reinterpret_cast<const float4 *>(grad_out + (int64_t)v8[e] * D);
+#pragma unroll
+                    for (int ch = 0; ch < CH; ++ch) {
+                        int c4 = ch * LPR + lane;
+                        if (c4 < d4) r[e][ch] = __ldg(src + c4);
+                    }
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < BATCH; ++e) {
+                if (ib + e < i1) {
+                    if (k8[e] != cur_key) {
+                        flush(run_start, ib + e);
+                        u += 1;
+                        cur_key = k8[e];
+                        run_start = ib + e;
+#pragma unroll
+                        for (int ch = 0; ch < CH; ++ch) acc[ch][0] = acc[ch][1] = acc[ch][2] = acc[ch][3] = 0.0;
+                    }
+#pragma unroll
+                    for (int ch = 0; ch < CH; ++ch) {
+                        int c4 = ch * LPR + lane;
+                        if (c4 < d4) {
+                            acc[ch][0] += (double)r[e][ch].x;
+                            acc[ch][1] += (double)r[e][ch].y;
+                            acc[ch][2] += (double)r[e][ch].z;
+                            acc[ch][3] += (double)r[e][ch].w;
+                        }
+                    }
+                }
+            }
+        }
+        flush(run_start, i1);
+    }
+    absmax_push<LPR>(tr, absmax);
+}
+
+// one warp per cut segment: SG = 32 / LPR lane groups stride over the pieces, then a
+// fixed butterfly adds the groups
+template <int LPR, int CH>
+__global__ void __launch_bounds__(256)
+seg_fixup_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ seg_start,
+                 const double *__restrict__ partials, const u32 *__restrict__ long_list,
+                 const u32 *__restrict__ counters, float *__restrict__ grad_rows, u32 *__restrict__ absmax,
+                 const int64_t *__restrict__ row_off, int T, int D)
+{
+    extern __shared__ unsigned char smem_raw[];
+    int64_t *s_off = reinterpret_cast<int64_t *>(smem_raw);
+    for (int t = threadIdx.x; t <= T; t += blockDim.x) s_off[t] = row_off[t];
+    __syncthreads();
+    constexpr int SG = 32 / LPR;
+    const int d4 = D >> 2;
+    const int wl = threadIdx.x & 31;
+    const int sub = wl / LPR, lane = wl % LPR;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const u32 count = counters[CNT_LONG];
+    for (int64_t s = warp; s < count; s += n_warps) {
+        const u32 u = long_list[s];
+        const u32 a = seg_start[u], e = seg_start[u + 1];
+        const int64_t c0 = a / SEG_CHUNK, c1 = (e - 1) / SEG_CHUNK;
+        const int64_t npieces = c1 - c0 + 1;
+        double acc[CH][4];
+#pragma unroll
+        for (int ch = 0; ch < CH; ++ch) acc[ch][0] = acc[ch][1] = acc[ch][2] = acc[ch][3] = 0.0;
+#pragma unroll 4
+        for (int64_t p = sub; p < npieces; p += SG) {
+            const double *src = partials + ((size_t)(c0 + p) * 2 + (p == 0 ? 1 : 0)) * D;
+#pragma unroll
+            for (int ch = 0; ch < CH; ++ch) {
+                int c4 = ch * LPR + lane;
+                if (c4 < d4) {
+                    double2 x = __ldcg(reinterpret_cast<const double2 *>(src + 4 * c4));
+                    double2 y = __ldcg(reinterpret_cast<const double2 *>(src + 4 * c4 + 2));
+                    acc[ch][0] += x.x; acc[ch][1] += x.y; acc[ch][2] += y.x; acc[ch][3] += y.y;
+                }
+            }
+        }
+#pragma unroll
+        for (int o = LPR; o < 32; o <<= 1) {
+#pragma unroll
+            for (int ch = 0; ch < CH; ++ch)
+#pragma unroll
+                for (int q = 0; q < 4; ++q) acc[ch][q] += __shfl_xor_sync(0xffffffffu, acc[ch][q], o);
+        }
+        float m = 0.f;
+#pragma unroll
+        for (int ch = 0; ch < CH; ++ch) {
+            int c4 = ch * LPR + lane;
+            if (c4 < d4) {
+                float4 r = make_float4((float)acc[ch][0], (float)acc[ch][1], (float)acc[ch][2], (float)acc[ch][3]);
+                if (sub == 0) *reinterpret_cast<float4 *>(grad_rows + (int64_t)u * D + 4 * c4) = r;
+                m = fmaxf(fmaxf(m, fmaxf(fabsf(r.x), fabsf(r.y))), fmaxf(fabsf(r.z), fabsf(r.w)));
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if (wl == 0 && m > 0.f) {
+            const int t = dq_table_of(s_off, T, (int64_t)keys[a]);
+            atomicMax(&absmax[t], __float_as_uint(m));
+        }
+    }
+}
+
+template <int LPR, int CH>
+int launch_reduce(dqrm_ctx *ctx, const Layout &y, char *ws, const u32 *keys, const u32 *vals,
+                  const float *grad_out, float *grad_rows, int64_t L, int64_t G, cudaStream_t st)
+{
+    const size_t smem = (size_t)(ctx->T + 1) * sizeof(int64_t);
+    const int64_t groups_per_block = 256 / LPR;
+    int64_t blocks = (y.num_chunks + groups_per_block - 1) / groups_per_block;
+    int64_t cap = (int64_t)ctx->num_sms * 8;
+    int grid = (int)(blocks < 1 ? 1 : (blocks > cap ? cap : blocks));
+    u32 *counters = reinterpret_cast<u32 *>(ws + y.counters);
+    u32 *absmax = reinterpret_cast<u32 *>(ws + y.absmax);
+    seg_reduce_kernel<LPR, CH><<<grid, 256, smem, st>>>(
+        keys, vals, reinterpret_cast<const u32 *>(ws + y.seg_start), reinterpret_cast<const u32 *>(ws + y.chunk_first),
+        grad_out, grad_rows, reinterpret_cast<double *>(ws + y.partials), reinterpret_cast<u32 *>(ws + y.long_list),
+        counters, absmax, ctx->d_row_off, ctx->T, ctx->D, L, G, y.num_chunks, ctx->d_status);
+    DQRM_CUDA_TRY(ctx, cudaGetLastError());
+    int64_t fb = (y.num_chunks + 7) / 8;      // one warp per cut segment, at most num_chunks of them
+    int fgrid = (int)(fb < 1 ? 1 : (fb > cap ? cap : fb));
+    seg_fixup_kernel<LPR, CH><<<fgrid, 256, smem, st>>>(
+        keys, reinterpret_cast<const u32 *>(ws + y.seg_start), reinterpret_cast<const double *>(ws + y.partials),
+        reinterpret_cast<const u32 *>(ws + y.long_list), counters, grad_rows, absmax, ctx->d_row_off, ctx->T, ctx->D);
+    DQRM_CUDA_TRY(ctx, cudaGetLastError());
+    return DQRM_OK;
+}
+
+}  // namespace
+
+size_t dq_bwd_ws_bytes(const dqrm_ctx *ctx, int64_t L, int64_t G)
+{
+    (void)G;
+    return make_layout(ctx, L).total;
+}
+
+int dq_launch_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, const int32_t *offsets,
+                  int32_t *unique_rows, int32_t *uniq_off, float *grad_rows, int B, int64_t L,
+                  void *ws_, size_t ws_bytes, cudaStream_t st, const u32 **absmax_bits_out)
+{
+    const Layout y = make_layout(ctx, L);
+    if (ws_bytes < y.total) return DQRM_ERR_WORKSPACE;
+    char *ws = reinterpret_cast<char *>(ws_);
+    const int64_t G = (int64_t)ctx->T * B;
+    if (absmax_bits_out) *absmax_bits_out = reinterpret_cast<const u32 *>(ws + y.absmax);
+    DQRM_CUDA_TRY(ctx, cudaMemsetAsync(ws, 0, y.zero_bytes, st));
+    if (L == 0) {
+        DQRM_CUDA_TRY(ctx, cudaMemsetAsync(uniq_off, 0, sizeof(int32_t) * (ctx->T + 1), st));
+        return DQRM_OK;
+    }
+    u32 *keys[2] = {reinterpret_cast<u32 *>(ws + y.keys_a), reinterpret_cast<u32 *>(ws + y.keys_b)};
+    u32 *vals[2] = {reinterpret_cast<u32 *>(ws + y.vals_a), reinterpret_cast<u32 *>(ws + y.vals_b)};
+    u32 *thist[2] = {reinterpret_cast<u32 *>(ws + y.tilehist_a), reinterpret_cast<u32 *>(ws + y.tilehist_b)};
+    u32 *ghist = reinterpret_cast<u32 *>(ws + y.ghist);
+    {
+        int64_t blocks = (G + 255) / 256;
+        int64_t cap = (int64_t)ctx->num_sms * 8;
+        int grid = (int)(blocks > cap ? cap : blocks);
+        prepare_kernel<<<grid, 256, 0, st>>>(indices, offsets, ctx->d_row_off, ctx->T, B, G, L, keys[0], vals[0],
+                                             ghist, thist[0], y.num_tiles, y.passes, y.digit_bits, ctx->d_status);
+        DQRM_CUDA_TRY(ctx, cudaGetLastError());
+    }
+    for (int p = 0; p < y.passes; ++p) {
+        const bool has_next = p + 1 < y.passes;
+        u32 *cur = thist[p & 1], *nxt = has_next ? thist[(p + 1) & 1] : nullptr;
+        int scan_grid = (y.nb * 32 + 255) / 256;
+        sort_scan_kernel<<<scan_grid, 256, 0, st>>>(cur, ghist + p * NB_MAX, y.nb, y.num_tiles, nxt,
+                                                    has_next ? (int64_t)y.nb * y.num_tiles : 0);
+        DQRM_CUDA_TRY(ctx, cudaGetLastError());
+        sort_scatter_kernel<<<(unsigned)y.num_tiles, ST_THREADS, 0, st>>>(
+            keys[p & 1], vals[p & 1], keys[(p + 1) & 1], vals[(p + 1) & 1], cur, nxt, L, p * y.digit_bits, y.nb,
+            (p + 1) * y.digit_bits, y.num_tiles, ctx->d_status);
+        DQRM_CUDA_TRY(ctx, cudaGetLastError());
+    }
+    const u32 *skeys = keys[y.passes & 1], *svals = vals[y.passes & 1];
+    seg_count_kernel<<<(unsigned)y.num_tiles, ST_THREADS, 0, st>>>(skeys, L, reinterpret_cast<u32 *>(ws + y.tile_heads));
+    DQRM_CUDA_TRY(ctx, cudaGetLastError());
+    seg_emit_kernel<<<(unsigned)y.num_tiles, ST_THREADS, (size_t)(ctx->T + 1) * sizeof(int64_t), st>>>(
+        skeys, L, reinterpret_cast<const u32 *>(ws + y.tile_heads), ctx->d_row_off, ctx->T,
+        reinterpret_cast<u32 *>(ws + y.seg_start), reinterpret_cast<u32 *>(ws + y.chunk_first), unique_rows, uniq_off,
+        reinterpret_cast<u32 *>(ws + y.counters));
+    DQRM_CUDA_TRY(ctx, cudaGetLastError());
+
+    const int d4 = ctx->D / 4;
+#define DQ_RED(LPR, CH) return launch_reduce<LPR, CH>(ctx, y, ws, skeys, svals, grad_out, grad_rows, L, G, st)
+    if (d4 <= 1) DQ_RED(1, 1);
+    if (d4 <= 2) DQ_RED(2, 1);
+    if (d4 <= 4) DQ_RED(4, 1);
+    if (d4 <= 8) DQ_RED(8, 1);
+    if (d4 <= 16) DQ_RED(16, 1);
+    if (d4 <= 32) DQ_RED(32, 1);
+    if (d4 <= 64) DQ_RED(32, 2);
+    if (d4 <= 128) DQ_RED(32, 4);
+    DQ_RED(32, 8);
+#undef DQ_RED
+}

@@ -1,0 +1,206 @@
+// INT8 gradient quantiser and touched-row SGD update (paper Appendix B.1): the values of
+// the sparse embedding gradient are quantised to INT8 with one scale per table, fixed
+// by the bit width and the tensor's own abs-max, and the local step is taken with the
+// dequantised gradient on the FP32 master rows (Section 3.1).
+//
+// Three variants of one row-streaming kernel share the addressing: quantise only,
+// update only (from stored codes), and quantise + update fused (the training step).
+// A group of LPR lanes owns one unique row; rows are distinct, so the read-modify-write
+// of the master rows needs no atomics.  All streams are 128-bit per lane.
+#include "common.cuh"
+
+namespace {
+
+constexpr int QU_THREADS = 256;
+enum { MODE_QUANT = 0, MODE_UPDATE = 1, MODE_FUSED = 2 };
+
+// largest t with uoff[t] <= u, skipping empty tables
+__device__ __forceinline__ int table_of_row(const int32_t *uoff, int T, int64_t u)
+{
+    int lo = 0, hi = T;
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (uoff[mid] <= u) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+__global__ void __launch_bounds__(QU_THREADS)
+absmax_kernel(const float *__restrict__ grad_rows, const int32_t *__restrict__ uniq_off, int T, int D,
+              u32 *__restrict__ absmax)
+{
+    extern __shared__ unsigned char smem_raw[];
+    int32_t *s_uoff = reinterpret_cast<int32_t *>(smem_raw);      // [T+1]
+    u32 *s_max = reinterpret_cast<u32 *>(s_uoff + (T + 1));       // [T]
+    for (int t = threadIdx.x; t <= T; t += QU_THREADS) s_uoff[t] = uniq_off[t];
+    for (int t = threadIdx.x; t < T; t += QU_THREADS) s_max[t] = 0u;
+    __syncthreads();
+    const int d4 = D >> 2;
+    const int64_t n4 = (int64_t)s_uoff[T] * d4;
+    const float4 *g4 = reinterpret_cast<const float4 *>(grad_rows);
+    int cur_t = -1;
+    int64_t cur_end4 = -1;
+    float m = 0.f;
+    for (int64_t base = (int64_t)blockIdx.x * QU_THREADS; base < n4; base += (int64_t)gridDim.x * QU_THREADS) {
+        int64_t i = base + threadIdx.x;
+        bool ok = i < n4;
+        float v = 0.f;
+        int t = cur_t;
+        if (ok) {
+            float4 x = __ldg(g4 + i);
+            v = fmaxf(fmaxf(fabsf(x.x), fabsf(x.y)), fmaxf(fabsf(x.z), fabsf(x.w)));
+            if (i >= cur_end4) {
+                t = table_of_row(s_uoff, T, i / d4);
+                cur_end4 = (int64_t)s_uoff[t + 1] * d4;
+            }
+        }
+        if (t != cur_t) {
+            if (cur_t >= 0 && m > 0.f) atomicMax(&s_max[cur_t], __float_as_uint(m));
+            cur_t = t;
+            m = 0.f;
+        }
+        m = fmaxf(m, v);
+    }
+    if (cur_t >= 0 && m > 0.f) atomicMax(&s_max[cur_t], __float_as_uint(m));
+    __syncthreads();
+    for (int t = threadIdx.x; t < T; t += QU_THREADS)
+        if (s_max[t]) atomicMax(&absmax[t], s_max[t]);
+}
+
+template <int MODE, int LPR, int CH>
+__global__ void __launch_bounds__(QU_THREADS)
+row_stream_kernel(float *__restrict__ tables, const int64_t *__restrict__ row_off,
+                  const int32_t *__restrict__ unique_rows, const int32_t *__restrict__ uniq_off,
+                  const float *__restrict__ grad_rows, const u32 *__restrict__ absmax,
+                  int8_t *__restrict__ codes, float *__restrict__ grad_scales, float lr, int T, int D)
+{
+    extern __shared__ unsigned char smem_raw[];
+    int32_t *s_uoff = reinterpret_cast<int32_t *>(smem_raw);      // [T+1]
+    for (int t = threadIdx.x; t <= T; t += QU_THREADS) s_uoff[t] = uniq_off[t];
+    __syncthreads();
+    if (MODE != MODE_UPDATE && blockIdx.x == 0) {
+        for (int t = threadIdx.x; t < T; t += QU_THREADS)
+            grad_scales[t] = dq_scale_from_absmax(__uint_as_float(absmax[t]), 8);
+    }
+    const int d4 = D >> 2;
+    const int64_t U = s_uoff[T];
+    const int lane = threadIdx.x % LPR;
+    const int64_t group = ((int64_t)blockIdx.x * QU_THREADS + threadIdx.x) / LPR;
+    const int64_t n_groups = (int64_t)gridDim.x * QU_THREADS / LPR;
+    int cur_t = -1;
+    int64_t cur_end = -1, r0 = 0;
+    float s = 1.f;
+    for (int64_t u = group; u < U; u += n_groups) {
+        if (u >= cur_end) {
+            cur_t = table_of_row(s_uoff, T, u);
+            cur_end = s_uoff[cur_t + 1];
+            if (MODE != MODE_QUANT) r0 = __ldg(row_off + cur_t);
+            s = (MODE == MODE_UPDATE) ? __ldg(grad_scales + cur_t)
+                                      : dq_scale_from_absmax(__uint_as_float(__ldg(absmax + cur_t)), 8);
+        }
+        float4 *wrow = nullptr;
+        if (MODE != MODE_QUANT) wrow = reinterpret_cast<float4 *>(tables + (r0 + __ldg(unique_rows + u)) * D);
+        int q[CH][4];
+        float4 w[CH];
+#pragma unroll
+        for (int ch = 0; ch < CH; ++ch) {
+            int c4 = ch * LPR + lane;
+            if (c4 < d4) {
+                if (MODE == MODE_UPDATE) {
+                    char4 c = *reinterpret_cast<const char4 *>(codes + u * D + 4 * c4);
+                    q[ch][0] = c.x; q[ch][1] = c.y; q[ch][2] = c.z; q[ch][3] = c.w;
+                } else {
+                    float4 g = __ldg(reinterpret_cast<const float4 *>(grad_rows + u * D) + c4);
+                    q[ch][0] = dq_code(g.x, s, -128.f, 127.f);
+                    q[ch][1] = dq_code(g.y, s, -128.f, 127.f);
+                    q[ch][2] = dq_code(g.z, s, -128.f, 127.f);
+                    q[ch][3] = dq_code(g.w, s, -128.f, 127.f);
+                }
+                if (MODE != MODE_QUANT) w[ch] = wrow[c4];
+            }
+        }
+#pragma unroll
+        for (int ch = 0; ch < CH; ++ch) {
+            int c4 = ch * LPR + lane;
+            if (c4 < d4) {
+                if (MODE != MODE_UPDATE) {
+                    char4 c = make_char4((signed char)q[ch][0], (signed char)q[ch][1], (signed char)q[ch][2],
+                                         (signed char)q[ch][3]);
+                    *reinterpret_cast<char4 *>(codes + u * D + 4 * c4) = c;
+                }
+                if (MODE != MODE_QUANT) {
+                    float4 x = w[ch];
+                    x.x = __fsub_rn(x.x, __fmul_rn(lr, dq_dequant(q[ch][0], s)));
+                    x.y = __fsub_rn(x.y, __fmul_rn(lr, dq_dequant(q[ch][1], s)));
+                    x.z = __fsub_rn(x.z, __fmul_rn(lr, dq_dequant(q[ch][2], s)));
+                    x.w = __fsub_rn(x.w, __fmul_rn(lr, dq_dequant(q[ch][3], s)));
+                    wrow[c4] = x;
+                }
+            }
+        }
+    }
+}
+
+template <int MODE, int LPR, int CH>
+int launch_rows(dqrm_ctx *ctx, float *tables, const int32_t *unique_rows, const int32_t *uniq_off,
+                const float *grad_rows, const u32 *absmax, int8_t *codes, float *grad_scales, float lr,
+                cudaStream_t st)
+{
+    const size_t smem = (size_t)(ctx->T + 1) * sizeof(int32_t);
+    int grid = ctx->num_sms * 8;      // U lives on the device: persistent grid-stride
+    row_stream_kernel<MODE, LPR, CH><<<grid, QU_THREADS, smem, st>>>(tables, ctx->d_row_off, unique_rows, uniq_off,
+                                                                     grad_rows, absmax, codes, grad_scales, lr,
+                                                                     ctx->T, ctx->D);
+    DQRM_CUDA_TRY(ctx, cudaGetLastError());
+    return DQRM_OK;
+}
+
+template <int MODE>
+int dispatch(dqrm_ctx *ctx, float *tables, const int32_t *unique_rows, const int32_t *uniq_off,
+             const float *grad_rows, const u32 *absmax, int8_t *codes, float *grad_scales, float lr,
+             cudaStream_t st)
+{
+    const int d4 = ctx->D / 4;
+#define DQ_ROWS(LPR, CH) \
+    return launch_rows<MODE, LPR, CH>(ctx, tables, unique_rows, uniq_off, grad_rows, absmax, codes, grad_scales, lr, st)
+    if (d4 <= 1) DQ_ROWS(1, 1);
+    if (d4 <= 2) DQ_ROWS(2, 1);
+    if (d4 <= 4) DQ_ROWS(4, 1);
+    if (d4 <= 8) DQ_ROWS(8, 1);
+    if (d4 <= 16) DQ_ROWS(16, 1);
+    if (d4 <= 32) DQ_ROWS(32, 1);
+    if (d4 <= 64) DQ_ROWS(32, 2);
+    if (d4 <= 128) DQ_ROWS(32, 4);
+    DQ_ROWS(32, 8);
+#undef DQ_ROWS
+}
+
+}  // namespace
+
+size_t dq_quant_ws_bytes(const dqrm_ctx *ctx) { return align_up(sizeof(u32) * ctx->T, 256); }
+
+int dq_launch_grad_quant(dqrm_ctx *ctx, const float *grad_rows, const int32_t *uniq_off, int8_t *codes,
+                         float *grad_scales, void *ws, size_t ws_bytes, cudaStream_t st)
+{
+    if (ws_bytes < dq_quant_ws_bytes(ctx)) return DQRM_ERR_WORKSPACE;
+    u32 *absmax = reinterpret_cast<u32 *>(ws);
+    DQRM_CUDA_TRY(ctx, cudaMemsetAsync(absmax, 0, sizeof(u32) * ctx->T, st));
+    const size_t smem = (size_t)(ctx->T + 1) * sizeof(int32_t) + (size_t)ctx->T * sizeof(u32);
+    absmax_kernel<<<ctx->num_sms * 8, QU_THREADS, smem, st>>>(grad_rows, uniq_off, ctx->T, ctx->D, absmax);
+    DQRM_CUDA_TRY(ctx, cudaGetLastError());
+    return dispatch<MODE_QUANT>(ctx, nullptr, nullptr, uniq_off, grad_rows, absmax, codes, grad_scales, 0.f, st);
+}
+
+int dq_launch_row_update(dqrm_ctx *ctx, float *tables, const int32_t *unique_rows, const int32_t *uniq_off,
+                         const int8_t *codes, const float *grad_scales, float lr, cudaStream_t st)
+{
+    return dispatch<MODE_UPDATE>(ctx, tables, unique_rows, uniq_off, nullptr, nullptr, const_cast<int8_t *>(codes),
+                                 const_cast<float *>(grad_scales), lr, st);
+}
+
+int dq_launch_quant_update(dqrm_ctx *ctx, float *tables, const int32_t *unique_rows, const int32_t *uniq_off,
+                           const float *grad_rows, const u32 *absmax_bits, int8_t *codes, float *grad_scales,
+                           float lr, cudaStream_t st)
+{
+    return dispatch<MODE_FUSED>(ctx, tables, unique_rows, uniq_off, grad_rows, absmax_bits, codes, grad_scales, lr, st);
+}

@@ -1,0 +1,152 @@
+"""GPU parity: every call of the C ABI against the CPU oracle on the same seeded inputs.
+
+Bars: integer outputs (weight codes, gradient codes, unique rows, offsets) and scales are
+bit-exact; FP32 sums (pooled outputs, summed gradients) are within 1e-5 relative / 1e-6
+absolute; the update, fed identical inputs, is bit-exact."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+
+from dqrm_inputs import workloads as W
+from gpu_util import Case, assert_close_fp32, bit_equal
+
+pytestmark = pytest.mark.gpu
+
+
+def _cases():
+    kg = W.kaggle()
+    tb = W.terabyte()
+    mh = W.multihot()
+    return {
+        "tiny": W.tiny(),
+        # 26 tables, feature 16, 53,248 lookups = 26 sort tiles, the last one ragged
+        "kaggle_small": W.scaled_down(kg, total_rows=300_000, B=2048, name="kaggle_small"),
+        # feature 64, 26 * 1500 = 39,000 lookups: ragged tile and ragged 32-entry chunk
+        "terabyte_small": W.scaled_down(tb, total_rows=400_000, B=1500, name="terabyte_small"),
+        # multi-hot, duplicate heavy (Zipf 1.2 over 3000 rows, ~20 per bag)
+        "multihot_small": W.scaled_down(mh, total_rows=26 * 3000, B=300, name="multihot_small"),
+        "sweep_d16_b2_uniform": W.sweep(D=16, bits=2, zipf=False, rows=200_000, B=5000),
+        "sweep_d32_b4_zipf": W.sweep(D=32, bits=4, zipf=True, rows=200_000, B=5000),
+        "sweep_d64_b8_uniform": W.sweep(D=64, bits=8, zipf=False, rows=100_000, B=3000),
+        "sweep_d128_b8_zipf": W.sweep(D=128, bits=8, zipf=True, rows=50_000, B=3000),
+        # feature sizes that are not a power of two / need several vectors per lane
+        "odd_d20": replace(W.scaled_down(kg, total_rows=50_000, B=333), D=20, name="odd_d20"),
+        "wide_d384": W.Workload("wide_d384", (700, 90, 5000), D=384, B=257, alpha=1.1, bits=8),
+        "one_row_tables": W.Workload("one_row_tables", (1, 1, 7, 1), D=16, B=100, alpha=1.05, bits=4),
+    }
+
+
+CASES = _cases()
+
+
+@pytest.fixture(scope="module", params=sorted(CASES))
+def case(request):
+    c = Case(CASES[request.param])
+    c.tables_np = W.tables_np(c.wl)
+    yield c
+    c.ctx.close()
+
+
+def test_scale_refresh_bit_exact(case, oracle):
+    d_tables = case.dev(case.tables_np)
+    scales, minmax = case.gpu_refresh(d_tables)
+    o_scales, o_minmax = oracle.scale_refresh(case.tables_np, case.row_off, case.wl.D, case.bits_np)
+    assert bit_equal(scales.cpu().numpy(), o_scales)
+    assert (minmax.cpu().numpy() == o_minmax).all()
+
+
+def test_scale_refresh_extreme_positions(case, oracle):
+    # plant the extreme at the first / last element of each table and mid-arena
+    tables = case.tables_np.copy()
+    off = case.row_off
+    rng = np.random.default_rng(5)
+    for t in range(case.wl.T):
+        flat = tables[off[t]:off[t + 1]].reshape(-1)
+        pos = [0, flat.size - 1, int(rng.integers(flat.size))][t % 3]
+        flat[pos] = (-1) ** t * (3.0 + t)
+    scales, minmax = case.gpu_refresh(case.dev(tables))
+    o_scales, o_minmax = oracle.scale_refresh(tables, off, case.wl.D, case.bits_np)
+    assert bit_equal(scales.cpu().numpy(), o_scales)
+    assert (minmax.cpu().numpy() == o_minmax).all()
+
+
+@pytest.mark.parametrize("step", [0, 1])
+def test_forward(case, oracle, step):
+    idx, off, _ = case.batch(step)
+    o_scales, _ = oracle.scale_refresh(case.tables_np, case.row_off, case.wl.D, case.bits_np)
+    if step == 1:
+        o_scales = (o_scales * np.float32(0.37)).astype(np.float32)   # stale scale: clamp is live
+    want_codes = case.wl.bits <= 8
+    out, codes = case.gpu_fwd(case.dev(case.tables_np), idx, off, case.dev(o_scales), want_codes)
+    if want_codes:
+        o_out, o_codes = oracle.emb_fwd(case.tables_np, case.row_off, case.wl.D, case.wl.B, idx, off, o_scales,
+                                        case.bits_np, want_codes=True)
+        assert bit_equal(codes, o_codes)
+    else:
+        o_out = oracle.emb_fwd(case.tables_np, case.row_off, case.wl.D, case.wl.B, idx, off, o_scales, case.bits_np)
+    assert_close_fp32(out, o_out, "pooled output")
+    # same order, same FP64 accumulator: expected to agree to the bit
+    assert bit_equal(out, o_out)
+
+
+@pytest.mark.parametrize("step", [0, 2])
+def test_backward(case, oracle, step):
+    idx, off, go = case.batch(step)
+    ur, uo, gr = case.gpu_bwd(idx, off, go)
+    o_ur, o_uo, o_gr = oracle.emb_bwd(go, case.wl.T, case.wl.D, case.wl.B, idx, off)
+    assert bit_equal(uo, o_uo)
+    assert bit_equal(ur, o_ur)
+    assert_close_fp32(gr, o_gr, "summed gradients")
+    # determinism: a second run gives the same bits
+    ur2, uo2, gr2 = case.gpu_bwd(idx, off, go)
+    assert bit_equal(gr, gr2) and bit_equal(ur, ur2) and bit_equal(uo, uo2)
+    # FP64 accumulation makes the rounded sums equal the oracle's except for double-rounding ties
+    mism = int((gr.view(np.int32) != o_gr.view(np.int32)).sum())
+    assert mism <= max(1, gr.size // 100_000), f"{mism} of {gr.size} summed gradients differ in the last bit"
+
+
+def test_grad_quant_and_update_bit_exact(case, oracle):
+    idx, off, go = case.batch(3)
+    o_ur, o_uo, o_gr = oracle.emb_bwd(go, case.wl.T, case.wl.D, case.wl.B, idx, off)
+    codes, gs = case.gpu_quant(o_gr, o_uo)
+    o_codes, o_gs = oracle.grad_quant_int8(o_gr, o_uo, case.wl.D)
+    assert bit_equal(gs, o_gs)
+    assert bit_equal(codes, o_codes)
+    d_tables = case.dev(case.tables_np)
+    case.gpu_update(d_tables, o_ur, o_uo, o_codes, o_gs, case.wl.lr)
+    o_tables = case.tables_np.copy()
+    oracle.row_update(o_tables, case.row_off, case.wl.D, o_ur, o_uo, o_codes, o_gs, case.wl.lr)
+    assert bit_equal(d_tables.cpu().numpy(), o_tables)
+
+
+def test_train_step_equals_separate_calls_and_oracle(case, oracle):
+    import torch
+
+    wl = case.wl
+    idx, off, go = case.batch(4)
+    L = len(idx)
+    o_tables = case.tables_np.copy()
+    o_scales, _ = oracle.scale_refresh(o_tables, case.row_off, wl.D, case.bits_np)
+    r = oracle.train_step(o_tables, case.row_off, wl.D, wl.B, idx, off, go, o_scales, case.bits_np, wl.lr)
+    d_tables = case.dev(case.tables_np)
+    out = case.empty((wl.B, wl.T, wl.D), torch.float32)
+    ur = case.empty(max(L, 1), torch.int32)
+    uo = case.empty(wl.T + 1, torch.int32)
+    gr = case.empty((max(L, 1), wl.D), torch.float32)
+    codes = case.empty((max(L, 1), wl.D), torch.int8)
+    gs = case.empty(wl.T, torch.float32)
+    case.ctx.train_step(d_tables, case.dev(idx), case.dev(off), case.dev(go), case.dev(o_scales), case.bits, out,
+                        ur, uo, gr, codes, gs, wl.lr, B=wl.B, L=L)
+    case.ctx.raise_on_device_error()
+    U = int(r["uniq_off"][-1])
+    assert bit_equal(uo.cpu().numpy(), r["uniq_off"])
+    assert bit_equal(ur.cpu().numpy()[:U], r["unique_rows"])
+    assert bit_equal(out.cpu().numpy(), r["out"])
+    assert_close_fp32(gr.cpu().numpy()[:U], r["grad_rows"])
+    if bit_equal(gr.cpu().numpy()[:U], r["grad_rows"]):
+        assert bit_equal(gs.cpu().numpy(), r["grad_scales"])
+        assert bit_equal(codes.cpu().numpy()[:U], r["codes"])
+        assert bit_equal(d_tables.cpu().numpy(), o_tables)
+    else:
+        assert_close_fp32(d_tables.cpu().numpy(), o_tables, "updated weights")
