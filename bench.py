@@ -1,0 +1,381 @@
+#!/usr/bin/env python
+"""Benchmark of the QAT embedding step (forward + backward + INT8 gradient quantisation +
+touched-row update, scale refresh every `period` steps) on synthetic Criteo-shaped data.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+Prints ONE JSON line.  `value` is whole-job lookups/s with inputs resident in HBM,
+`e2e` the same through the host-buffer entry point (copies inside the timed region),
+`roofline` the dominant kernel against the measured HBM copy rate, `cpu_baseline` the
+CPU oracle timed on the host cores.  With --impl reference the oracle itself is timed.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "QAT embedding lookups/sec (fwd+bwd+update)"
+UNIT = "lookups/s"
+N_BATCHES = 16
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def get_workload(name):
+    from dqrm_inputs import workloads as W
+
+    if name in W.BY_NAME:
+        return W.BY_NAME[name]()
+    if name == "kaggle_smoke":      # small stand-in used by the tests of this script
+        return W.scaled_down(W.kaggle(), total_rows=200_000, B=1024, name="kaggle_smoke")
+    raise SystemExit(f"unknown workload {name}; choose from {sorted(W.BY_NAME)}")
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def algorithmic_bytes(wl, L, G, U):
+    """Bytes the method must move per call (each touched row once)."""
+    D = wl.D
+    fwd = 4 * L + 4 * G + 4 * D * U + 4 * D * G
+    bwd = 4 * D * G + 4 * L + 4 * G + 4 * U + 4 * D * U
+    qu = 4 * D * U + D * U + 4 * U + 8 * D * U          # read grads, write codes, read rows, RMW rows
+    return {"fwd": fwd, "bwd": bwd, "quant_update": qu, "step": fwd + bwd + qu,
+            "refresh": wl.table_bytes()}
+
+
+# kernel -> which algorithmic byte count bounds it (the sort kernels carry no algorithmic
+# bytes of their own: they are implementation cost of the backward)
+KERNEL_BYTES = {
+    "fwd_kernel": lambda ab, wl, L, G, U: ab["fwd"],
+    "seg_reduce_kernel": lambda ab, wl, L, G, U: 4 * wl.D * G + 4 * wl.D * U,
+    "row_stream_kernel<fused>": lambda ab, wl, L, G, U: ab["quant_update"],
+    "refresh_kernel": lambda ab, wl, L, G, U: ab["refresh"],
+}
+
+
+def oracle_sample(wl, tables_h, n_steps, period):
+    """Times the CPU oracle, as it stands, on `n_steps` full batches and one refresh."""
+    import numpy as np
+    import oracle
+    from dqrm_inputs import workloads as W
+
+    off = wl.row_off()
+    bits = np.full(wl.T, wl.bits, dtype=np.int32)
+    samplers = W.make_samplers(wl)
+    t0 = time.perf_counter()
+    scales, _ = oracle.scale_refresh(tables_h, off, wl.D, bits)
+    t_refresh = time.perf_counter() - t0
+    t_steps, lookups = 0.0, 0
+    for s in range(n_steps):
+        idx, offs = W.make_batch(wl, s, samplers)
+        go = W.grad_out_np(wl, s)
+        t0 = time.perf_counter()
+        oracle.train_step(tables_h, off, wl.D, wl.B, idx, offs, go, scales, bits, wl.lr)
+        t_steps += time.perf_counter() - t0
+        lookups += len(idx)
+    per_step = t_steps / n_steps + t_refresh / period
+    return (lookups / n_steps) / per_step, t_steps / n_steps, t_refresh
+
+
+def host_tables(wl):
+    import torch
+    from dqrm_inputs import workloads as W
+
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    return W.tables_torch(wl, dev).cpu().numpy()
+
+
+def run_reference(args):
+    """The oracle on the host cores, timed step by step (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import numpy as np
+    import oracle
+    from dqrm_inputs import workloads as W
+
+    oracle.build()
+    wl = get_workload(args.workload)
+    tables_h = host_tables(wl)
+    off = wl.row_off()
+    bits = np.full(wl.T, wl.bits, dtype=np.int32)
+    samplers = W.make_samplers(wl)
+    t0 = time.perf_counter()
+    scales, _ = oracle.scale_refresh(tables_h, off, wl.D, bits)
+    t_refresh = time.perf_counter() - t0
+    batches = [(*W.make_batch(wl, s, samplers), W.grad_out_np(wl, s)) for s in range(min(4, args.warmup + args.steps))]
+    for s in range(args.warmup):
+        idx, offs, go = batches[s % len(batches)]
+        oracle.train_step(tables_h, off, wl.D, wl.B, idx, offs, go, scales, bits, wl.lr)
+    t0 = time.perf_counter()
+    lookups = 0
+    for s in range(args.steps):
+        idx, offs, go = batches[s % len(batches)]
+        oracle.train_step(tables_h, off, wl.D, wl.B, idx, offs, go, scales, bits, wl.lr)
+        lookups += len(idx)
+    dt = time.perf_counter() - t0 + args.steps * t_refresh / wl.period
+    value = lookups / dt
+    sample = (f"{args.steps} full steps of batch {wl.B} (fwd+bwd+int8 quant+update) plus one whole-table "
+              f"refresh of {wl.table_bytes() / 1e9:.2f} GB charged at 1/{wl.period} per step")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "tables": wl.T, "dim": wl.D, "batch": wl.B, "bits": wl.bits,
+                   "refresh_period": wl.period},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    import paper_2410_20046_b200 as dq
+    from dqrm_inputs import workloads as W
+    from paper_2410_20046_b200 import harness
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dq.load_library()
+
+    wl = get_workload(args.workload)
+    G = wl.T * wl.B
+    tables = W.tables_torch(wl, "cuda")
+    tables_h = tables.cpu().numpy() if (rank == 0 and world == 1 and not args.no_cpu_baseline) else None
+
+    # every rank is a full replica that takes its own B samples (weak scaling, no exchange)
+    samplers = W.make_samplers(wl)
+    batches = []
+    for b in range(N_BATCHES):
+        step_id = harness.batch_id(b, rank, world, N_BATCHES)
+        idx, offs = W.make_batch(wl, step_id, samplers)
+        offs_h = offs
+        U = sum(len(np.unique(idx[offs_h[t * wl.B]:offs_h[(t + 1) * wl.B]])) for t in range(wl.T))
+        batches.append(dict(L=len(idx), U=U, idx_h=torch.from_numpy(idx).pin_memory(),
+                            off_h=torch.from_numpy(offs).pin_memory(),
+                            go=W.grad_out_torch(wl, step_id, "cuda")))
+    for b in batches:
+        b["idx"], b["off"] = b["idx_h"].cuda(), b["off_h"].cuda()
+        b["go_h"] = b["go"].cpu().pin_memory()
+    Lmax = max(b["L"] for b in batches)
+    Lavg = sum(b["L"] for b in batches) / N_BATCHES
+    Uavg = sum(b["U"] for b in batches) / N_BATCHES
+
+    ctx = dq.Context(wl.row_off(), wl.D, Lmax, G, host_step=True)
+    bits = torch.full((wl.T,), wl.bits, dtype=torch.int32, device="cuda")
+    scales = torch.empty(wl.T, dtype=torch.float32, device="cuda")
+    out = torch.empty((wl.B, wl.T, wl.D), dtype=torch.float32, device="cuda")
+    out_h = torch.empty((wl.B, wl.T, wl.D), dtype=torch.float32).pin_memory()
+    ur = torch.empty(Lmax, dtype=torch.int32, device="cuda")
+    uo = torch.empty(wl.T + 1, dtype=torch.int32, device="cuda")
+    gr = torch.empty((Lmax, wl.D), dtype=torch.float32, device="cuda")
+    codes = torch.empty((Lmax, wl.D), dtype=torch.int8, device="cuda")
+    gs = torch.empty(wl.T, dtype=torch.float32, device="cuda")
+
+    def step(s):
+        if s % wl.period == 0:
+            ctx.scale_refresh(tables, bits, scales)
+        b = batches[s % N_BATCHES]
+        ctx.train_step(tables, b["idx"], b["off"], b["go"], scales, bits, out, ur, uo, gr, codes, gs, wl.lr,
+                       B=wl.B, L=b["L"])
+
+    def step_host(s):
+        if s % wl.period == 0:
+            ctx.scale_refresh(tables, bits, scales)
+        b = batches[s % N_BATCHES]
+        ctx.train_step_host(tables, b["idx_h"], b["off_h"], b["go_h"], scales, bits, out_h, wl.lr, B=wl.B, L=b["L"])
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(fn, steps, warmup, sample_clocks=False):
+        for s in range(warmup):
+            fn(s)
+        sync_all()
+        sampler = ClockSampler(local_rank) if (sample_clocks and rank == 0) else None
+        if sampler:
+            sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n0 = ctx.launch_count()
+        e0.record()
+        for s in range(steps):
+            fn(warmup + s)
+        e1.record()
+        sync_all()
+        ms = e0.elapsed_time(e1)
+        clocks = sampler.stop() if sampler else None
+        launches = ctx.launch_count() - n0
+        ms = harness.max_over_ranks(ms, device="cuda")
+        return ms, clocks, launches
+
+    warm = max(3, args.warmup)
+    ms, clocks, launches = timed(step, args.steps, warm, sample_clocks=True)
+    ctx.raise_on_device_error()
+    lookups_per_step = Lavg * world
+    value = harness.job_throughput(Lavg, world, args.steps, ms)
+
+    e2e_steps = max(3, min(args.steps, args.e2e_steps))
+    ms_e2e, _, _ = timed(step_host, e2e_steps, 3)
+    ctx.raise_on_device_error()
+    e2e_value = lookups_per_step * e2e_steps / (ms_e2e * 1e-3)
+    h2d = int(4 * Lavg + 4 * (G + 1) + 4 * G * wl.D)
+    d2h = int(4 * G * wl.D)
+
+    # per-kernel times: a second pass over the same steps with an event after every launch
+    prof_steps = min(args.steps, 200)
+    for s in range(3):
+        step(s)
+    torch.cuda.synchronize()
+    ctx.profile_begin()
+    for s in range(prof_steps):
+        step(warm + s)
+    prof = ctx.profile_end()
+    total_prof_ms = sum(v[0] for v in prof.values())
+    kernels = {k: {"launches": v[1], "ms_total": round(v[0], 4), "us_per_launch": round(1e3 * v[0] / v[1], 3),
+                   "share": round(v[0] / total_prof_ms, 4)} for k, v in sorted(prof.items(), key=lambda kv: -kv[1][0])}
+
+    peak, peak_kind = measured_peak()
+    ab = algorithmic_bytes(wl, Lavg, G, Uavg)
+    dominant = max((k for k in prof if k in KERNEL_BYTES), key=lambda k: prof[k][0])
+    dom_bytes = KERNEL_BYTES[dominant](ab, wl, Lavg, G, Uavg)
+    dom_s = prof[dominant][0] * 1e-3 / prof[dominant][1]
+    achieved = dom_bytes / dom_s / 1e9
+    per_kernel_roofline = {}
+    for k in prof:
+        if k in KERNEL_BYTES:
+            by = KERNEL_BYTES[k](ab, wl, Lavg, G, Uavg)
+            gbs = by / (prof[k][0] * 1e-3 / prof[k][1]) / 1e9
+            per_kernel_roofline[k] = {"algorithmic_bytes": int(by), "GB/s": round(gbs, 1),
+                                      "frac_of_" + peak_kind: round(gbs / peak, 4)}
+    step_bytes = ab["step"] + ab["refresh"] / wl.period
+    step_gbs = step_bytes * world / (ms * 1e-3 / args.steps) / 1e9
+
+    cpu_baseline = None
+    if tables_h is not None:
+        n = 2 if wl.table_bytes() > 1e9 else 3
+        v, t_step, t_ref = oracle_sample(wl, tables_h, n, wl.period)
+        cpu_baseline = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
+                        "sample": (f"{n} full steps of batch {wl.B} ({t_step * 1e3:.0f} ms each) plus one whole-table "
+                                   f"refresh ({t_ref * 1e3:.0f} ms) charged at 1/{wl.period} per step")}
+
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": warm, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": wl.name, "tables": wl.T, "dim": wl.D, "batch_per_gpu": wl.B,
+                       "lookups_per_step_per_gpu": Lavg, "unique_rows_per_step": Uavg, "unique_fraction": Uavg / Lavg,
+                       "bits": wl.bits, "grad_bits": 8, "refresh_period": wl.period, "table_bytes": wl.table_bytes(),
+                       "parallelism": f"{world} replica(s), batch sharded by sample, no exchange",
+                       "l2": f"{N_BATCHES} distinct pre-staged batches cycled; their rows, gradients and outputs "
+                             f"exceed the 126 MB L2 and the table is {wl.table_bytes() / 1e9:.2f} GB"},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+            "roofline": {"bound": "hbm", "kernel": dominant, "achieved": round(achieved, 1), "peak": peak,
+                         "peak_kind": peak_kind, "unit": "GB/s", "frac": round(achieved / peak, 4),
+                         "frac_of_8TBps_nominal": round(achieved / NOMINAL_HBM_GBS, 4), "traffic": None,
+                         "algorithmic_bytes_per_launch": int(dom_bytes)},
+            "step_roofline": {"algorithmic_bytes_per_step": int(step_bytes), "GB/s": round(step_gbs, 1),
+                              "frac_of_" + peak_kind: round(step_gbs / peak / world, 4),
+                              "frac_of_8TBps_nominal": round(step_gbs / NOMINAL_HBM_GBS / world, 4)},
+            "kernel_rooflines": per_kernel_roofline,
+            "kernels": kernels,
+            "cpu_baseline": cpu_baseline,
+        }))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="kaggle_b16384")
+    ap.add_argument("--e2e-steps", type=int, default=50)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

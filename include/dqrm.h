@@ -168,6 +168,24 @@ int dqrm_train_step_host(dqrm_ctx *ctx, float *tables, const int32_t *h_indices,
                          float lr, int B, int64_t L,
                          void *workspace, size_t workspace_bytes, void *stream);
 
+/* ---- launch accounting and timing aid (no counterpart in the paper) ----------------
+ * dqrm_launch_count: kernels this context has launched since it was created (memsets
+ * and copies are not counted).
+ * dqrm_profile_begin / dqrm_profile_end: between the two, every launch of this context
+ * is followed by a cudaEvent on its stream; _end synchronises the stream and returns,
+ * per kernel id (0 .. dqrm_kernel_count()-1), the summed milliseconds between the event
+ * before and the event after its launches, and the number of launches.  Both arrays are
+ * HOST arrays of at least dqrm_kernel_count() entries.  At most 4096 launches are
+ * recorded per begin/end pair; later ones are counted but not timed.  Event recording
+ * perturbs back-to-back launches slightly, so headline timings are taken with profiling
+ * off.  dqrm_kernel_name gives the kernel's name for an id. */
+int64_t dqrm_launch_count(const dqrm_ctx *ctx);
+int dqrm_profile_begin(dqrm_ctx *ctx, void *stream);
+int dqrm_profile_end(dqrm_ctx *ctx, void *stream, float *h_ms_per_kernel,
+                     int32_t *h_launches_per_kernel, int n);
+const char *dqrm_kernel_name(int kernel_id);
+int dqrm_kernel_count(void);
+
 #ifdef __cplusplus
 }
 #endif

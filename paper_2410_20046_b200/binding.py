@@ -38,6 +38,11 @@ SIGNATURES = {
                              _vp, _sz, _vp]),
     "dqrm_host_step_workspace_bytes": (_sz, [_vp, _i64, _i64]),
     "dqrm_train_step_host": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _f, _i, _i64, _vp, _sz, _vp]),
+    "dqrm_launch_count": (_i64, [_vp]),
+    "dqrm_profile_begin": (_i, [_vp, _vp]),
+    "dqrm_profile_end": (_i, [_vp, _vp, ctypes.POINTER(_f), ctypes.POINTER(ctypes.c_int32), _i]),
+    "dqrm_kernel_name": (ctypes.c_char_p, [_i]),
+    "dqrm_kernel_count": (_i, []),
 }
 
 _lib = None
@@ -145,6 +150,20 @@ class Context:
 
     def raise_on_device_error(self, stream=None):
         self._check("dqrm_check_status", self.check_status(stream))
+
+    def launch_count(self) -> int:
+        return int(self.lib.dqrm_launch_count(self._h))
+
+    def profile_begin(self, stream=None):
+        self._check("dqrm_profile_begin", self.lib.dqrm_profile_begin(self._h, _stream(stream)))
+
+    def profile_end(self, stream=None):
+        """-> {kernel name: (milliseconds, launches)} for the launches since profile_begin"""
+        n = int(self.lib.dqrm_kernel_count())
+        ms = (_f * n)()
+        cnt = (ctypes.c_int32 * n)()
+        self._check("dqrm_profile_end", self.lib.dqrm_profile_end(self._h, _stream(stream), ms, cnt, n))
+        return {self.lib.dqrm_kernel_name(k).decode(): (float(ms[k]), int(cnt[k])) for k in range(n) if cnt[k]}
 
     # ---- the calls of include/dqrm.h ----
     def scale_refresh(self, tables, bits, scales, minmax=None, stream=None):

@@ -93,6 +93,11 @@ int dqrm_destroy(dqrm_ctx *ctx)
     if (ctx->d_status) cudaFree(ctx->d_status);
     if (ctx->d_done) cudaFree(ctx->d_done);
     if (ctx->h_status_pinned) cudaFreeHost(ctx->h_status_pinned);
+    if (ctx->prof_events) {
+        for (int i = 0; i < DQ_PROF_MAX; ++i) cudaEventDestroy(ctx->prof_events[i]);
+        delete[] ctx->prof_events;
+    }
+    delete[] ctx->prof_ids;
     delete[] ctx->h_row_off;
     delete ctx;
     return DQRM_OK;
@@ -123,6 +128,53 @@ int dqrm_check_status(dqrm_ctx *ctx, void *stream)
 }
 
 int dqrm_last_cuda_error(const dqrm_ctx *ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+int64_t dqrm_launch_count(const dqrm_ctx *ctx) { return ctx ? ctx->launch_count : 0; }
+
+int dqrm_profile_begin(dqrm_ctx *ctx, void *stream)
+{
+    if (!ctx) return DQRM_ERR_INVALID_ARG;
+    if (!ctx->prof_events) {
+        ctx->prof_events = new (std::nothrow) cudaEvent_t[DQ_PROF_MAX];
+        ctx->prof_ids = new (std::nothrow) int[DQ_PROF_MAX];
+        if (!ctx->prof_events || !ctx->prof_ids) return DQRM_ERR_INVALID_ARG;
+        for (int i = 0; i < DQ_PROF_MAX; ++i) DQRM_CUDA_TRY(ctx, cudaEventCreate(&ctx->prof_events[i]));
+    }
+    ctx->prof_n = 0;
+    ctx->prof_on = 1;
+    dq_mark(ctx, as_stream(stream), DQ_K_BEGIN);
+    return DQRM_OK;
+}
+
+int dqrm_profile_end(dqrm_ctx *ctx, void *stream, float *h_ms_per_kernel, int32_t *h_launches_per_kernel, int n)
+{
+    if (!ctx || !h_ms_per_kernel || !h_launches_per_kernel || n < DQ_K_COUNT) return DQRM_ERR_INVALID_ARG;
+    ctx->prof_on = 0;
+    DQRM_CUDA_TRY(ctx, cudaStreamSynchronize(as_stream(stream)));
+    for (int k = 0; k < n; ++k) { h_ms_per_kernel[k] = 0.f; h_launches_per_kernel[k] = 0; }
+    for (int i = 1; i < ctx->prof_n; ++i) {
+        float ms = 0.f;
+        DQRM_CUDA_TRY(ctx, cudaEventElapsedTime(&ms, ctx->prof_events[i - 1], ctx->prof_events[i]));
+        const int id = ctx->prof_ids[i];
+        if (id == DQ_K_BEGIN) continue;          // a gap between profiled calls, not a launch
+        h_ms_per_kernel[id] += ms;
+        h_launches_per_kernel[id] += 1;
+    }
+    ctx->prof_n = 0;
+    return DQRM_OK;
+}
+
+const char *dqrm_kernel_name(int kernel_id)
+{
+    static const char *names[DQ_K_COUNT] = {
+        "begin", "refresh_kernel", "fwd_kernel", "memset", "prepare_kernel", "sort_scan_kernel",
+        "sort_scatter_kernel", "seg_count_kernel", "seg_emit_kernel", "seg_reduce_kernel", "seg_fixup_kernel",
+        "absmax_kernel", "row_stream_kernel<quant>", "row_stream_kernel<update>", "row_stream_kernel<fused>",
+        "copy"};
+    return (kernel_id >= 0 && kernel_id < DQ_K_COUNT) ? names[kernel_id] : "?";
+}
+
+int dqrm_kernel_count(void) { return DQ_K_COUNT; }
 
 const char *dqrm_status_string(int status)
 {
@@ -192,6 +244,7 @@ int dqrm_train_step(dqrm_ctx *ctx, float *tables, const int32_t *indices, const 
     if (L > 0 && (!indices || !unique_rows || !grad_rows || !codes)) return DQRM_ERR_INVALID_ARG;
     if (!ws_ok(workspace, workspace_bytes, dq_bwd_ws_bytes(ctx, L, (int64_t)ctx->T * B))) return DQRM_ERR_WORKSPACE;
     cudaStream_t st = as_stream(stream);
+    if (ctx->prof_on) dq_mark(ctx, st, DQ_K_BEGIN);
     int rc = dq_launch_fwd(ctx, tables, indices, offsets, scales, bits, out, nullptr, B, L, st);
     if (rc != DQRM_OK) return rc;
     const u32 *absmax = nullptr;

@@ -574,12 +574,14 @@ int launch_reduce(dqrm_ctx *ctx, const Layout &y, char *ws, const u32 *keys, con
         grad_out, grad_rows, reinterpret_cast<double *>(ws + y.partials), reinterpret_cast<u32 *>(ws + y.long_list),
         counters, absmax, ctx->d_row_off, ctx->T, ctx->D, L, G, y.num_chunks, ctx->d_status);
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
+    dq_mark(ctx, st, DQ_K_SEG_REDUCE);
     int64_t fb = (y.num_chunks + 7) / 8;      // one warp per cut segment, at most num_chunks of them
     int fgrid = (int)(fb < 1 ? 1 : (fb > cap ? cap : fb));
     seg_fixup_kernel<LPR, CH><<<fgrid, 256, smem, st>>>(
         keys, reinterpret_cast<const u32 *>(ws + y.seg_start), reinterpret_cast<const double *>(ws + y.partials),
         reinterpret_cast<const u32 *>(ws + y.long_list), counters, grad_rows, absmax, ctx->d_row_off, ctx->T, ctx->D);
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
+    dq_mark(ctx, st, DQ_K_SEG_FIXUP);
     return DQRM_OK;
 }
 
@@ -601,6 +603,7 @@ int dq_launch_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, 
     const int64_t G = (int64_t)ctx->T * B;
     if (absmax_bits_out) *absmax_bits_out = reinterpret_cast<const u32 *>(ws + y.absmax);
     DQRM_CUDA_TRY(ctx, cudaMemsetAsync(ws, 0, y.zero_bytes, st));
+    dq_mark(ctx, st, DQ_K_MEMSET);
     if (L == 0) {
         DQRM_CUDA_TRY(ctx, cudaMemsetAsync(uniq_off, 0, sizeof(int32_t) * (ctx->T + 1), st));
         return DQRM_OK;
@@ -616,6 +619,7 @@ int dq_launch_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, 
         prepare_kernel<<<grid, 256, 0, st>>>(indices, offsets, ctx->d_row_off, ctx->T, B, G, L, keys[0], vals[0],
                                              ghist, thist[0], y.num_tiles, y.passes, y.digit_bits, ctx->d_status);
         DQRM_CUDA_TRY(ctx, cudaGetLastError());
+        dq_mark(ctx, st, DQ_K_PREPARE);
     }
     for (int p = 0; p < y.passes; ++p) {
         const bool has_next = p + 1 < y.passes;
@@ -624,19 +628,23 @@ int dq_launch_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, 
         sort_scan_kernel<<<scan_grid, 256, 0, st>>>(cur, ghist + p * NB_MAX, y.nb, y.num_tiles, nxt,
                                                     has_next ? (int64_t)y.nb * y.num_tiles : 0);
         DQRM_CUDA_TRY(ctx, cudaGetLastError());
+        dq_mark(ctx, st, DQ_K_SORT_SCAN);
         sort_scatter_kernel<<<(unsigned)y.num_tiles, ST_THREADS, 0, st>>>(
             keys[p & 1], vals[p & 1], keys[(p + 1) & 1], vals[(p + 1) & 1], cur, nxt, L, p * y.digit_bits, y.nb,
             (p + 1) * y.digit_bits, y.num_tiles, ctx->d_status);
         DQRM_CUDA_TRY(ctx, cudaGetLastError());
+        dq_mark(ctx, st, DQ_K_SORT_SCATTER);
     }
     const u32 *skeys = keys[y.passes & 1], *svals = vals[y.passes & 1];
     seg_count_kernel<<<(unsigned)y.num_tiles, ST_THREADS, 0, st>>>(skeys, L, reinterpret_cast<u32 *>(ws + y.tile_heads));
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
+    dq_mark(ctx, st, DQ_K_SEG_COUNT);
     seg_emit_kernel<<<(unsigned)y.num_tiles, ST_THREADS, (size_t)(ctx->T + 1) * sizeof(int64_t), st>>>(
         skeys, L, reinterpret_cast<const u32 *>(ws + y.tile_heads), ctx->d_row_off, ctx->T,
         reinterpret_cast<u32 *>(ws + y.seg_start), reinterpret_cast<u32 *>(ws + y.chunk_first), unique_rows, uniq_off,
         reinterpret_cast<u32 *>(ws + y.counters));
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
+    dq_mark(ctx, st, DQ_K_SEG_EMIT);
 
     const int d4 = ctx->D / 4;
 #define DQ_RED(LPR, CH) return launch_reduce<LPR, CH>(ctx, y, ws, skeys, svals, grad_out, grad_rows, L, G, st)

@@ -19,7 +19,30 @@ struct dqrm_ctx {
     int device = 0;
     int num_sms = 0;
     int key_bits = 1;               // bits of an arena row number
+    // launch accounting and optional per-launch timing (see dqrm_profile_*)
+    int64_t launch_count = 0;
+    int prof_on = 0, prof_n = 0;
+    cudaEvent_t *prof_events = nullptr;   // [DQ_PROF_MAX]
+    int *prof_ids = nullptr;              // [DQ_PROF_MAX] kernel id that ENDS at event i
 };
+
+enum {
+    DQ_K_BEGIN = 0, DQ_K_REFRESH, DQ_K_FWD, DQ_K_MEMSET, DQ_K_PREPARE, DQ_K_SORT_SCAN, DQ_K_SORT_SCATTER,
+    DQ_K_SEG_COUNT, DQ_K_SEG_EMIT, DQ_K_SEG_REDUCE, DQ_K_SEG_FIXUP, DQ_K_ABSMAX, DQ_K_QUANT, DQ_K_UPDATE,
+    DQ_K_QUANT_UPDATE, DQ_K_COPY, DQ_K_COUNT
+};
+constexpr int DQ_PROF_MAX = 4096;
+
+// called right after every launch: counts it and, when profiling is on, drops an event
+static inline void dq_mark(dqrm_ctx *ctx, cudaStream_t st, int kernel_id)
+{
+    if (kernel_id != DQ_K_BEGIN && kernel_id != DQ_K_MEMSET && kernel_id != DQ_K_COPY) ctx->launch_count++;
+    if (ctx->prof_on && ctx->prof_n < DQ_PROF_MAX) {
+        ctx->prof_ids[ctx->prof_n] = kernel_id;
+        cudaEventRecord(ctx->prof_events[ctx->prof_n], st);
+        ctx->prof_n++;
+    }
+}
 
 #define DQRM_CUDA_TRY(ctx, call)                                   \
     do {                                                           \

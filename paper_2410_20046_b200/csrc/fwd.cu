@@ -137,6 +137,7 @@ int launch(dqrm_ctx *ctx, const float *tables, const int32_t *indices, const int
     fwd_kernel<LPR, CH, NB><<<grid, FW_THREADS, 0, st>>>(tables, ctx->d_row_off, indices, offsets, scales, bits,
                                                          out, codes_out, ctx->T, ctx->D, B, G, L, ctx->d_status);
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
+    dq_mark(ctx, st, DQ_K_FWD);
     return DQRM_OK;
 }
 

@@ -152,6 +152,7 @@ int launch_rows(dqrm_ctx *ctx, float *tables, const int32_t *unique_rows, const 
                                                                      grad_rows, absmax, codes, grad_scales, lr,
                                                                      ctx->T, ctx->D);
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
+    dq_mark(ctx, st, MODE == MODE_QUANT ? DQ_K_QUANT : (MODE == MODE_UPDATE ? DQ_K_UPDATE : DQ_K_QUANT_UPDATE));
     return DQRM_OK;
 }
 
@@ -186,8 +187,10 @@ int dq_launch_grad_quant(dqrm_ctx *ctx, const float *grad_rows, const int32_t *u
     u32 *absmax = reinterpret_cast<u32 *>(ws);
     DQRM_CUDA_TRY(ctx, cudaMemsetAsync(absmax, 0, sizeof(u32) * ctx->T, st));
     const size_t smem = (size_t)(ctx->T + 1) * sizeof(int32_t) + (size_t)ctx->T * sizeof(u32);
+    dq_mark(ctx, st, DQ_K_MEMSET);
     absmax_kernel<<<ctx->num_sms * 8, QU_THREADS, smem, st>>>(grad_rows, uniq_off, ctx->T, ctx->D, absmax);
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
+    dq_mark(ctx, st, DQ_K_ABSMAX);
     return dispatch<MODE_QUANT>(ctx, nullptr, nullptr, uniq_off, grad_rows, absmax, codes, grad_scales, 0.f, st);
 }
 

@@ -147,5 +147,6 @@ int dq_launch_refresh(dqrm_ctx *ctx, const float *tables, const int32_t *bits, f
                                                    ctx->T, ctx->D, n4, bits, scales, minmax,
                                                    reinterpret_cast<u32 *>(ws), ctx->d_done);
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
+    dq_mark(ctx, st, DQ_K_REFRESH);
     return DQRM_OK;
 }
