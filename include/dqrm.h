@@ -61,6 +61,7 @@ extern "C" {
 #define DQRM_ERR_CUDA          (-3)  /* a CUDA runtime call failed; see dqrm_last_cuda_error */
 #define DQRM_ERR_INDEX_RANGE   (-4)  /* device saw an index outside [0, R_t) or a bad offset */
 #define DQRM_ERR_TIMEOUT       (-5)  /* reserved: a bounded device-side wait ran out */
+#define DQRM_ERR_STATIC_LIMIT  (-6)  /* size exceeds the built-in scratch of a *_static call */
 
 typedef struct dqrm_ctx dqrm_ctx;
 
@@ -167,6 +168,29 @@ int dqrm_train_step_host(dqrm_ctx *ctx, float *tables, const int32_t *h_indices,
                          const float *scales, const int32_t *bits, float *h_out,
                          float lr, int B, int64_t L,
                          void *workspace, size_t workspace_bytes, void *stream);
+
+/* ---- allocation-free gradient quantiser (the paper has no counterpart) -------------
+ * Same result as dqrm_grad_quant_int8, for callers that must not allocate device memory
+ * when they quantise: code that runs inside a host framework which has already claimed
+ * the GPU's memory for its own pool, or a serving / real-time loop that cannot afford the
+ * device-wide synchronisation a cudaMalloc or cudaFree implies.  It needs no context and
+ * no workspace: T and D are passed directly, and the per-table abs-max scratch lives in a
+ * fixed array inside the library image (DQRM_STATIC_MAX_TABLES 32-bit words = 4 KB, held
+ * by every GPU that loads the library until the process exits).  The call performs no
+ * cudaMalloc / cudaFree and uses no allocating library routine.
+ *   T            number of tables, 1 .. DQRM_STATIC_MAX_TABLES; larger T returns
+ *                DQRM_ERR_STATIC_LIMIT and launches nothing
+ *   D            feature size, multiple of 4, 4 .. 1024
+ *   grad_rows in [U][D], uniq_off in [T+1], codes out [U][D] int8, grad_scales out [T]
+ *                (device pointers, caller-owned, as for dqrm_grad_quant_int8)
+ * The first call on each device looks up the array's device address (the device that is
+ * current at the call is used); make that first call outside any stream capture.
+ * All calls on a device share the one array, which still holds the previous call's maxima:
+ * each call clears the T entries it uses on `stream` before its kernels run.  Two calls
+ * that can overlap on the GPU (different streams, no dependency) race on it; order them. */
+#define DQRM_STATIC_MAX_TABLES 1024
+int dqrm_grad_quant_int8_static(int T, int D, const float *grad_rows, const int32_t *uniq_off,
+                                int8_t *codes, float *grad_scales, void *stream);
 
 /* ---- launch accounting and timing aid (no counterpart in the paper) ----------------
  * dqrm_launch_count: kernels this context has launched since it was created (memsets

@@ -8,5 +8,6 @@ There is no CPU fallback: importing the binding without the built library raises
 """
 from .binding import (  # noqa: F401
     DqrmError, Context, load_library, LIB_PATH,
-    OK, ERR_INVALID_ARG, ERR_WORKSPACE, ERR_CUDA, ERR_INDEX_RANGE, ERR_TIMEOUT,
+    OK, ERR_INVALID_ARG, ERR_WORKSPACE, ERR_CUDA, ERR_INDEX_RANGE, ERR_TIMEOUT, ERR_STATIC_LIMIT,
+    STATIC_MAX_TABLES, grad_quant_int8_static,
 )

@@ -14,6 +14,8 @@ ERR_WORKSPACE = -2
 ERR_CUDA = -3
 ERR_INDEX_RANGE = -4
 ERR_TIMEOUT = -5
+ERR_STATIC_LIMIT = -6
+STATIC_MAX_TABLES = 1024
 
 _vp = ctypes.c_void_p
 _i = ctypes.c_int
@@ -38,6 +40,7 @@ SIGNATURES = {
                              _vp, _sz, _vp]),
     "dqrm_host_step_workspace_bytes": (_sz, [_vp, _i64, _i64]),
     "dqrm_train_step_host": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _f, _i, _i64, _vp, _sz, _vp]),
+    "dqrm_grad_quant_int8_static": (_i, [_i, _i, _vp, _vp, _vp, _vp, _vp]),
     "dqrm_launch_count": (_i64, [_vp]),
     "dqrm_profile_begin": (_i, [_vp, _vp]),
     "dqrm_profile_end": (_i, [_vp, _vp, ctypes.POINTER(_f), ctypes.POINTER(ctypes.c_int32), _i]),
@@ -224,3 +227,16 @@ class Context:
             _ptr(h_offsets, torch.int32, "cpu"), _ptr(h_grad_out, torch.float32, "cpu"),
             _ptr(scales, torch.float32), _ptr(bits, torch.int32), _ptr(h_out, torch.float32, "cpu"),
             float(lr), int(B), int(L), self._hws_ptr, self.host_workspace_bytes, _stream(stream)))
+
+
+def grad_quant_int8_static(T, D, grad_rows, uniq_off, codes, grad_scales, stream=None) -> int:
+    """``dqrm_grad_quant_int8_static``: the gradient quantiser for callers that must not
+    allocate device memory (no context, no workspace; scratch is a fixed array inside the
+    library).  Returns the status code instead of raising, so that the size limit can be
+    handled by the caller."""
+    import torch
+
+    lib = load_library()
+    return int(lib.dqrm_grad_quant_int8_static(
+        int(T), int(D), _ptr(grad_rows, torch.float32), _ptr(uniq_off, torch.int32), _ptr(codes, torch.int8),
+        _ptr(grad_scales, torch.float32), _stream(stream)))

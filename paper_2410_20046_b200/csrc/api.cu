@@ -185,6 +185,7 @@ const char *dqrm_status_string(int status)
     case DQRM_ERR_CUDA: return "CUDA runtime error";
     case DQRM_ERR_INDEX_RANGE: return "index or offset out of range (detected on the device)";
     case DQRM_ERR_TIMEOUT: return "bounded device-side wait ran out";
+    case DQRM_ERR_STATIC_LIMIT: return "size exceeds the built-in scratch of an allocation-free call";
     default: return "unknown status";
     }
 }

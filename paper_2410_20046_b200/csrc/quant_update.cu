@@ -207,3 +207,73 @@ int dq_launch_quant_update(dqrm_ctx *ctx, float *tables, const int32_t *unique_r
 {
     return dispatch<MODE_FUSED>(ctx, tables, unique_rows, uniq_off, grad_rows, absmax_bits, codes, grad_scales, lr, st);
 }
+
+// ---------------------------------------------------------------------------------
+// Allocation-free variant of the INT8 gradient quantiser.
+//
+// Some users of this library may not allocate device memory at the point where they
+// quantise gradients: a plug-in that runs inside another framework's step after that
+// framework has reserved the whole HBM for its own pool (a cudaMalloc there fails or
+// fragments the pool), or a latency-critical loop in which the implicit device-wide
+// synchronisation of cudaMalloc/cudaFree would stall every other stream.  Such callers
+// have no way to provide the per-table abs-max scratch word that dqrm_grad_quant_int8
+// takes from its workspace, and they cannot create a context either (dqrm_create
+// allocates).  For them the scratch lives in the array below, which is part of the
+// loaded module: every GPU that loads the library holds these 4 KB until the process
+// exits.  The name `g_static_absmax` is only a handle in host code; the device address
+// is looked up once per device with cudaGetSymbolAddress and cached.
+// ---------------------------------------------------------------------------------
+static __device__ __align__(256) u32 g_static_absmax[DQRM_STATIC_MAX_TABLES];
+
+namespace {
+
+constexpr int STATIC_MAX_DEVICES = 64;
+struct StaticSlot {
+    u32 *absmax = nullptr;   // device address of g_static_absmax on this device
+    int num_sms = 0;
+    bool ready = false;
+};
+StaticSlot g_static_slots[STATIC_MAX_DEVICES];
+
+}  // namespace
+
+extern "C" int dqrm_grad_quant_int8_static(int T, int D, const float *grad_rows, const int32_t *uniq_off,
+                                           int8_t *codes, float *grad_scales, void *stream)
+{
+    if (T <= 0 || D < 4 || D > 1024 || (D % 4) != 0 || !grad_rows || !uniq_off || !codes || !grad_scales)
+        return DQRM_ERR_INVALID_ARG;
+    if (T > DQRM_STATIC_MAX_TABLES) return DQRM_ERR_STATIC_LIMIT;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= STATIC_MAX_DEVICES) {
+        (void)cudaGetLastError();
+        return DQRM_ERR_CUDA;
+    }
+    StaticSlot &slot = g_static_slots[dev];
+    if (!slot.ready) {
+        // first call on this device: resolve the array's device address (with this device current)
+        u32 *p = nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void **>(&p), g_static_absmax) != cudaSuccess || !p ||
+            cudaDeviceGetAttribute(&slot.num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return DQRM_ERR_CUDA;
+        }
+        slot.absmax = p;
+        slot.ready = true;
+    }
+    // a stack context carries the shape to the shared launch helpers; nothing is allocated
+    dqrm_ctx tmp;
+    tmp.T = T;
+    tmp.D = D;
+    tmp.device = dev;
+    tmp.num_sms = slot.num_sms;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    // the array keeps the previous call's maxima: clear the entries this call uses
+    if (cudaMemsetAsync(slot.absmax, 0, sizeof(u32) * T, st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return DQRM_ERR_CUDA;
+    }
+    const size_t smem = (size_t)(T + 1) * sizeof(int32_t) + (size_t)T * sizeof(u32);
+    absmax_kernel<<<tmp.num_sms * 8, QU_THREADS, smem, st>>>(grad_rows, uniq_off, T, D, slot.absmax);
+    if (cudaGetLastError() != cudaSuccess) return DQRM_ERR_CUDA;
+    return dispatch<MODE_QUANT>(&tmp, nullptr, nullptr, uniq_off, grad_rows, slot.absmax, codes, grad_scales, 0.f, st);
+}
