@@ -192,6 +192,16 @@ int dqrm_train_step_host(dqrm_ctx *ctx, float *tables, const int32_t *h_indices,
 int dqrm_grad_quant_int8_static(int T, int D, const float *grad_rows, const int32_t *uniq_off,
                                 int8_t *codes, float *grad_scales, void *stream);
 
+/* ---- quantiser self-check (no counterpart in the paper) ----------------------------
+ * The kernels evaluate Q(x; s, b) without the IEEE division sequence where a scale is
+ * shared by many elements, and fall back to the division near rounding ties.  This call
+ * compares that evaluation with the plain definition clamp(round_half_even(x / s)) for
+ * the `count` FP32 bit patterns first_bits, first_bits+1, ... (count <= 2^32, wrapping)
+ * and ADDS the number of disagreements to *mismatches (device uint64, caller-zeroed).
+ * NaN patterns are skipped.  Expected result: 0 for every scale and bit width. */
+int dqrm_selfcheck_quantizer(dqrm_ctx *ctx, float scale, int bits, uint32_t first_bits, uint64_t count,
+                             uint64_t *mismatches, void *stream);
+
 /* ---- launch accounting and timing aid (no counterpart in the paper) ----------------
  * dqrm_launch_count: kernels this context has launched since it was created (memsets
  * and copies are not counted).

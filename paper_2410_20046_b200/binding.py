@@ -41,6 +41,7 @@ SIGNATURES = {
     "dqrm_host_step_workspace_bytes": (_sz, [_vp, _i64, _i64]),
     "dqrm_train_step_host": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _f, _i, _i64, _vp, _sz, _vp]),
     "dqrm_grad_quant_int8_static": (_i, [_i, _i, _vp, _vp, _vp, _vp, _vp]),
+    "dqrm_selfcheck_quantizer": (_i, [_vp, _f, _i, ctypes.c_uint32, ctypes.c_uint64, _vp, _vp]),
     "dqrm_launch_count": (_i64, [_vp]),
     "dqrm_profile_begin": (_i, [_vp, _vp]),
     "dqrm_profile_end": (_i, [_vp, _vp, ctypes.POINTER(_f), ctypes.POINTER(ctypes.c_int32), _i]),
@@ -153,6 +154,13 @@ class Context:
 
     def raise_on_device_error(self, stream=None):
         self._check("dqrm_check_status", self.check_status(stream))
+
+    def selfcheck_quantizer(self, scale, bits, first_bits, count, mismatches, stream=None):
+        import torch
+
+        self._check("dqrm_selfcheck_quantizer", self.lib.dqrm_selfcheck_quantizer(
+            self._h, float(scale), int(bits), int(first_bits) & 0xFFFFFFFF, int(count),
+            _ptr(mismatches, torch.int64), _stream(stream)))
 
     def launch_count(self) -> int:
         return int(self.lib.dqrm_launch_count(self._h))

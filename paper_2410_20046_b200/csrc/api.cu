@@ -170,7 +170,7 @@ const char *dqrm_kernel_name(int kernel_id)
         "begin", "refresh_kernel", "fwd_kernel", "memset", "prepare_kernel", "sort_scan_kernel",
         "sort_scatter_kernel", "seg_count_kernel", "seg_emit_kernel", "seg_reduce_kernel", "seg_fixup_kernel",
         "absmax_kernel", "row_stream_kernel<quant>", "row_stream_kernel<update>", "row_stream_kernel<fused>",
-        "copy"};
+        "copy", "seg_fixup_big_kernel"};
     return (kernel_id >= 0 && kernel_id < DQ_K_COUNT) ? names[kernel_id] : "?";
 }
 

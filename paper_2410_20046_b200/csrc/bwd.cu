@@ -20,6 +20,7 @@
 // for bit.  The per-table abs-max of the summed gradient (needed by the INT8 gradient
 // quantiser) is folded into the last two kernels.
 #include "common.cuh"
+#include "seg_reduce.cuh"
 
 namespace {
 
@@ -29,7 +30,7 @@ constexpr int ST_TILE = ST_THREADS * ST_ITEMS;   // 2048 entries per tile
 constexpr int ST_WARPS = ST_THREADS / 32;
 constexpr int NB_MAX = 512;                      // bins per pass (<= 9 bit digits)
 constexpr int MAX_PASSES = 4;
-constexpr int SEG_CHUNK = 32;                    // sorted entries per reduce work item
+constexpr int SEG_CHUNK = segred::CHUNK;         // sorted entries per reduce work item
 
 struct Layout {
     int passes, digit_bits, nb;
@@ -70,8 +71,8 @@ Layout make_layout(const dqrm_ctx *ctx, int64_t L)
     return y;
 }
 
-// counters[]: 0 = number of cut segments, 1 = U
-enum { CNT_LONG = 0, CNT_U = 1 };
+// counters[]: see segred::CNT_*
+using segred::CNT_U;
 
 // ---------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
@@ -330,258 +331,47 @@ seg_emit_kernel(const u32 *__restrict__ keys, int64_t L, const u32 *__restrict__
 }
 
 // ---------------------------------------------------------------------------------
-template <int LPR>
-__device__ __forceinline__ u32 group_mask()
-{
-    if constexpr (LPR >= 32) {
-        return 0xffffffffu;
-    } else {
-        const int lane = threadIdx.x & 31;
-        return ((1u << LPR) - 1u) << (lane / LPR * LPR);
-    }
-}
-
-template <int LPR>
-__device__ __forceinline__ float group_max(float m)
-{
-    const u32 gm = group_mask<LPR>();
-#pragma unroll
-    for (int o = LPR / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(gm, m, o));
-    return m;
-}
-
-// per-thread tracker of the abs-max of one table at a time
-struct AbsmaxTracker {
-    int t = -1;
-    int64_t t_end = -1;
-    float m = 0.f;
-};
-
-template <int LPR>
-__device__ __forceinline__ void absmax_push(AbsmaxTracker &tr, u32 *absmax)
-{
-    // called group-uniformly
-    float m = group_max<LPR>(tr.m);
-    if ((threadIdx.x % LPR) == 0 && tr.t >= 0 && m > 0.f) atomicMax(&absmax[tr.t], __float_as_uint(m));
-    tr.m = 0.f;
-}
-
-template <int LPR>
-__device__ __forceinline__ void absmax_note(AbsmaxTracker &tr, u32 key, float m, const int64_t *s_off, int T,
-                                            u32 *absmax)
-{
-    if ((int64_t)key >= tr.t_end) {      // keys only ascend along a group's work
-        absmax_push<LPR>(tr, absmax);
-        tr.t = dq_table_of(s_off, T, (int64_t)key);
-        tr.t_end = s_off[tr.t + 1];
-    }
-    tr.m = fmaxf(tr.m, m);
-}
-
-template <int LPR, int CH>
-__global__ void __launch_bounds__(256)
-seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
-                  const u32 *__restrict__ seg_start, const u32 *__restrict__ chunk_first,
-                  const float *__restrict__ grad_out, float *__restrict__ grad_rows,
-                  double *__restrict__ partials, u32 *__restrict__ long_list, u32 *__restrict__ counters,
-                  u32 *__restrict__ absmax, const int64_t *__restrict__ row_off, int T, int D,
-                  int64_t L, int64_t G, int64_t num_chunks, int *__restrict__ status)
-{
-    extern __shared__ unsigned char smem_raw[];
-    int64_t *s_off = reinterpret_cast<int64_t *>(smem_raw);
-    for (int t = threadIdx.x; t <= T; t += blockDim.x) s_off[t] = row_off[t];
-    __syncthreads();
-
-    constexpr int BATCH = 8;
-    const int d4 = D >> 2;
-    const int lane = threadIdx.x % LPR;
-    const int64_t group = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / LPR;
-    const int64_t n_groups = (int64_t)gridDim.x * blockDim.x / LPR;
-    AbsmaxTracker tr;
-
-    for (int64_t c = group; c < num_chunks; c += n_groups) {
-        const int64_t i0 = c * SEG_CHUNK;
-        const int64_t i1 = min(i0 + (int64_t)SEG_CHUNK, L);
-        u32 u = chunk_first[c];
-        u32 cur_key = keys[i0];
-        int64_t run_start = i0;
-        double acc[CH][4];
-#pragma unroll
-        for (int ch = 0; ch < CH; ++ch) acc[ch][0] = acc[ch][1] = acc[ch][2] = acc[ch][3] = 0.0;
-
-        auto flush = [&](int64_t a, int64_t b) {
-            // run [a, b) of segment u; interior runs are whole segments by construction
-            bool begins = true, ends = true;
-            if (a == i0) begins = (seg_start[u] == (u32)a);
-            if (b == i1) ends = (seg_start[u + 1] == (u32)b);
-            if (begins && ends) {
-                float m = 0.f;
-#pragma unroll
-                for (int ch = 0; ch < CH; ++ch) {
-                    int c4 = ch * LPR + lane;
-                    if (c4 < d4) {
-                        float4 r = make_float4((float)acc[ch][0], (float)acc[ch][1], (float)acc[ch][2], (float)acc[ch][3]);
-                        *reinterpret_cast<float4 *>(grad_rows + (int64_t)u * D + 4 * c4) = r;
-                        m = fmaxf(fmaxf(m, fmaxf(fabsf(r.x), fabsf(r.y))), fmaxf(fabsf(r.z), fabsf(r.w)));
-                    }
-                }
-                absmax_note<LPR>(tr, cur_key, m, s_off, T, absmax);
-            } else {
-                const int slot = begins ? 1 : 0;
-                double *p = partials + ((size_t)c * 2 + slot) * D;
-#pragma unroll
-                for (int ch = 0; ch < CH; ++ch) {
-                    int c4 = ch * LPR + lane;
-                    if (c4 < d4) {
-                        *reinterpret_cast<double2 *>(p + 4 * c4) = make_double2(acc[ch][0], acc[ch][1]);
-                        *reinterpret_cast<double2 *>(p + 4 * c4 + 2) = make_double2(acc[ch][2], acc[ch][3]);
-                    }
-                }
-                if (begins && lane == 0) long_list[atomicAdd(&counters[CNT_LONG], 1u)] = u;
-            }
-        };
-
-        for (int64_t ib = i0; ib < i1; ib += BATCH) {
-            u32 k8[BATCH], v8[BATCH];
-#pragma unroll
-            for (int e = 0; e < BATCH; ++e) {
-                bool ok = ib + e < i1;
-                k8[e] = ok ? keys[ib + e] : 0u;
-                v8[e] = ok ? vals[ib + e] : 0u;
-                if (ok && (int64_t)v8[e] >= G) { dq_report(status, DQRM_ERR_INDEX_RANGE); v8[e] = 0u; }
-            }
-            float4 r[BATCH][CH];
-#pragma unroll
-            for (int e = 0; e < BATCH; ++e) {
-                if (ib + e < i1) {
-                    const float4 *src = reinterpret_cast<const float4 *>(grad_out + (int64_t)v8[e] * D);
-#pragma unroll
-                    for (int ch = 0; ch < CH; ++ch) {
-                        int c4 = ch * LPR + lane;
-                        if (c4 < d4) r[e][ch] = __ldg(src + c4);
-                    }
-                }
-            }
-#pragma unroll
-            for (int e = 0; e < BATCH; ++e) {
-                if (ib + e < i1) {
-                    if (k8[e] != cur_key) {
-                        flush(run_start, ib + e);
-                        u += 1;
-                        cur_key = k8[e];
-                        run_start = ib + e;
-#pragma unroll
-                        for (int ch = 0; ch < CH; ++ch) acc[ch][0] = acc[ch][1] = acc[ch][2] = acc[ch][3] = 0.0;
-                    }
-#pragma unroll
-                    for (int ch = 0; ch < CH; ++ch) {
-                        int c4 = ch * LPR + lane;
-                        if (c4 < d4) {
-                            acc[ch][0] += (double)r[e][ch].x;
-                            acc[ch][1] += (double)r[e][ch].y;
-                            acc[ch][2] += (double)r[e][ch].z;
-                            acc[ch][3] += (double)r[e][ch].w;
-                        }
-                    }
-                }
-            }
-        }
-        flush(run_start, i1);
-    }
-    absmax_push<LPR>(tr, absmax);
-}
-
-// one warp per cut segment: SG = 32 / LPR lane groups stride over the pieces, then a
-// fixed butterfly adds the groups
-template <int LPR, int CH>
-__global__ void __launch_bounds__(256)
-seg_fixup_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ seg_start,
-                 const double *__restrict__ partials, const u32 *__restrict__ long_list,
-                 const u32 *__restrict__ counters, float *__restrict__ grad_rows, u32 *__restrict__ absmax,
-                 const int64_t *__restrict__ row_off, int T, int D)
-{
-    extern __shared__ unsigned char smem_raw[];
-    int64_t *s_off = reinterpret_cast<int64_t *>(smem_raw);
-    for (int t = threadIdx.x; t <= T; t += blockDim.x) s_off[t] = row_off[t];
-    __syncthreads();
-    constexpr int SG = 32 / LPR;
-    const int d4 = D >> 2;
-    const int wl = threadIdx.x & 31;
-    const int sub = wl / LPR, lane = wl % LPR;
-    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
-    const u32 count = counters[CNT_LONG];
-    for (int64_t s = warp; s < count; s += n_warps) {
-        const u32 u = long_list[s];
-        const u32 a = seg_start[u], e = seg_start[u + 1];
-        const int64_t c0 = a / SEG_CHUNK, c1 = (e - 1) / SEG_CHUNK;
-        const int64_t npieces = c1 - c0 + 1;
-        double acc[CH][4];
-#pragma unroll
-        for (int ch = 0; ch < CH; ++ch) acc[ch][0] = acc[ch][1] = acc[ch][2] = acc[ch][3] = 0.0;
-#pragma unroll 4
-        for (int64_t p = sub; p < npieces; p += SG) {
-            const double *src = partials + ((size_t)(c0 + p) * 2 + (p == 0 ? 1 : 0)) * D;
-#pragma unroll
-            for (int ch = 0; ch < CH; ++ch) {
-                int c4 = ch * LPR + lane;
-                if (c4 < d4) {
-                    double2 x = __ldcg(reinterpret_cast<const double2 *>(src + 4 * c4));
-                    double2 y = __ldcg(reinterpret_cast<const double2 *>(src + 4 * c4 + 2));
-                    acc[ch][0] += x.x; acc[ch][1] += x.y; acc[ch][2] += y.x; acc[ch][3] += y.y;
-                }
-            }
-        }
-#pragma unroll
-        for (int o = LPR; o < 32; o <<= 1) {
-#pragma unroll
-            for (int ch = 0; ch < CH; ++ch)
-#pragma unroll
-                for (int q = 0; q < 4; ++q) acc[ch][q] += __shfl_xor_sync(0xffffffffu, acc[ch][q], o);
-        }
-        float m = 0.f;
-#pragma unroll
-        for (int ch = 0; ch < CH; ++ch) {
-            int c4 = ch * LPR + lane;
-            if (c4 < d4) {
-                float4 r = make_float4((float)acc[ch][0], (float)acc[ch][1], (float)acc[ch][2], (float)acc[ch][3]);
-                if (sub == 0) *reinterpret_cast<float4 *>(grad_rows + (int64_t)u * D + 4 * c4) = r;
-                m = fmaxf(fmaxf(m, fmaxf(fabsf(r.x), fabsf(r.y))), fmaxf(fabsf(r.z), fabsf(r.w)));
-            }
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-        if (wl == 0 && m > 0.f) {
-            const int t = dq_table_of(s_off, T, (int64_t)keys[a]);
-            atomicMax(&absmax[t], __float_as_uint(m));
-        }
-    }
-}
-
 template <int LPR, int CH>
 int launch_reduce(dqrm_ctx *ctx, const Layout &y, char *ws, const u32 *keys, const u32 *vals,
                   const float *grad_out, float *grad_rows, int64_t L, int64_t G, cudaStream_t st)
 {
+    using namespace segred;
     const size_t smem = (size_t)(ctx->T + 1) * sizeof(int64_t);
-    const int64_t groups_per_block = 256 / LPR;
-    int64_t blocks = (y.num_chunks + groups_per_block - 1) / groups_per_block;
-    int64_t cap = (int64_t)ctx->num_sms * 8;
+    const int64_t cap = (int64_t)ctx->num_sms * 8;
+    int64_t blocks = (y.num_chunks + 7) / 8;                 // one warp per chunk
     int grid = (int)(blocks < 1 ? 1 : (blocks > cap ? cap : blocks));
     u32 *counters = reinterpret_cast<u32 *>(ws + y.counters);
     u32 *absmax = reinterpret_cast<u32 *>(ws + y.absmax);
+    const u32 *seg_start = reinterpret_cast<const u32 *>(ws + y.seg_start);
+    double *partials = reinterpret_cast<double *>(ws + y.partials);
+    u32 *long_list = reinterpret_cast<u32 *>(ws + y.long_list);
     seg_reduce_kernel<LPR, CH><<<grid, 256, smem, st>>>(
-        keys, vals, reinterpret_cast<const u32 *>(ws + y.seg_start), reinterpret_cast<const u32 *>(ws + y.chunk_first),
-        grad_out, grad_rows, reinterpret_cast<double *>(ws + y.partials), reinterpret_cast<u32 *>(ws + y.long_list),
-        counters, absmax, ctx->d_row_off, ctx->T, ctx->D, L, G, y.num_chunks, ctx->d_status);
+        keys, vals, seg_start, reinterpret_cast<const u32 *>(ws + y.chunk_first), grad_out, grad_rows, partials,
+        long_list, counters, absmax, ctx->d_row_off, ctx->T, ctx->D, L, G, y.num_chunks, ctx->d_status);
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
     dq_mark(ctx, st, DQ_K_SEG_REDUCE);
-    int64_t fb = (y.num_chunks + 7) / 8;      // one warp per cut segment, at most num_chunks of them
-    int fgrid = (int)(fb < 1 ? 1 : (fb > cap ? cap : fb));
-    seg_fixup_kernel<LPR, CH><<<fgrid, 256, smem, st>>>(
-        keys, reinterpret_cast<const u32 *>(ws + y.seg_start), reinterpret_cast<const double *>(ws + y.partials),
-        reinterpret_cast<const u32 *>(ws + y.long_list), counters, grad_rows, absmax, ctx->d_row_off, ctx->T, ctx->D);
+    int fgrid = (int)(blocks < (int64_t)ctx->num_sms * 4 ? (blocks < 1 ? 1 : blocks) : (int64_t)ctx->num_sms * 4);
+    seg_fixup_kernel<LPR, CH><<<fgrid, 256, smem, st>>>(keys, seg_start, partials, long_list, counters, grad_rows,
+                                                        absmax, ctx->d_row_off, ctx->T, ctx->D);
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
     dq_mark(ctx, st, DQ_K_SEG_FIXUP);
+    const size_t big_smem = (size_t)(256 / LPR) * ctx->D * sizeof(double);
+    if (big_smem > 48 * 1024) {
+        static bool raised = false;
+        if (!raised) {
+            DQRM_CUDA_TRY(ctx, cudaFuncSetAttribute(seg_fixup_big_kernel<LPR, CH>,
+                                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)big_smem));
+            raised = true;
+        }
+    }
+    int bgrid = (int)((y.num_chunks + BIG_PIECES - 1) / BIG_PIECES);     // at most this many big segments
+    if (bgrid > ctx->num_sms * 2) bgrid = ctx->num_sms * 2;
+    if (bgrid < 1) bgrid = 1;
+    seg_fixup_big_kernel<LPR, CH><<<bgrid, 256, big_smem, st>>>(keys, seg_start, partials, long_list, counters,
+                                                                 grad_rows, absmax, ctx->d_row_off, ctx->T, ctx->D,
+                                                                 y.num_chunks);
+    DQRM_CUDA_TRY(ctx, cudaGetLastError());
+    dq_mark(ctx, st, DQ_K_SEG_FIXUP_BIG);
     return DQRM_OK;
 }
 

@@ -29,7 +29,7 @@ struct dqrm_ctx {
 enum {
     DQ_K_BEGIN = 0, DQ_K_REFRESH, DQ_K_FWD, DQ_K_MEMSET, DQ_K_PREPARE, DQ_K_SORT_SCAN, DQ_K_SORT_SCATTER,
     DQ_K_SEG_COUNT, DQ_K_SEG_EMIT, DQ_K_SEG_REDUCE, DQ_K_SEG_FIXUP, DQ_K_ABSMAX, DQ_K_QUANT, DQ_K_UPDATE,
-    DQ_K_QUANT_UPDATE, DQ_K_COPY, DQ_K_COUNT
+    DQ_K_QUANT_UPDATE, DQ_K_COPY, DQ_K_SEG_FIXUP_BIG, DQ_K_COUNT
 };
 constexpr int DQ_PROF_MAX = 4096;
 
@@ -74,6 +74,82 @@ __device__ __forceinline__ int dq_code(float x, float s, float lo, float hi)
 }
 
 __device__ __forceinline__ float dq_dequant(int q, float s) { return __fmul_rn((float)q, s); }
+
+// ---------------------------------------------------------------------------------
+// The same codes without the IEEE-division sequence, for a scale shared by many elements,
+// four elements at a time.
+//
+//   QuantScale holds s and r = RN(1/s).  q0 = RN(x * r) equals x/s up to a relative error
+//   below 2^-22 (one rounding of r, one of the product), and RN(x/s) is within 2^-24 of
+//   x/s.  Only half-integers of magnitude below 2^(b-1) decide a b-bit code (beyond them the
+//   clamp gives the same code either way), and there |q0 - RN(x/s)| < 2^(b-23).  So if q0 is
+//   farther than TOL = 2^(b-21) from every half-integer, rounding q0 gives the same code as
+//   rounding RN(x/s).  Vectors with an element inside that window (about one in 10^4 for
+//   4-bit codes) are redone with the IEEE division.  Rounding to an integer is done by
+//   adding and subtracting 1.5*2^23 (round-to-nearest-even, no conversion instruction);
+//   the result is the code as a float, which is also what the dequantiser multiplies.
+//   The multiplies and adds use the packed two-float instructions of sm_100.
+//   Bit widths above 10 and scales outside [2^-100, 2^100] always take the IEEE path.
+// ---------------------------------------------------------------------------------
+struct QuantScale {
+    float s, r, lo, hi, tie_lim;
+    bool fast;
+};
+
+__device__ __forceinline__ QuantScale dq_make_scale(float s, int bits)
+{
+    QuantScale q;
+    q.s = s;
+    q.r = __frcp_rn(s);
+    q.lo = -(float)(1 << (bits - 1));
+    q.hi = (float)((1 << (bits - 1)) - 1);
+    q.tie_lim = 0.5f - (float)(1 << (bits - 1)) * 9.5367431640625e-07f;     // 0.5 - 2^(b-21)
+    q.fast = (bits <= 10) && (s >= 7.8886090522101181e-31f) && (s <= 1.2676506002282294e+30f);
+    return q;
+}
+
+// one code as a float by the plain definition
+__device__ __forceinline__ float dq_codef_ieee(float x, const QuantScale &q)
+{
+    // "+ 0" turns the -0.0 that rintf gives for small negative quotients into the +0.0 an integer code has
+    return __fadd_rn(fminf(fmaxf(rintf(__fdiv_rn(x, q.s)), q.lo), q.hi), 0.0f);
+}
+
+// codes (as floats, integer values in [lo, hi]) and dequantised values of four elements
+__device__ __forceinline__ void dq_fq4(const float4 &v, const QuantScale &q, float4 &codes, float4 &deq)
+{
+    const float MAGIC = 12582912.0f;                   // 1.5 * 2^23
+    bool done = false;
+    if (q.fast) {
+        const float2 r2 = make_float2(q.r, q.r), m2 = make_float2(MAGIC, MAGIC), nm2 = make_float2(-MAGIC, -MAGIC);
+        const float2 neg1 = make_float2(-1.f, -1.f);
+        const float2 qa = __fmul2_rn(make_float2(v.x, v.y), r2), qb = __fmul2_rn(make_float2(v.z, v.w), r2);
+        const float2 ra = __fadd2_rn(__fadd2_rn(qa, m2), nm2), rb = __fadd2_rn(__fadd2_rn(qb, m2), nm2);
+        const float2 da = __ffma2_rn(ra, neg1, qa), db = __ffma2_rn(rb, neg1, qb);     // q0 - rint(q0)
+        const float m = fmaxf(fmaxf(fabsf(da.x), fabsf(da.y)), fmaxf(fabsf(db.x), fabsf(db.y)));
+        if (m < q.tie_lim) {
+            codes = make_float4(fminf(fmaxf(ra.x, q.lo), q.hi), fminf(fmaxf(ra.y, q.lo), q.hi),
+                                fminf(fmaxf(rb.x, q.lo), q.hi), fminf(fmaxf(rb.y, q.lo), q.hi));
+            done = true;
+        }
+    }
+    if (!done)
+        codes = make_float4(dq_codef_ieee(v.x, q), dq_codef_ieee(v.y, q), dq_codef_ieee(v.z, q), dq_codef_ieee(v.w, q));
+    const float2 s2 = make_float2(q.s, q.s);
+    const float2 ea = __fmul2_rn(make_float2(codes.x, codes.y), s2), eb = __fmul2_rn(make_float2(codes.z, codes.w), s2);
+    deq = make_float4(ea.x, ea.y, eb.x, eb.y);
+}
+
+
+// 16-byte asynchronous copy global -> shared (data never passes through registers)
+__device__ __forceinline__ void dq_cp_async16(void *smem_dst, const void *gmem_src)
+{
+    unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16;\n" ::"r"(d), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void dq_cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void dq_cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
 
 __device__ __forceinline__ void dq_report(int *status, int code)
 {

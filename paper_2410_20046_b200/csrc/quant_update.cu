@@ -90,6 +90,7 @@ row_stream_kernel(float *__restrict__ tables, const int64_t *__restrict__ row_of
     int cur_t = -1;
     int64_t cur_end = -1, r0 = 0;
     float s = 1.f;
+    QuantScale qs = dq_make_scale(1.f, 8);
     for (int64_t u = group; u < U; u += n_groups) {
         if (u >= cur_end) {
             cur_t = table_of_row(s_uoff, T, u);
@@ -97,10 +98,11 @@ row_stream_kernel(float *__restrict__ tables, const int64_t *__restrict__ row_of
             if (MODE != MODE_QUANT) r0 = __ldg(row_off + cur_t);
             s = (MODE == MODE_UPDATE) ? __ldg(grad_scales + cur_t)
                                       : dq_scale_from_absmax(__uint_as_float(__ldg(absmax + cur_t)), 8);
+            qs = dq_make_scale(s, 8);
         }
         float4 *wrow = nullptr;
         if (MODE != MODE_QUANT) wrow = reinterpret_cast<float4 *>(tables + (r0 + __ldg(unique_rows + u)) * D);
-        int q[CH][4];
+        float q[CH][4];            // integer codes held as floats
         float4 w[CH];
 #pragma unroll
         for (int ch = 0; ch < CH; ++ch) {
@@ -111,10 +113,9 @@ row_stream_kernel(float *__restrict__ tables, const int64_t *__restrict__ row_of
                     q[ch][0] = c.x; q[ch][1] = c.y; q[ch][2] = c.z; q[ch][3] = c.w;
                 } else {
                     float4 g = __ldg(reinterpret_cast<const float4 *>(grad_rows + u * D) + c4);
-                    q[ch][0] = dq_code(g.x, s, -128.f, 127.f);
-                    q[ch][1] = dq_code(g.y, s, -128.f, 127.f);
-                    q[ch][2] = dq_code(g.z, s, -128.f, 127.f);
-                    q[ch][3] = dq_code(g.w, s, -128.f, 127.f);
+                    float4 cd, dq_unused;
+                    dq_fq4(g, qs, cd, dq_unused);
+                    q[ch][0] = cd.x; q[ch][1] = cd.y; q[ch][2] = cd.z; q[ch][3] = cd.w;
                 }
                 if (MODE != MODE_QUANT) w[ch] = wrow[c4];
             }
@@ -124,16 +125,16 @@ row_stream_kernel(float *__restrict__ tables, const int64_t *__restrict__ row_of
             int c4 = ch * LPR + lane;
             if (c4 < d4) {
                 if (MODE != MODE_UPDATE) {
-                    char4 c = make_char4((signed char)q[ch][0], (signed char)q[ch][1], (signed char)q[ch][2],
-                                         (signed char)q[ch][3]);
+                    char4 c = make_char4((signed char)(int)q[ch][0], (signed char)(int)q[ch][1],
+                                         (signed char)(int)q[ch][2], (signed char)(int)q[ch][3]);
                     *reinterpret_cast<char4 *>(codes + u * D + 4 * c4) = c;
                 }
                 if (MODE != MODE_QUANT) {
                     float4 x = w[ch];
-                    x.x = __fsub_rn(x.x, __fmul_rn(lr, dq_dequant(q[ch][0], s)));
-                    x.y = __fsub_rn(x.y, __fmul_rn(lr, dq_dequant(q[ch][1], s)));
-                    x.z = __fsub_rn(x.z, __fmul_rn(lr, dq_dequant(q[ch][2], s)));
-                    x.w = __fsub_rn(x.w, __fmul_rn(lr, dq_dequant(q[ch][3], s)));
+                    x.x = __fsub_rn(x.x, __fmul_rn(lr, __fmul_rn(q[ch][0], s)));
+                    x.y = __fsub_rn(x.y, __fmul_rn(lr, __fmul_rn(q[ch][1], s)));
+                    x.z = __fsub_rn(x.z, __fmul_rn(lr, __fmul_rn(q[ch][2], s)));
+                    x.w = __fsub_rn(x.w, __fmul_rn(lr, __fmul_rn(q[ch][3], s)));
                     wrow[c4] = x;
                 }
             }

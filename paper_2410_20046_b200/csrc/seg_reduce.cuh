@@ -1,0 +1,378 @@
+// Segmented reduction of the upstream gradient over the sorted lookups (second half of
+// the backward; paper Section 4.3 / Appendix B.1: duplicates of a row are coalesced).
+//
+// Input: keys[L] (arena rows, ascending), vals[L] (row of grad_out for each lookup, in
+// stable order), chunk_first[c] = index of the segment that holds sorted entry 32*c,
+// seg_start[U+1].  One warp owns one chunk of 32 sorted entries.  The warp's SG = 32/LPR
+// lane groups each gather one upstream-gradient row per step (LPR lanes x 128 bit), the
+// rows of a step are combined by a segmented warp-shuffle scan keyed on the row id, and a
+// carry links the steps.  All sums are FP64 and have a shape fixed by the entry
+// positions, so results are reproducible.  A run that is a whole segment is rounded to
+// FP32 and written; a run cut by the chunk boundary leaves an FP64 partial and the
+// segment is finished by one of the fix-up kernels (a warp for up to 32 pieces, a block
+// beyond that).  The per-table abs-max of the rounded sums is collected on the way.
+#pragma once
+#include "common.cuh"
+
+namespace segred {
+
+constexpr int CHUNK = 32;            // sorted entries per warp work item
+constexpr int BIG_PIECES = 32;       // cut segments with more pieces go to the block-wide fix-up
+enum { CNT_LONG = 0, CNT_U = 1, CNT_BIG = 2 };
+
+template <int LPR>
+__device__ __forceinline__ u32 group_mask()
+{
+    if constexpr (LPR >= 32) {
+        return 0xffffffffu;
+    } else {
+        const int lane = threadIdx.x & 31;
+        return ((1u << LPR) - 1u) << (lane / LPR * LPR);
+    }
+}
+
+template <int LPR>
+__device__ __forceinline__ float group_max(float m)
+{
+    const u32 gm = group_mask<LPR>();
+#pragma unroll
+    for (int o = LPR / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(gm, m, o));
+    return m;
+}
+
+// running abs-max of one table at a time (keys only ascend along a lane group's work)
+struct AbsmaxTracker {
+    int t = -1;
+    int64_t t_end = -1;
+    float m = 0.f;
+};
+
+template <int LPR>
+__device__ __forceinline__ void absmax_push(AbsmaxTracker &tr, u32 *absmax)
+{
+    float m = group_max<LPR>(tr.m);      // called group-uniformly
+    if ((threadIdx.x % LPR) == 0 && tr.t >= 0 && m > 0.f) atomicMax(&absmax[tr.t], __float_as_uint(m));
+    tr.m = 0.f;
+}
+
+template <int LPR>
+__device__ __forceinline__ void absmax_note(AbsmaxTracker &tr, u32 key, float m, const int64_t *s_off, int T,
+                                            u32 *absmax)
+{
+    if ((int64_t)key >= tr.t_end) {
+        absmax_push<LPR>(tr, absmax);
+        tr.t = dq_table_of(s_off, T, (int64_t)key);
+        tr.t_end = s_off[tr.t + 1];
+    }
+    tr.m = fmaxf(tr.m, m);
+}
+
+template <int CH>
+__device__ __forceinline__ float round_store(const double (&acc)[CH][4], float *dst_row, int lane, int lpr, int d4)
+{
+    float m = 0.f;
+#pragma unroll
+    for (int ch = 0; ch < CH; ++ch) {
+        int c4 = ch * lpr + lane;
+        if (c4 < d4) {
+            float4 r = make_float4((float)acc[ch][0], (float)acc[ch][1], (float)acc[ch][2], (float)acc[ch][3]);
+            *reinterpret_cast<float4 *>(dst_row + 4 * c4) = r;
+            m = fmaxf(fmaxf(m, fmaxf(fabsf(r.x), fabsf(r.y))), fmaxf(fabsf(r.z), fabsf(r.w)));
+        }
+    }
+    return m;
+}
+
+template <int LPR, int CH>
+__global__ void __launch_bounds__(256)
+seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
+                  const u32 *__restrict__ seg_start, const u32 *__restrict__ chunk_first,
+                  const float *__restrict__ grad_out, float *__restrict__ grad_rows,
+                  double *__restrict__ partials, u32 *__restrict__ long_list, u32 *__restrict__ counters,
+                  u32 *__restrict__ absmax, const int64_t *__restrict__ row_off, int T, int D,
+                  int64_t L, int64_t G, int64_t num_chunks, int *__restrict__ status)
+{
+    extern __shared__ unsigned char smem_raw[];
+    int64_t *s_off = reinterpret_cast<int64_t *>(smem_raw);
+    for (int t = threadIdx.x; t <= T; t += blockDim.x) s_off[t] = row_off[t];
+    __syncthreads();
+
+    constexpr int SG = 32 / LPR;                 // lane groups per warp = entries per step
+    constexpr int STEPS = CHUNK / SG;            // steps per chunk
+    constexpr int PRE = STEPS < 8 ? STEPS : 8;   // steps whose rows are loaded together
+    const int d4 = D >> 2;
+    const int wl = threadIdx.x & 31;
+    const int sub = wl / LPR, lane = wl % LPR;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    AbsmaxTracker tr;
+
+    for (int64_t c = warp; c < num_chunks; c += n_warps) {
+        const int64_t i0 = c * CHUNK;
+        const int n = (int)min((int64_t)CHUNK, L - i0);
+        u32 my_key = 0xFFFFFFFFu, my_val = 0u;
+        if (wl < n) {
+            my_key = keys[i0 + wl];
+            my_val = vals[i0 + wl];
+            if ((int64_t)my_val >= G) { dq_report(status, DQRM_ERR_INDEX_RANGE); my_val = 0u; }
+        }
+        const bool has_prev = i0 > 0, has_next = i0 + n < L;
+        const u32 prev_key = has_prev ? keys[i0 - 1] : 0u;
+        const u32 next_key = has_next ? keys[i0 + n] : 0u;
+        const u32 up_key = __shfl_up_sync(0xffffffffu, my_key, 1);
+        const bool head = (wl < n) && (wl == 0 ? (!has_prev || my_key != prev_key) : (my_key != up_key));
+        const u32 headmask = __ballot_sync(0xffffffffu, head);
+        const u32 down_key = __shfl_down_sync(0xffffffffu, my_key, 1);
+        const bool tail = (wl < n) && (wl == n - 1 || down_key != my_key);
+        const u32 tailmask = __ballot_sync(0xffffffffu, tail);
+        const bool continues_after = has_next && next_key == __shfl_sync(0xffffffffu, my_key, n - 1);
+        const u32 u0 = chunk_first[c];
+
+        double carry[CH][4];
+        u32 carry_key = 0xFFFFFFFFu;
+#pragma unroll
+        for (int ch = 0; ch < CH; ++ch) carry[ch][0] = carry[ch][1] = carry[ch][2] = carry[ch][3] = 0.0;
+
+#pragma unroll 1
+        for (int st0 = 0; st0 < STEPS; st0 += PRE) {
+            float4 row[PRE][CH];
+#pragma unroll
+            for (int p = 0; p < PRE; ++p) {
+                const int e = (st0 + p) * SG + sub;
+                const u32 v = __shfl_sync(0xffffffffu, my_val, e & 31);
+                if (e < n) {
+                    const float4 *src = reinterpret_cast<const float4 *>(grad_out + (int64_t)v * D);
+#pragma unroll
+                    for (int ch = 0; ch < CH; ++ch) {
+                        int c4 = ch * LPR + lane;
+                        if (c4 < d4) row[p][ch] = __ldg(src + c4);
+                    }
+                }
+            }
+#pragma unroll
+            for (int p = 0; p < PRE; ++p) {
+                const int e = (st0 + p) * SG + sub;
+                const bool valid = e < n;
+                const u32 key_e = __shfl_sync(0xffffffffu, my_key, e & 31);
+                double acc[CH][4];
+#pragma unroll
+                for (int ch = 0; ch < CH; ++ch) {
+                    int c4 = ch * LPR + lane;
+                    bool on = valid && c4 < d4;
+                    acc[ch][0] = on ? (double)row[p][ch].x : 0.0;
+                    acc[ch][1] = on ? (double)row[p][ch].y : 0.0;
+                    acc[ch][2] = on ? (double)row[p][ch].z : 0.0;
+                    acc[ch][3] = on ? (double)row[p][ch].w : 0.0;
+                }
+                // segmented inclusive scan over the SG entries of this step
+#pragma unroll
+                for (int o = 1; o < SG; o <<= 1) {
+                    const u32 key_o = __shfl_up_sync(0xffffffffu, key_e, o * LPR);
+                    const bool take = valid && sub >= o && key_o == key_e;
+#pragma unroll
+                    for (int ch = 0; ch < CH; ++ch)
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            double other = __shfl_up_sync(0xffffffffu, acc[ch][q], o * LPR);
+                            if (take) acc[ch][q] += other;
+                        }
+                }
+                // link to the previous step
+                if (valid && key_e == carry_key) {
+#pragma unroll
+                    for (int ch = 0; ch < CH; ++ch)
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) acc[ch][q] += carry[ch][q];
+                }
+                // the last lane group's running sum is the next step's carry
+                carry_key = __shfl_sync(0xffffffffu, valid ? key_e : 0xFFFFFFFFu, (SG - 1) * LPR + lane);
+#pragma unroll
+                for (int ch = 0; ch < CH; ++ch)
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        carry[ch][q] = __shfl_sync(0xffffffffu, acc[ch][q], (SG - 1) * LPR + lane);
+
+                if (valid && ((tailmask >> e) & 1u)) {
+                    // entry e closes a run inside this chunk
+                    const u32 below = headmask & (0xffffffffu >> (31 - e));      // heads at entries 0..e
+                    const bool begins = below != 0u;                            // the run's head is in this chunk
+                    const u32 u = u0 + __popc(below & ~1u);
+                    const bool ends = !(e == n - 1 && continues_after);
+                    if (begins && ends) {
+                        float m = round_store<CH>(acc, grad_rows + (int64_t)u * D, lane, LPR, d4);
+                        absmax_note<LPR>(tr, key_e, m, s_off, T, absmax);
+                    } else {
+                        double *pdst = partials + ((size_t)c * 2 + (begins ? 1 : 0)) * D;
+#pragma unroll
+                        for (int ch = 0; ch < CH; ++ch) {
+                            int c4 = ch * LPR + lane;
+                            if (c4 < d4) {
+                                *reinterpret_cast<double2 *>(pdst + 4 * c4) = make_double2(acc[ch][0], acc[ch][1]);
+                                *reinterpret_cast<double2 *>(pdst + 4 * c4 + 2) = make_double2(acc[ch][2], acc[ch][3]);
+                            }
+                        }
+                        if (begins && lane == 0) {
+                            const u32 a = seg_start[u], b = seg_start[u + 1];
+                            const u32 npieces = (b - 1) / CHUNK - a / CHUNK + 1;
+                            if (npieces > BIG_PIECES)
+                                long_list[num_chunks - 1 - atomicAdd(&counters[CNT_BIG], 1u)] = u;
+                            else
+                                long_list[atomicAdd(&counters[CNT_LONG], 1u)] = u;
+                        }
+                    }
+                }
+            }
+        }
+    }
+    // every lane group flushes its last table's maximum (group-uniform)
+    absmax_push<LPR>(tr, absmax);
+}
+
+// pieces of cut segment [a, e): chunk a/32 holds the first (slot 1), later chunks slot 0
+__device__ __forceinline__ const double *piece_ptr(const double *partials, int64_t c0, int64_t p, int D)
+{
+    return partials + ((size_t)(c0 + p) * 2 + (p == 0 ? 1 : 0)) * D;
+}
+
+template <int CH>
+__device__ __forceinline__ void add_pieces(double (&acc)[CH][4], const double *partials, int64_t c0,
+                                           int64_t p_begin, int64_t p_end, int64_t stride, int D, int lane,
+                                           int lpr, int d4)
+{
+    constexpr int UN = 4;
+    for (int64_t p = p_begin; p < p_end; p += stride * UN) {
+        double2 x[UN][CH], y[UN][CH];
+#pragma unroll
+        for (int k = 0; k < UN; ++k) {
+            const int64_t pk = p + k * stride;
+            if (pk < p_end) {
+                const double *src = piece_ptr(partials, c0, pk, D);
+#pragma unroll
+                for (int ch = 0; ch < CH; ++ch) {
+                    int c4 = ch * lpr + lane;
+                    if (c4 < d4) {
+                        x[k][ch] = __ldcg(reinterpret_cast<const double2 *>(src + 4 * c4));
+                        y[k][ch] = __ldcg(reinterpret_cast<const double2 *>(src + 4 * c4 + 2));
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < UN; ++k) {
+            if (p + k * stride < p_end) {
+#pragma unroll
+                for (int ch = 0; ch < CH; ++ch) {
+                    int c4 = ch * lpr + lane;
+                    if (c4 < d4) {
+                        acc[ch][0] += x[k][ch].x; acc[ch][1] += x[k][ch].y;
+                        acc[ch][2] += y[k][ch].x; acc[ch][3] += y[k][ch].y;
+                    }
+                }
+            }
+        }
+    }
+}
+
+// one warp per cut segment of at most BIG_PIECES pieces
+template <int LPR, int CH>
+__global__ void __launch_bounds__(256)
+seg_fixup_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ seg_start,
+                 const double *__restrict__ partials, const u32 *__restrict__ long_list,
+                 const u32 *__restrict__ counters, float *__restrict__ grad_rows, u32 *__restrict__ absmax,
+                 const int64_t *__restrict__ row_off, int T, int D)
+{
+    extern __shared__ unsigned char smem_raw[];
+    int64_t *s_off = reinterpret_cast<int64_t *>(smem_raw);
+    for (int t = threadIdx.x; t <= T; t += blockDim.x) s_off[t] = row_off[t];
+    __syncthreads();
+    constexpr int SG = 32 / LPR;
+    const int d4 = D >> 2;
+    const int wl = threadIdx.x & 31;
+    const int sub = wl / LPR, lane = wl % LPR;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const u32 count = counters[CNT_LONG];
+    for (int64_t s = warp; s < count; s += n_warps) {
+        const u32 u = long_list[s];
+        const u32 a = seg_start[u], e = seg_start[u + 1];
+        const int64_t c0 = a / CHUNK, c1 = (e - 1) / CHUNK;
+        double acc[CH][4];
+#pragma unroll
+        for (int ch = 0; ch < CH; ++ch) acc[ch][0] = acc[ch][1] = acc[ch][2] = acc[ch][3] = 0.0;
+        add_pieces<CH>(acc, partials, c0, sub, c1 - c0 + 1, SG, D, lane, LPR, d4);
+#pragma unroll
+        for (int o = LPR; o < 32; o <<= 1)
+#pragma unroll
+            for (int ch = 0; ch < CH; ++ch)
+#pragma unroll
+                for (int q = 0; q < 4; ++q) acc[ch][q] += __shfl_xor_sync(0xffffffffu, acc[ch][q], o);
+        float m = 0.f;
+        if (sub == 0) m = round_store<CH>(acc, grad_rows + (int64_t)u * D, lane, LPR, d4);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if (wl == 0 && m > 0.f) atomicMax(&absmax[dq_table_of(s_off, T, (int64_t)keys[a])], __float_as_uint(m));
+    }
+}
+
+// one block per cut segment of more than BIG_PIECES pieces (hot rows)
+template <int LPR, int CH>
+__global__ void __launch_bounds__(256)
+seg_fixup_big_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ seg_start,
+                     const double *__restrict__ partials, const u32 *__restrict__ long_list,
+                     const u32 *__restrict__ counters, float *__restrict__ grad_rows, u32 *__restrict__ absmax,
+                     const int64_t *__restrict__ row_off, int T, int D, int64_t num_chunks)
+{
+    extern __shared__ unsigned char smem_raw[];
+    constexpr int NSG = 256 / LPR;
+    double *s_part = reinterpret_cast<double *>(smem_raw);            // [NSG][D]
+    const int d4 = D >> 2;
+    const int sub = threadIdx.x / LPR, lane = threadIdx.x % LPR;
+    const u32 count = counters[CNT_BIG];
+    for (u32 s = blockIdx.x; s < count; s += gridDim.x) {
+        const u32 u = long_list[num_chunks - 1 - s];
+        const u32 a = seg_start[u], e = seg_start[u + 1];
+        const int64_t c0 = a / CHUNK, c1 = (e - 1) / CHUNK;
+        double acc[CH][4];
+#pragma unroll
+        for (int ch = 0; ch < CH; ++ch) acc[ch][0] = acc[ch][1] = acc[ch][2] = acc[ch][3] = 0.0;
+        add_pieces<CH>(acc, partials, c0, sub, c1 - c0 + 1, NSG, D, lane, LPR, d4);
+        __syncthreads();
+#pragma unroll
+        for (int ch = 0; ch < CH; ++ch) {
+            int c4 = ch * LPR + lane;
+            if (c4 < d4) {
+                double *dst = s_part + (size_t)sub * D + 4 * c4;
+                dst[0] = acc[ch][0]; dst[1] = acc[ch][1]; dst[2] = acc[ch][2]; dst[3] = acc[ch][3];
+            }
+        }
+        __syncthreads();
+        if (sub == 0) {
+            // lane group 0 adds the NSG sub-sums in order
+            float m = 0.f;
+#pragma unroll
+            for (int ch = 0; ch < CH; ++ch) {
+                int c4 = ch * LPR + lane;
+                if (c4 < d4) {
+                    double t0 = 0, t1 = 0, t2 = 0, t3 = 0;
+                    for (int g = 0; g < NSG; ++g) {
+                        const double *src = s_part + (size_t)g * D + 4 * c4;
+                        t0 += src[0]; t1 += src[1]; t2 += src[2]; t3 += src[3];
+                    }
+                    float4 r = make_float4((float)t0, (float)t1, (float)t2, (float)t3);
+                    *reinterpret_cast<float4 *>(grad_rows + (int64_t)u * D + 4 * c4) = r;
+                    m = fmaxf(fmaxf(m, fmaxf(fabsf(r.x), fabsf(r.y))), fmaxf(fabsf(r.z), fabsf(r.w)));
+                }
+            }
+            m = group_max<LPR>(m);
+            if (lane == 0 && m > 0.f) {
+                // row_off is read from global memory here: this path runs for a handful of hot rows
+                int lo = 0, hi = T;
+                const int64_t key = (int64_t)keys[a];
+                while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (row_off[mid] <= key) lo = mid; else hi = mid; }
+                atomicMax(&absmax[lo], __float_as_uint(m));
+            }
+        }
+    }
+}
+
+}  // namespace segred
