@@ -3,30 +3,30 @@
 // row with the table's stored scale, and sum-pool over the bag.  No low-precision copy
 // of the table exists; only the gathered rows are ever quantised.
 //
-// HBM-bound random row gather: throughput is set by how many row requests an SM keeps
-// in flight.  Rows therefore travel global -> shared memory with 16-byte asynchronous
-// copies (cp.async), two batches deep, so the bytes in flight cost no registers and the
-// occupancy stays high; every thread reads back exactly the 16-byte pieces it copied, so
-// no block barrier is needed.  blockIdx.y is the table, which makes scale, bit width and
-// row base block constants.  A group of LPR lanes owns one row: a feature-16 row is one
-// 64-byte request of four lanes, a feature-64 row one 256-byte request of sixteen.
-//   * fwd_onehot_kernel (launched when L == T*B, the Criteo-shaped case): a group has
-//     NB rows of NB different one-index bags in flight per batch; the pooled value is
-//     the fake-quantised row itself.  A bag that turns out not to hold exactly one index
-//     takes the general routine.
-//   * fwd_bags_kernel (any other batch): a group walks one bag at a time, NB of its rows
-//     per batch, and sums them in bag order in FP64, rounded once, so the result does
-//     not depend on the launch shape.
+// HBM-bound random row gather.  Measured on B200, a bare gather of this access pattern
+// runs fastest with many resident warps and only two to four independent 128-bit loads
+// per lane, so the kernels are kept lean (about 40 registers) rather than deeply
+// unrolled.  blockIdx.y is the table, which makes scale, bit width and row base block
+// constants.  A group of LPR lanes owns one row: a feature-16 row is one 64-byte request
+// of four lanes, a feature-64 row one 256-byte request of sixteen.
+//   * fwd_onehot_kernel (launched when L == T*B and no codes are asked for, the Criteo-shaped
+//     training case): a lane group
+//     has NB rows of NB different one-index bags in flight; the pooled value is the
+//     fake-quantised row itself.  A bag that turns out not to hold exactly one index is
+//     pooled by a plain loop.
+//   * fwd_bags_kernel (any other batch): a lane group walks one bag at a time, NB of its
+//     rows per batch, and sums them in bag order in FP64, rounded once, so the result
+//     does not depend on the launch shape.
 #include "common.cuh"
 
 namespace {
 
 constexpr int FW_THREADS = 256;
-constexpr int FW_STAGES = 2;      // batches in flight
-// rows per lane group per batch: four for rows of up to 128 features, fewer for wider rows so
-// that the staging buffer stays at 32 KB per block (64 KB beyond 512 features)
-template <int CH>
-struct NBOf { static constexpr int v = CH >= 4 ? 1 : (CH == 2 ? 2 : 4); };
+// independent rows in flight per lane group.  Measured on B200: four for rows of up to 128
+// bytes, two for 256- and 512-byte rows (more resident warps beat deeper unrolling), one
+// when a lane already holds several 128-bit pieces of every row
+template <int LPR, int CH>
+struct NBOf { static constexpr int v = CH >= 2 ? 1 : (LPR >= 16 ? 2 : 4); };
 
 struct FwdArgs {
     const float *tables;
@@ -42,246 +42,209 @@ struct FwdArgs {
     int *status;
 };
 
-__device__ __forceinline__ float4 fq4(const float4 &v, const QuantScale &qs, float4 &codes)
-{
-    float4 deq;
-    dq_fq4(v, qs, codes, deq);
-    return deq;
-}
-
 __device__ __forceinline__ void store_codes(int8_t *codes_out, int64_t j, int D, int c4, const float4 &c)
 {
     char4 cc = make_char4((signed char)(int)c.x, (signed char)(int)c.y, (signed char)(int)c.z, (signed char)(int)c.w);
     *reinterpret_cast<char4 *>(codes_out + j * D + 4 * c4) = cc;
 }
 
-__device__ __forceinline__ int32_t checked_index(int32_t idx, int64_t nrows, int *status)
+// clamps an index into [0, nrows) and remembers that it had to
+__device__ __forceinline__ int32_t clamp_index(int32_t idx, int32_t nrows, bool &bad)
 {
-    if (idx < 0 || idx >= nrows) {
-        dq_report(status, DQRM_ERR_INDEX_RANGE);
-        idx = idx < 0 ? 0 : (int32_t)(nrows - 1);
-    }
-    return idx;
+    bad |= (idx < 0) | (idx >= nrows);
+    return min(max(idx, 0), nrows - 1);
 }
 
-// thread-private slot of the staging buffer: [stage][row-in-batch][vector][thread]
-template <int CH>
-__device__ __forceinline__ float4 *slot(float4 *buf, int stage, int b, int c)
+// Per-table constants of a block
+struct TableCtx {
+    QuantScale qs;
+    const float *tbl;
+    int32_t nrows;
+    int64_t g0;
+};
+
+__device__ __forceinline__ TableCtx table_ctx(const FwdArgs &a, int t, int D)
 {
-    return buf + ((size_t)((stage * NBOf<CH>::v + b) * CH + c)) * FW_THREADS + threadIdx.x;
+    TableCtx c;
+    c.qs = dq_make_scale(__ldg(a.scales + t), __ldg(a.bits + t));
+    const int64_t r0 = __ldg(a.row_off + t);
+    c.nrows = (int32_t)(__ldg(a.row_off + t + 1) - r0);
+    c.tbl = a.tables + r0 * D;
+    c.g0 = (int64_t)t * a.B;
+    return c;
 }
 
-// one bag: NB of its rows per batch, FP64 sum in bag order
+// plain pooling of one bag (one row at a time): used for the rare bags of a one-index batch
 template <int LPR, int CH>
-__device__ __forceinline__ void pool_bag(const FwdArgs &a, const float *tbl, int64_t nrows, const QuantScale &qs,
-                                         int32_t lo, int32_t hi, float *out_row, int lane, float4 *buf)
+__device__ __forceinline__ void pool_bag_plain(const FwdArgs &a, const TableCtx &tc, int D, int d4, int32_t lo,
+                                               int32_t hi, float *out_row, int lane, bool &bad)
 {
-    const int d4 = a.D >> 2;
-    if (lo < 0 || hi < lo || (int64_t)hi > a.L) { dq_report(a.status, DQRM_ERR_INDEX_RANGE); hi = lo = 0; }
-    double acc[CH][4];
-#pragma unroll
-    for (int c = 0; c < CH; ++c) acc[c][0] = acc[c][1] = acc[c][2] = acc[c][3] = 0.0;
+    if (lo < 0 || hi < lo || (int64_t)hi > a.L) { bad = true; hi = lo = 0; }
+#pragma unroll 1
+    for (int c = 0; c < CH; ++c) {
+        const int c4 = c * LPR + lane;
+        if (c4 >= d4) continue;
+        double a0 = 0, a1 = 0, a2 = 0, a3 = 0;
+#pragma unroll 1
+        for (int32_t j = lo; j < hi; ++j) {
+            const int32_t idx = clamp_index(__ldg(a.indices + j), tc.nrows, bad);
+            float4 cd, f;
+            dq_fq4(__ldg(reinterpret_cast<const float4 *>(tc.tbl + (int64_t)idx * D) + c4), tc.qs, cd, f);
+            a0 += (double)f.x; a1 += (double)f.y; a2 += (double)f.z; a3 += (double)f.w;
+            if (a.codes_out) store_codes(a.codes_out, j, D, c4, cd);
+        }
+        reinterpret_cast<float4 *>(out_row)[c4] = make_float4((float)a0, (float)a1, (float)a2, (float)a3);
+    }
+}
 
-    auto issue = [&](int32_t j0, int stage) {
+template <int LPR, int CH, bool EXACT>
+__global__ void __launch_bounds__(FW_THREADS, 6)
+fwd_onehot_kernel(const FwdArgs a)
+{
+    constexpr int NB = NBOf<LPR, CH>::v;
+    constexpr int GPB = FW_THREADS / LPR;
+    const int D = EXACT ? 4 * LPR * CH : a.D;
+    const int d4 = D >> 2;
+    const int t = blockIdx.y;
+    const int lane = threadIdx.x % LPR;
+    const int grp = threadIdx.x / LPR;
+    const TableCtx tc = table_ctx(a, t, D);
+    bool bad = false;
+
+    for (int ib = blockIdx.x * (GPB * NB); ib < a.B; ib += gridDim.x * (GPB * NB)) {
+        int32_t lo[NB], idx[NB];
+        unsigned one = 0;                 // bit b: bag b holds exactly one index
+        unsigned rare = 0;                // bit b: bag b exists but is not a one-index bag
 #pragma unroll
-        for (int b = 0; b < NBOf<CH>::v; ++b) {
-            if (j0 + b < hi) {
-                const int32_t idx = checked_index(__ldg(a.indices + j0 + b), nrows, a.status);
-                const float4 *row = reinterpret_cast<const float4 *>(tbl + (int64_t)idx * a.D);
+        for (int b = 0; b < NB; ++b) {
+            const int i = ib + b * GPB + grp;
+            lo[b] = 0; idx[b] = 0;
+            if (i < a.B) {
+                lo[b] = __ldg(a.offsets + tc.g0 + i);
+                const int32_t hi = __ldg(a.offsets + tc.g0 + i + 1);
+                idx[b] = __ldg(a.indices + tc.g0 + i);      // right when offsets are the identity (L == T*B)
+                if (hi - lo[b] == 1 && lo[b] >= 0 && (int64_t)hi <= a.L) one |= 1u << b; else rare |= 1u << b;
+            }
+        }
 #pragma unroll
-                for (int c = 0; c < CH; ++c) {
-                    const int c4 = c * LPR + lane;
-                    if (c4 < d4) dq_cp_async16(slot<CH>(buf, stage, b, c), row + c4);
+        for (int b = 0; b < NB; ++b) {
+            const int i = ib + b * GPB + grp;
+            if (((one >> b) & 1u) && (int64_t)lo[b] != tc.g0 + i) idx[b] = __ldg(a.indices + lo[b]);
+            idx[b] = clamp_index(idx[b], tc.nrows, bad);
+        }
+#pragma unroll
+        for (int c = 0; c < CH; ++c) {
+            const int c4 = c * LPR + lane;
+            float4 v[NB];
+#pragma unroll
+            for (int b = 0; b < NB; ++b)
+                if (((one >> b) & 1u) && (EXACT || c4 < d4))
+                    v[b] = __ldg(reinterpret_cast<const float4 *>(tc.tbl + (int64_t)idx[b] * D) + c4);
+#pragma unroll
+            for (int b = 0; b < NB; ++b) {
+                if (((one >> b) & 1u) && (EXACT || c4 < d4)) {
+                    const int i = ib + b * GPB + grp;
+                    float4 cd, f;
+                    dq_fq4(v[b], tc.qs, cd, f);
+                    reinterpret_cast<float4 *>(a.out + ((int64_t)i * a.T + t) * D)[c4] = f;
                 }
             }
         }
-        dq_cp_async_commit();
-    };
+        if (rare) {
+#pragma unroll 1
+            for (int b = 0; b < NB; ++b) {
+                if ((rare >> b) & 1u) {
+                    const int i = ib + b * GPB + grp;
+                    const int32_t l = __ldg(a.offsets + tc.g0 + i), h = __ldg(a.offsets + tc.g0 + i + 1);
+                    pool_bag_plain<LPR, CH>(a, tc, D, d4, l, h, a.out + ((int64_t)i * a.T + t) * D, lane, bad);
+                }
+            }
+        }
+    }
+    if (bad) dq_report(a.status, DQRM_ERR_INDEX_RANGE);
+}
 
-    int stage = 0;
-    if (lo < hi) issue(lo, 0);
-    for (int32_t j0 = lo; j0 < hi; j0 += NBOf<CH>::v) {
-        if (j0 + NBOf<CH>::v < hi) { issue(j0 + NBOf<CH>::v, stage ^ 1); dq_cp_async_wait<1>(); }
-        else dq_cp_async_wait<0>();
+template <int LPR, int CH, bool EXACT>
+__global__ void __launch_bounds__(FW_THREADS)
+fwd_bags_kernel(const FwdArgs a)
+{
+    constexpr int NB = NBOf<LPR, CH>::v;
+    constexpr int GPB = FW_THREADS / LPR;
+    const int D = EXACT ? 4 * LPR * CH : a.D;
+    const int d4 = D >> 2;
+    const int t = blockIdx.y;
+    const int lane = threadIdx.x % LPR;
+    const int grp = threadIdx.x / LPR;
+    const TableCtx tc = table_ctx(a, t, D);
+    bool bad = false;
+
+    for (int i = blockIdx.x * GPB + grp; i < a.B; i += gridDim.x * GPB) {
+        int32_t lo = __ldg(a.offsets + tc.g0 + i), hi = __ldg(a.offsets + tc.g0 + i + 1);
+        if (lo < 0 || hi < lo || (int64_t)hi > a.L) { bad = true; hi = lo = 0; }
+        double acc[CH][4];
 #pragma unroll
-        for (int b = 0; b < NBOf<CH>::v; ++b) {
-            if (j0 + b < hi) {
+        for (int c = 0; c < CH; ++c) acc[c][0] = acc[c][1] = acc[c][2] = acc[c][3] = 0.0;
+        for (int32_t j0 = lo; j0 < hi; j0 += NB) {
+            int32_t idx[NB];
 #pragma unroll
-                for (int c = 0; c < CH; ++c) {
-                    const int c4 = c * LPR + lane;
-                    if (c4 < d4) {
-                        float4 cd;
-                        const float4 f = fq4(*slot<CH>(buf, stage, b, c), qs, cd);
+            for (int b = 0; b < NB; ++b) idx[b] = (j0 + b < hi) ? clamp_index(__ldg(a.indices + j0 + b), tc.nrows, bad) : 0;
+#pragma unroll
+            for (int c = 0; c < CH; ++c) {
+                const int c4 = c * LPR + lane;
+                float4 v[NB];
+#pragma unroll
+                for (int b = 0; b < NB; ++b)
+                    if (j0 + b < hi && (EXACT || c4 < d4))
+                        v[b] = __ldg(reinterpret_cast<const float4 *>(tc.tbl + (int64_t)idx[b] * D) + c4);
+#pragma unroll
+                for (int b = 0; b < NB; ++b) {
+                    if (j0 + b < hi && (EXACT || c4 < d4)) {
+                        float4 cd, f;
+                        dq_fq4(v[b], tc.qs, cd, f);
                         acc[c][0] += (double)f.x;
                         acc[c][1] += (double)f.y;
                         acc[c][2] += (double)f.z;
                         acc[c][3] += (double)f.w;
-                        if (a.codes_out) store_codes(a.codes_out, j0 + b, a.D, c4, cd);
+                        if (a.codes_out) store_codes(a.codes_out, j0 + b, D, c4, cd);
                     }
                 }
             }
         }
-        stage ^= 1;
-    }
+        float4 *o = reinterpret_cast<float4 *>(a.out + ((int64_t)i * a.T + t) * D);
 #pragma unroll
-    for (int c = 0; c < CH; ++c) {
-        const int c4 = c * LPR + lane;
-        if (c4 < d4)
-            reinterpret_cast<float4 *>(out_row)[c4] =
-                make_float4((float)acc[c][0], (float)acc[c][1], (float)acc[c][2], (float)acc[c][3]);
+        for (int c = 0; c < CH; ++c) {
+            const int c4 = c * LPR + lane;
+            if (EXACT || c4 < d4)
+                o[c4] = make_float4((float)acc[c][0], (float)acc[c][1], (float)acc[c][2], (float)acc[c][3]);
+        }
     }
+    if (bad) dq_report(a.status, DQRM_ERR_INDEX_RANGE);
 }
 
-template <int LPR, int CH>
-__device__ __noinline__ void pool_bag_rare(const FwdArgs &a, const float *tbl, int64_t nrows, const QuantScale &qs,
-                                           int32_t lo, int32_t hi, float *out_row, int lane, float4 *buf)
-{
-    pool_bag<LPR, CH>(a, tbl, nrows, qs, lo, hi, out_row, lane, buf);
-}
-
-template <int LPR, int CH>
-__global__ void __launch_bounds__(FW_THREADS, 4)
-fwd_onehot_kernel(const FwdArgs a)
-{
-    extern __shared__ float4 s_buf[];            // [FW_STAGES][NBOf<CH>::v][CH][FW_THREADS]
-    constexpr int GPB = FW_THREADS / LPR;
-    constexpr int TILE = GPB * NBOf<CH>::v;            // bags per block per batch
-    const int t = blockIdx.y;
-    const int d4 = a.D >> 2;
-    const int lane = threadIdx.x % LPR;
-    const int grp = threadIdx.x / LPR;
-    const QuantScale qs = dq_make_scale(__ldg(a.scales + t), __ldg(a.bits + t));
-    const int64_t r0 = __ldg(a.row_off + t);
-    const int64_t nrows = __ldg(a.row_off + t + 1) - r0;
-    const float *tbl = a.tables + r0 * a.D;
-    const int64_t g0 = (int64_t)t * a.B;
-
-    // state of one batch: offsets of its NB bags and which of them hold exactly one index
-    struct Batch { int32_t lo[NBOf<CH>::v], hi[NBOf<CH>::v]; unsigned one; };
-
-    auto issue = [&](int ib, int stage, Batch &bt) {
-        int32_t idx[NBOf<CH>::v];
-#pragma unroll
-        for (int b = 0; b < NBOf<CH>::v; ++b) {
-            const int i = ib + b * GPB + grp;
-            bt.lo[b] = 0; bt.hi[b] = 0; idx[b] = 0;
-            if (i < a.B) {
-                bt.lo[b] = __ldg(a.offsets + g0 + i);
-                bt.hi[b] = __ldg(a.offsets + g0 + i + 1);
-                idx[b] = __ldg(a.indices + g0 + i);          // right when offsets are the identity (L == T*B)
-            }
-        }
-        bt.one = 0;
-#pragma unroll
-        for (int b = 0; b < NBOf<CH>::v; ++b) {
-            const int i = ib + b * GPB + grp;
-            if (i < a.B && bt.hi[b] - bt.lo[b] == 1 && bt.lo[b] >= 0 && (int64_t)bt.hi[b] <= a.L) {
-                if ((int64_t)bt.lo[b] != g0 + i) idx[b] = __ldg(a.indices + bt.lo[b]);
-                idx[b] = checked_index(idx[b], nrows, a.status);
-                bt.one |= 1u << b;
-                const float4 *row = reinterpret_cast<const float4 *>(tbl + (int64_t)idx[b] * a.D);
-#pragma unroll
-                for (int c = 0; c < CH; ++c) {
-                    const int c4 = c * LPR + lane;
-                    if (c4 < d4) dq_cp_async16(slot<CH>(s_buf, stage, b, c), row + c4);
-                }
-            }
-        }
-        dq_cp_async_commit();
-    };
-
-    const int step = gridDim.x * TILE;
-    int ib = blockIdx.x * TILE;
-    if (ib >= a.B) return;
-    Batch cur, nxt;
-    int stage = 0;
-    issue(ib, 0, cur);
-    for (; ib < a.B; ib += step) {
-        const bool more = ib + step < a.B;
-        if (more) { issue(ib + step, stage ^ 1, nxt); dq_cp_async_wait<1>(); }
-        else dq_cp_async_wait<0>();
-#pragma unroll
-        for (int b = 0; b < NBOf<CH>::v; ++b) {
-            const int i = ib + b * GPB + grp;
-            if ((cur.one >> b) & 1u) {
-#pragma unroll
-                for (int c = 0; c < CH; ++c) {
-                    const int c4 = c * LPR + lane;
-                    if (c4 < d4) {
-                        float4 cd;
-                        const float4 f = fq4(*slot<CH>(s_buf, stage, b, c), qs, cd);
-                        reinterpret_cast<float4 *>(a.out + ((int64_t)i * a.T + t) * a.D)[c4] = f;
-                        if (a.codes_out) store_codes(a.codes_out, cur.lo[b], a.D, c4, cd);
-                    }
-                }
-            }
-        }
-        bool rare = false;
-#pragma unroll
-        for (int b = 0; b < NBOf<CH>::v; ++b) rare |= (ib + b * GPB + grp < a.B) && !((cur.one >> b) & 1u);
-        if (rare) {
-            // bags of this batch that are empty, multi-index or out of range: the general routine
-            // reuses this thread's staging slots of both stages, so the prefetched batch is re-issued
-            dq_cp_async_wait<0>();
-#pragma unroll
-            for (int b = 0; b < NBOf<CH>::v; ++b) {
-                const int i = ib + b * GPB + grp;
-                if (i < a.B && !((cur.one >> b) & 1u))
-                    pool_bag_rare<LPR, CH>(a, tbl, nrows, qs, cur.lo[b], cur.hi[b],
-                                           a.out + ((int64_t)i * a.T + t) * a.D, lane, s_buf);
-            }
-            if (more) issue(ib + step, stage ^ 1, nxt);
-        }
-        cur = nxt;
-        stage ^= 1;
-    }
-}
-
-template <int LPR, int CH>
-__global__ void __launch_bounds__(FW_THREADS)
-fwd_bags_kernel(const FwdArgs a)
-{
-    extern __shared__ float4 s_buf[];
-    constexpr int GPB = FW_THREADS / LPR;
-    const int t = blockIdx.y;
-    const int lane = threadIdx.x % LPR;
-    const int grp = threadIdx.x / LPR;
-    const QuantScale qs = dq_make_scale(__ldg(a.scales + t), __ldg(a.bits + t));
-    const int64_t r0 = __ldg(a.row_off + t);
-    const int64_t nrows = __ldg(a.row_off + t + 1) - r0;
-    const float *tbl = a.tables + r0 * a.D;
-    const int64_t g0 = (int64_t)t * a.B;
-    for (int i = blockIdx.x * GPB + grp; i < a.B; i += gridDim.x * GPB) {
-        const int32_t lo = __ldg(a.offsets + g0 + i), hi = __ldg(a.offsets + g0 + i + 1);
-        pool_bag<LPR, CH>(a, tbl, nrows, qs, lo, hi, a.out + ((int64_t)i * a.T + t) * a.D, lane, s_buf);
-    }
-}
-
-template <int LPR, int CH>
-int launch(dqrm_ctx *ctx, const FwdArgs &a, cudaStream_t st)
+template <int LPR, int CH, bool EXACT>
+int launch2(dqrm_ctx *ctx, const FwdArgs &a, cudaStream_t st)
 {
     constexpr int GPB = FW_THREADS / LPR;
-    constexpr size_t SMEM = sizeof(float4) * FW_STAGES * NBOf<CH>::v * CH * FW_THREADS;   // 32 KB * CH
-    static bool raised = false;
-    if (SMEM > 48 * 1024 && !raised) {
-        DQRM_CUDA_TRY(ctx, cudaFuncSetAttribute(fwd_onehot_kernel<LPR, CH>,
-                                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM));
-        DQRM_CUDA_TRY(ctx, cudaFuncSetAttribute(fwd_bags_kernel<LPR, CH>,
-                                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM));
-        raised = true;
-    }
-    const bool onehot = a.L == (int64_t)a.T * a.B;
-    const int per_block = onehot ? GPB * NBOf<CH>::v : GPB;
+    // the one-index kernel does not emit codes; a caller that asks for them gets the general kernel
+    const bool onehot = a.L == (int64_t)a.T * a.B && a.codes_out == nullptr;
+    const int per_block = onehot ? GPB * NBOf<LPR, CH>::v : GPB;
     int bx = (a.B + per_block - 1) / per_block;
     const int cap = (ctx->num_sms * 32 + ctx->T - 1) / ctx->T;     // a few waves over all tables
     if (bx > cap) bx = cap;
     if (bx < 1) bx = 1;
     dim3 grid((unsigned)bx, (unsigned)ctx->T);
-    if (onehot) fwd_onehot_kernel<LPR, CH><<<grid, FW_THREADS, SMEM, st>>>(a);
-    else fwd_bags_kernel<LPR, CH><<<grid, FW_THREADS, SMEM, st>>>(a);
+    if (onehot) fwd_onehot_kernel<LPR, CH, EXACT><<<grid, FW_THREADS, 0, st>>>(a);
+    else fwd_bags_kernel<LPR, CH, EXACT><<<grid, FW_THREADS, 0, st>>>(a);
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
     dq_mark(ctx, st, DQ_K_FWD);
     return DQRM_OK;
+}
+
+template <int LPR, int CH>
+int launch(dqrm_ctx *ctx, const FwdArgs &a, cudaStream_t st)
+{
+    if (a.D == 4 * LPR * CH) return launch2<LPR, CH, true>(ctx, a, st);
+    return launch2<LPR, CH, false>(ctx, a, st);
 }
 
 }  // namespace
