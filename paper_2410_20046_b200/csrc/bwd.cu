@@ -331,26 +331,30 @@ seg_emit_kernel(const u32 *__restrict__ keys, int64_t L, const u32 *__restrict__
 }
 
 // ---------------------------------------------------------------------------------
-template <int LPR, int CH>
+// RL/RV/RC: lanes per row, floats per lane vector and vectors per lane of the reduce kernel;
+// LPR/CH: the same for the fix-up kernels (always 128-bit vectors)
+template <int RL, int RV, int RC, int LPR, int CH>
 int launch_reduce(dqrm_ctx *ctx, const Layout &y, char *ws, const u32 *keys, const u32 *vals,
                   const float *grad_out, float *grad_rows, int64_t L, int64_t G, cudaStream_t st)
 {
     using namespace segred;
     const size_t smem = (size_t)(ctx->T + 1) * sizeof(int64_t);
     const int64_t cap = (int64_t)ctx->num_sms * 8;
-    int64_t blocks = (y.num_chunks + 7) / 8;                 // one warp per chunk
+    const int64_t gpb = 256 / RL;                            // one lane group per chunk
+    int64_t blocks = (y.num_chunks + gpb - 1) / gpb;
     int grid = (int)(blocks < 1 ? 1 : (blocks > cap ? cap : blocks));
     u32 *counters = reinterpret_cast<u32 *>(ws + y.counters);
     u32 *absmax = reinterpret_cast<u32 *>(ws + y.absmax);
     const u32 *seg_start = reinterpret_cast<const u32 *>(ws + y.seg_start);
     double *partials = reinterpret_cast<double *>(ws + y.partials);
     u32 *long_list = reinterpret_cast<u32 *>(ws + y.long_list);
-    seg_reduce_kernel<LPR, CH><<<grid, 256, smem, st>>>(
+    seg_reduce_kernel<RL, RV, RC><<<grid, 256, smem, st>>>(
         keys, vals, seg_start, reinterpret_cast<const u32 *>(ws + y.chunk_first), grad_out, grad_rows, partials,
         long_list, counters, absmax, ctx->d_row_off, ctx->T, ctx->D, L, G, y.num_chunks, ctx->d_status);
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
     dq_mark(ctx, st, DQ_K_SEG_REDUCE);
-    int fgrid = (int)(blocks < (int64_t)ctx->num_sms * 4 ? (blocks < 1 ? 1 : blocks) : (int64_t)ctx->num_sms * 4);
+    int64_t fblocks = (y.num_chunks + 7) / 8;                // at most one cut segment per chunk, a warp each
+    int fgrid = (int)(fblocks < (int64_t)ctx->num_sms * 4 ? (fblocks < 1 ? 1 : fblocks) : (int64_t)ctx->num_sms * 4);
     seg_fixup_kernel<LPR, CH><<<fgrid, 256, smem, st>>>(keys, seg_start, partials, long_list, counters, grad_rows,
                                                         absmax, ctx->d_row_off, ctx->T, ctx->D);
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
@@ -436,16 +440,17 @@ int dq_launch_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, 
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
     dq_mark(ctx, st, DQ_K_SEG_EMIT);
 
-    const int d4 = ctx->D / 4;
-#define DQ_RED(LPR, CH) return launch_reduce<LPR, CH>(ctx, y, ws, skeys, svals, grad_out, grad_rows, L, G, st)
-    if (d4 <= 1) DQ_RED(1, 1);
-    if (d4 <= 2) DQ_RED(2, 1);
-    if (d4 <= 4) DQ_RED(4, 1);
-    if (d4 <= 8) DQ_RED(8, 1);
-    if (d4 <= 16) DQ_RED(16, 1);
-    if (d4 <= 32) DQ_RED(32, 1);
-    if (d4 <= 64) DQ_RED(32, 2);
-    if (d4 <= 128) DQ_RED(32, 4);
-    DQ_RED(32, 8);
+    const int D = ctx->D, d4 = D / 4;
+#define DQ_RED(RL, RV, RC, LPR, CH) \
+    return launch_reduce<RL, RV, RC, LPR, CH>(ctx, y, ws, skeys, svals, grad_out, grad_rows, L, G, st)
+    if (D <= 4) DQ_RED(4, 1, 1, 1, 1);
+    if (D <= 8) DQ_RED(8, 1, 1, 2, 1);
+    if (D <= 16) DQ_RED(16, 1, 1, 4, 1);
+    if (D <= 32) DQ_RED(16, 2, 1, 8, 1);
+    if (D <= 64) DQ_RED(16, 4, 1, 16, 1);
+    if (d4 <= 32) DQ_RED(32, 4, 1, 32, 1);
+    if (d4 <= 64) DQ_RED(32, 4, 2, 32, 2);
+    if (d4 <= 128) DQ_RED(32, 4, 4, 32, 4);
+    DQ_RED(32, 4, 8, 32, 8);
 #undef DQ_RED
 }

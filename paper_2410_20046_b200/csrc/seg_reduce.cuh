@@ -3,11 +3,9 @@
 //
 // Input: keys[L] (arena rows, ascending), vals[L] (row of grad_out for each lookup, in
 // stable order), chunk_first[c] = index of the segment that holds sorted entry 32*c,
-// seg_start[U+1].  One warp owns one chunk of 32 sorted entries.  The warp's SG = 32/LPR
-// lane groups each gather one upstream-gradient row per step (LPR lanes x 128 bit), the
-// rows of a step are combined by a segmented warp-shuffle scan keyed on the row id, and a
-// carry links the steps.  All sums are FP64 and have a shape fixed by the entry
-// positions, so results are reproducible.  A run that is a whole segment is rounded to
+// seg_start[U+1].  One lane group owns one chunk of 32 sorted entries and walks it in
+// order with a few upstream-gradient rows in flight.  All sums are FP64 and have a shape
+// fixed by the entry positions, so results are reproducible.  A run that is a whole segment is rounded to
 // FP32 and written; a run cut by the chunk boundary leaves an FP64 partial and the
 // segment is finished by one of the fix-up kernels (a warp for up to 32 pieces, a block
 // beyond that).  The per-table abs-max of the rounded sums is collected on the way.
@@ -83,7 +81,25 @@ __device__ __forceinline__ float round_store(const double (&acc)[CH][4], float *
     return m;
 }
 
-template <int LPR, int CH>
+// VEC consecutive floats (1, 2 or 4) as one load
+template <int VEC> struct Vec;
+template <> struct Vec<1> { typedef float type; };
+template <> struct Vec<2> { typedef float2 type; };
+template <> struct Vec<4> { typedef float4 type; };
+
+template <int VEC>
+__device__ __forceinline__ void vec_add(double (&acc)[VEC], const typename Vec<VEC>::type &v)
+{
+    if constexpr (VEC == 1) { acc[0] += (double)v; }
+    else if constexpr (VEC == 2) { acc[0] += (double)v.x; acc[1] += (double)v.y; }
+    else { acc[0] += (double)v.x; acc[1] += (double)v.y; acc[2] += (double)v.z; acc[3] += (double)v.w; }
+}
+
+// One lane group (LPR lanes) owns one chunk of 32 sorted entries and walks it in order,
+// NB upstream-gradient rows in flight at a time.  Lane `lane` holds, for ch < CH, the VEC
+// consecutive features starting at (ch*LPR + lane)*VEC; narrow rows use VEC = 1 or 2 so
+// that a row is still spread over 16 lanes and small feature sizes keep enough threads.
+template <int LPR, int VEC, int CH>
 __global__ void __launch_bounds__(256)
 seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
                   const u32 *__restrict__ seg_start, const u32 *__restrict__ chunk_first,
@@ -97,135 +113,119 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
     for (int t = threadIdx.x; t <= T; t += blockDim.x) s_off[t] = row_off[t];
     __syncthreads();
 
-    constexpr int SG = 32 / LPR;                 // lane groups per warp = entries per step
-    constexpr int STEPS = CHUNK / SG;            // steps per chunk
-    constexpr int PRE = STEPS < 8 ? STEPS : 8;   // steps whose rows are loaded together
-    const int d4 = D >> 2;
-    const int wl = threadIdx.x & 31;
-    const int sub = wl / LPR, lane = wl % LPR;
-    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    typedef typename Vec<VEC>::type vec_t;
+    constexpr int NB = 4;
+    const int dv = D / VEC;                       // vectors per row
+    const int lane = threadIdx.x % LPR;
+    const int64_t group = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / LPR;
+    const int64_t n_groups = (int64_t)gridDim.x * blockDim.x / LPR;
     AbsmaxTracker tr;
+    bool bad = false;
 
-    for (int64_t c = warp; c < num_chunks; c += n_warps) {
+    for (int64_t c = group; c < num_chunks; c += n_groups) {
         const int64_t i0 = c * CHUNK;
-        const int n = (int)min((int64_t)CHUNK, L - i0);
-        u32 my_key = 0xFFFFFFFFu, my_val = 0u;
-        if (wl < n) {
-            my_key = keys[i0 + wl];
-            my_val = vals[i0 + wl];
-            if ((int64_t)my_val >= G) { dq_report(status, DQRM_ERR_INDEX_RANGE); my_val = 0u; }
-        }
-        const bool has_prev = i0 > 0, has_next = i0 + n < L;
-        const u32 prev_key = has_prev ? keys[i0 - 1] : 0u;
-        const u32 next_key = has_next ? keys[i0 + n] : 0u;
-        const u32 up_key = __shfl_up_sync(0xffffffffu, my_key, 1);
-        const bool head = (wl < n) && (wl == 0 ? (!has_prev || my_key != prev_key) : (my_key != up_key));
-        const u32 headmask = __ballot_sync(0xffffffffu, head);
-        const u32 down_key = __shfl_down_sync(0xffffffffu, my_key, 1);
-        const bool tail = (wl < n) && (wl == n - 1 || down_key != my_key);
-        const u32 tailmask = __ballot_sync(0xffffffffu, tail);
-        const bool continues_after = has_next && next_key == __shfl_sync(0xffffffffu, my_key, n - 1);
-        const u32 u0 = chunk_first[c];
+        const int64_t i1 = min(i0 + (int64_t)CHUNK, L);
+        u32 u = chunk_first[c];
+        u32 cur_key = keys[i0];
+        int64_t run_start = i0;
+        double acc[CH][VEC];
+#pragma unroll
+        for (int ch = 0; ch < CH; ++ch)
+#pragma unroll
+            for (int q = 0; q < VEC; ++q) acc[ch][q] = 0.0;
 
-        double carry[CH][4];
-        u32 carry_key = 0xFFFFFFFFu;
-#pragma unroll
-        for (int ch = 0; ch < CH; ++ch) carry[ch][0] = carry[ch][1] = carry[ch][2] = carry[ch][3] = 0.0;
-
-#pragma unroll 1
-        for (int st0 = 0; st0 < STEPS; st0 += PRE) {
-            float4 row[PRE][CH];
-#pragma unroll
-            for (int p = 0; p < PRE; ++p) {
-                const int e = (st0 + p) * SG + sub;
-                const u32 v = __shfl_sync(0xffffffffu, my_val, e & 31);
-                if (e < n) {
-                    const float4 *src = reinterpret_cast<const float4 *>(grad_out + (int64_t)v * D);
-#pragma unroll
-                    for (int ch = 0; ch < CH; ++ch) {
-                        int c4 = ch * LPR + lane;
-                        if (c4 < d4) row[p][ch] = __ldg(src + c4);
-                    }
-                }
-            }
-#pragma unroll
-            for (int p = 0; p < PRE; ++p) {
-                const int e = (st0 + p) * SG + sub;
-                const bool valid = e < n;
-                const u32 key_e = __shfl_sync(0xffffffffu, my_key, e & 31);
-                double acc[CH][4];
+        // closes run [a, b) of segment u; runs strictly inside the chunk are whole segments
+        auto flush = [&](int64_t a, int64_t b) {
+            bool begins = true, ends = true;
+            if (a == i0) begins = (seg_start[u] == (u32)a);
+            if (b == i1) ends = (seg_start[u + 1] == (u32)b);
+            if (begins && ends) {
+                float m = 0.f;
 #pragma unroll
                 for (int ch = 0; ch < CH; ++ch) {
-                    int c4 = ch * LPR + lane;
-                    bool on = valid && c4 < d4;
-                    acc[ch][0] = on ? (double)row[p][ch].x : 0.0;
-                    acc[ch][1] = on ? (double)row[p][ch].y : 0.0;
-                    acc[ch][2] = on ? (double)row[p][ch].z : 0.0;
-                    acc[ch][3] = on ? (double)row[p][ch].w : 0.0;
-                }
-                // segmented inclusive scan over the SG entries of this step
-#pragma unroll
-                for (int o = 1; o < SG; o <<= 1) {
-                    const u32 key_o = __shfl_up_sync(0xffffffffu, key_e, o * LPR);
-                    const bool take = valid && sub >= o && key_o == key_e;
-#pragma unroll
-                    for (int ch = 0; ch < CH; ++ch)
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            double other = __shfl_up_sync(0xffffffffu, acc[ch][q], o * LPR);
-                            if (take) acc[ch][q] += other;
+                    const int cv = ch * LPR + lane;
+                    if (cv < dv) {
+                        float *dst = grad_rows + (int64_t)u * D + cv * VEC;
+                        if constexpr (VEC == 1) { float r = (float)acc[ch][0]; *dst = r; m = fmaxf(m, fabsf(r)); }
+                        else if constexpr (VEC == 2) {
+                            float2 r = make_float2((float)acc[ch][0], (float)acc[ch][1]);
+                            *reinterpret_cast<float2 *>(dst) = r;
+                            m = fmaxf(m, fmaxf(fabsf(r.x), fabsf(r.y)));
+                        } else {
+                            float4 r = make_float4((float)acc[ch][0], (float)acc[ch][1], (float)acc[ch][2], (float)acc[ch][3]);
+                            *reinterpret_cast<float4 *>(dst) = r;
+                            m = fmaxf(fmaxf(m, fmaxf(fabsf(r.x), fabsf(r.y))), fmaxf(fabsf(r.z), fabsf(r.w)));
                         }
+                    }
                 }
-                // link to the previous step
-                if (valid && key_e == carry_key) {
+                absmax_note<LPR>(tr, cur_key, m, s_off, T, absmax);
+            } else {
+                double *pdst = partials + ((size_t)c * 2 + (begins ? 1 : 0)) * D;
 #pragma unroll
-                    for (int ch = 0; ch < CH; ++ch)
+                for (int ch = 0; ch < CH; ++ch) {
+                    const int cv = ch * LPR + lane;
+                    if (cv < dv) {
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) acc[ch][q] += carry[ch][q];
+                        for (int q = 0; q < VEC; ++q) pdst[cv * VEC + q] = acc[ch][q];
+                    }
                 }
-                // the last lane group's running sum is the next step's carry
-                carry_key = __shfl_sync(0xffffffffu, valid ? key_e : 0xFFFFFFFFu, (SG - 1) * LPR + lane);
-#pragma unroll
-                for (int ch = 0; ch < CH; ++ch)
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        carry[ch][q] = __shfl_sync(0xffffffffu, acc[ch][q], (SG - 1) * LPR + lane);
+                if (begins && lane == 0) {
+                    const u32 sa = seg_start[u], sb = seg_start[u + 1];
+                    const u32 npieces = (sb - 1) / CHUNK - sa / CHUNK + 1;
+                    if (npieces > BIG_PIECES)
+                        long_list[num_chunks - 1 - atomicAdd(&counters[CNT_BIG], 1u)] = u;
+                    else
+                        long_list[atomicAdd(&counters[CNT_LONG], 1u)] = u;
+                }
+            }
+        };
 
-                if (valid && ((tailmask >> e) & 1u)) {
-                    // entry e closes a run inside this chunk
-                    const u32 below = headmask & (0xffffffffu >> (31 - e));      // heads at entries 0..e
-                    const bool begins = below != 0u;                            // the run's head is in this chunk
-                    const u32 u = u0 + __popc(below & ~1u);
-                    const bool ends = !(e == n - 1 && continues_after);
-                    if (begins && ends) {
-                        float m = round_store<CH>(acc, grad_rows + (int64_t)u * D, lane, LPR, d4);
-                        absmax_note<LPR>(tr, key_e, m, s_off, T, absmax);
-                    } else {
-                        double *pdst = partials + ((size_t)c * 2 + (begins ? 1 : 0)) * D;
+        for (int64_t ib = i0; ib < i1; ib += NB) {
+            u32 k[NB], v[NB];
 #pragma unroll
-                        for (int ch = 0; ch < CH; ++ch) {
-                            int c4 = ch * LPR + lane;
-                            if (c4 < d4) {
-                                *reinterpret_cast<double2 *>(pdst + 4 * c4) = make_double2(acc[ch][0], acc[ch][1]);
-                                *reinterpret_cast<double2 *>(pdst + 4 * c4 + 2) = make_double2(acc[ch][2], acc[ch][3]);
-                            }
-                        }
-                        if (begins && lane == 0) {
-                            const u32 a = seg_start[u], b = seg_start[u + 1];
-                            const u32 npieces = (b - 1) / CHUNK - a / CHUNK + 1;
-                            if (npieces > BIG_PIECES)
-                                long_list[num_chunks - 1 - atomicAdd(&counters[CNT_BIG], 1u)] = u;
-                            else
-                                long_list[atomicAdd(&counters[CNT_LONG], 1u)] = u;
-                        }
+            for (int e = 0; e < NB; ++e) {
+                const bool ok = ib + e < i1;
+                k[e] = ok ? keys[ib + e] : 0u;
+                v[e] = ok ? vals[ib + e] : 0u;
+                if (ok && (int64_t)v[e] >= G) { bad = true; v[e] = 0u; }
+            }
+            vec_t r[NB][CH];
+#pragma unroll
+            for (int e = 0; e < NB; ++e) {
+                if (ib + e < i1) {
+                    const vec_t *src = reinterpret_cast<const vec_t *>(grad_out + (int64_t)v[e] * D);
+#pragma unroll
+                    for (int ch = 0; ch < CH; ++ch) {
+                        const int cv = ch * LPR + lane;
+                        if (cv < dv) r[e][ch] = __ldg(src + cv);
+                    }
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < NB; ++e) {
+                if (ib + e < i1) {
+                    if (k[e] != cur_key) {
+                        flush(run_start, ib + e);
+                        u += 1;
+                        cur_key = k[e];
+                        run_start = ib + e;
+#pragma unroll
+                        for (int ch = 0; ch < CH; ++ch)
+#pragma unroll
+                            for (int q = 0; q < VEC; ++q) acc[ch][q] = 0.0;
+                    }
+#pragma unroll
+                    for (int ch = 0; ch < CH; ++ch) {
+                        const int cv = ch * LPR + lane;
+                        if (cv < dv) vec_add<VEC>(acc[ch], r[e][ch]);
                     }
                 }
             }
         }
+        flush(run_start, i1);
     }
-    // every lane group flushes its last table's maximum (group-uniform)
-    absmax_push<LPR>(tr, absmax);
+    absmax_push<LPR>(tr, absmax);      // group-uniform: all lanes of a group walk the same chunks
+    if (bad) dq_report(status, DQRM_ERR_INDEX_RANGE);
 }
 
 // pieces of cut segment [a, e): chunk a/32 holds the first (slot 1), later chunks slot 0
