@@ -114,9 +114,12 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
     __syncthreads();
 
     typedef typename Vec<VEC>::type vec_t;
-    constexpr int NB = 4;
+    constexpr int NB = VEC == 4 ? 4 : 8;          // rows in flight per lane
+    constexpr int EPL = CHUNK / LPR;              // chunk entries whose key and payload a lane holds
     const int dv = D / VEC;                       // vectors per row
     const int lane = threadIdx.x % LPR;
+    const u32 gmask = group_mask<LPR>();
+    const int gbase = (threadIdx.x & 31) / LPR * LPR;
     const int64_t group = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / LPR;
     const int64_t n_groups = (int64_t)gridDim.x * blockDim.x / LPR;
     AbsmaxTracker tr;
@@ -125,8 +128,26 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
     for (int64_t c = group; c < num_chunks; c += n_groups) {
         const int64_t i0 = c * CHUNK;
         const int64_t i1 = min(i0 + (int64_t)CHUNK, L);
+        // the chunk's keys and payloads: one coalesced load, then broadcast by shuffles
+        u32 kreg[EPL], vreg[EPL];
+#pragma unroll
+        for (int j = 0; j < EPL; ++j) {
+            const int64_t i = i0 + j * LPR + lane;
+            kreg[j] = i < i1 ? keys[i] : 0xFFFFFFFFu;
+            vreg[j] = i < i1 ? vals[i] : 0u;
+            if (i < i1 && (int64_t)vreg[j] >= G) { bad = true; vreg[j] = 0u; }
+        }
+        auto bcast = [&](const u32 (&reg)[EPL], int e) {     // entry e of the chunk, e uniform in the group
+            u32 r = reg[0];
+#pragma unroll
+            for (int j = 1; j < EPL; ++j) if (e / LPR == j) r = reg[j];
+            return __shfl_sync(gmask, r, gbase + (e % LPR));
+        };
+        // does the chunk's first run begin here, does its last run end here?  (neighbouring keys)
+        const bool first_begins = (i0 == 0) || (keys[i0 - 1] != bcast(kreg, 0));
+        const bool last_ends = (i1 == L) || (keys[i1] != bcast(kreg, (int)(i1 - i0) - 1));
         u32 u = chunk_first[c];
-        u32 cur_key = keys[i0];
+        u32 cur_key = bcast(kreg, 0);
         int64_t run_start = i0;
         double acc[CH][VEC];
 #pragma unroll
@@ -136,9 +157,8 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
 
         // closes run [a, b) of segment u; runs strictly inside the chunk are whole segments
         auto flush = [&](int64_t a, int64_t b) {
-            bool begins = true, ends = true;
-            if (a == i0) begins = (seg_start[u] == (u32)a);
-            if (b == i1) ends = (seg_start[u + 1] == (u32)b);
+            const bool begins = (a != i0) || first_begins;
+            const bool ends = (b != i1) || last_ends;
             if (begins && ends) {
                 float m = 0.f;
 #pragma unroll
@@ -184,10 +204,9 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
             u32 k[NB], v[NB];
 #pragma unroll
             for (int e = 0; e < NB; ++e) {
-                const bool ok = ib + e < i1;
-                k[e] = ok ? keys[ib + e] : 0u;
-                v[e] = ok ? vals[ib + e] : 0u;
-                if (ok && (int64_t)v[e] >= G) { bad = true; v[e] = 0u; }
+                const int ec = (int)(ib - i0) + e;           // < CHUNK because NB divides CHUNK
+                k[e] = bcast(kreg, ec);
+                v[e] = bcast(vreg, ec);
             }
             vec_t r[NB][CH];
 #pragma unroll
