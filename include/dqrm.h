@@ -192,6 +192,13 @@ int dqrm_train_step_host(dqrm_ctx *ctx, float *tables, const int32_t *h_indices,
 int dqrm_grad_quant_int8_static(int T, int D, const float *grad_rows, const int32_t *uniq_off,
                                 int8_t *codes, float *grad_scales, void *stream);
 
+/* ---- choice of the backward's sort (no counterpart in the paper) --------------------
+ * dqrm_emb_bwd and dqrm_train_step order the batch's lookups by row before they sum
+ * duplicates.  path 0 (default): one thread-block cluster per table sorts that table's
+ * lookups in distributed shared memory.  path 1: one global least-significant-digit radix
+ * sort over all tables.  Both give identical outputs; the choice only affects speed. */
+int dqrm_set_sort_path(dqrm_ctx *ctx, int path);
+
 /* ---- quantiser self-check (no counterpart in the paper) ----------------------------
  * The kernels evaluate Q(x; s, b) without the IEEE division sequence where a scale is
  * shared by many elements, and fall back to the division near rounding ties.  This call

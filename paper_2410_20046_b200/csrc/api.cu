@@ -131,6 +131,13 @@ int dqrm_last_cuda_error(const dqrm_ctx *ctx) { return ctx ? ctx->last_cuda_erro
 
 int64_t dqrm_launch_count(const dqrm_ctx *ctx) { return ctx ? ctx->launch_count : 0; }
 
+int dqrm_set_sort_path(dqrm_ctx *ctx, int path)
+{
+    if (!ctx || path < 0 || path > 1) return DQRM_ERR_INVALID_ARG;
+    ctx->sort_path = path;
+    return DQRM_OK;
+}
+
 int dqrm_profile_begin(dqrm_ctx *ctx, void *stream)
 {
     if (!ctx) return DQRM_ERR_INVALID_ARG;
@@ -170,7 +177,7 @@ const char *dqrm_kernel_name(int kernel_id)
         "begin", "refresh_kernel", "fwd_kernel", "memset", "prepare_kernel", "sort_scan_kernel",
         "sort_scatter_kernel", "seg_count_kernel", "seg_emit_kernel", "seg_reduce_kernel", "seg_fixup_kernel",
         "absmax_kernel", "row_stream_kernel<quant>", "row_stream_kernel<update>", "row_stream_kernel<fused>",
-        "copy", "seg_fixup_big_kernel"};
+        "copy", "seg_fixup_big_kernel", "cluster_sort_kernel"};
     return (kernel_id >= 0 && kernel_id < DQ_K_COUNT) ? names[kernel_id] : "?";
 }
 

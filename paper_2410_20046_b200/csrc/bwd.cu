@@ -21,6 +21,7 @@
 // quantiser) is folded into the last two kernels.
 #include "common.cuh"
 #include "seg_reduce.cuh"
+#include "cluster_sort.cuh"
 
 namespace {
 
@@ -406,6 +407,47 @@ int dq_launch_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, 
     u32 *vals[2] = {reinterpret_cast<u32 *>(ws + y.vals_a), reinterpret_cast<u32 *>(ws + y.vals_b)};
     u32 *thist[2] = {reinterpret_cast<u32 *>(ws + y.tilehist_a), reinterpret_cast<u32 *>(ws + y.tilehist_b)};
     u32 *ghist = reinterpret_cast<u32 *>(ws + y.ghist);
+    const u32 *skeys = nullptr, *svals = nullptr;
+    bool sorted = false;
+    if (ctx->sort_path != 1) {
+        // one eight-block cluster per table; falls through to the global radix sort if the launch is refused
+        csort::Args ca;
+        ca.indices = indices; ca.offsets = offsets; ca.row_off = ctx->d_row_off;
+        ca.T = ctx->T; ca.B = B; ca.L = L;
+        ca.keys_out = keys[0]; ca.vals_out = vals[0];
+        ca.gk[0] = keys[0]; ca.gk[1] = keys[1]; ca.gv[0] = vals[0]; ca.gv[1] = vals[1];
+        ca.cap = csort::choose_cap((L + ctx->T - 1) / ctx->T);
+        ca.status = ctx->d_status;
+        const size_t smem = csort::smem_bytes(ca.cap);
+        static bool raised = false;
+        cudaError_t e = cudaSuccess;
+        if (!raised) {
+            e = cudaFuncSetAttribute(csort::cluster_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)csort::smem_bytes(12288));
+            raised = (e == cudaSuccess);
+        }
+        if (e == cudaSuccess) {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3((unsigned)(ctx->T * csort::CLUSTER));
+            cfg.blockDim = dim3(csort::THREADS);
+            cfg.dynamicSmemBytes = smem;
+            cfg.stream = st;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = csort::CLUSTER; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr; cfg.numAttrs = 1;
+            e = cudaLaunchKernelEx(&cfg, csort::cluster_sort_kernel, ca);
+        }
+        if (e == cudaSuccess) {
+            dq_mark(ctx, st, DQ_K_CLUSTER_SORT);
+            skeys = keys[0]; svals = vals[0];
+            sorted = true;
+        } else {
+            (void)cudaGetLastError();
+            ctx->last_cuda_error = (int)e;
+        }
+    }
+    if (!sorted) {
     {
         int64_t blocks = (G + 255) / 256;
         int64_t cap = (int64_t)ctx->num_sms * 8;
@@ -429,7 +471,8 @@ int dq_launch_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, 
         DQRM_CUDA_TRY(ctx, cudaGetLastError());
         dq_mark(ctx, st, DQ_K_SORT_SCATTER);
     }
-    const u32 *skeys = keys[y.passes & 1], *svals = vals[y.passes & 1];
+        skeys = keys[y.passes & 1]; svals = vals[y.passes & 1];
+    }
     seg_count_kernel<<<(unsigned)y.num_tiles, ST_THREADS, 0, st>>>(skeys, L, reinterpret_cast<u32 *>(ws + y.tile_heads));
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
     dq_mark(ctx, st, DQ_K_SEG_COUNT);

@@ -1,0 +1,229 @@
+// Per-table stable sort of a batch's lookups by row, one thread-block cluster per table.
+//
+// The lookups of a batch arrive table-major, so sorting them by arena row is T independent
+// sorts of a few thousand to a few tens of thousands of keys each.  A cluster of eight
+// blocks owns one table: every block holds one eighth of the table's (row, payload) pairs
+// in shared memory, and a least-significant-digit radix sort (8-bit digits, only as many
+// passes as the table's row count needs) moves the pairs between the blocks' shared
+// memories with distributed-shared-memory stores.  Per pass: per-warp digit counts over
+// the block's slice (match_any, stable), the eight per-block histograms are exchanged
+// through DSMEM, every block derives its scatter offsets, ranks its slice again and
+// scatters.  Cluster barriers separate the phases; no block waits on anything else.
+// Tables whose lookups do not fit the shared-memory slices use the same algorithm on
+// global staging buffers.  The result - keys (arena rows) ascending, payloads (rows of
+// grad_out) in the original order within equal keys - is written table-major, which is
+// the globally sorted order the segmented reduction expects.
+#pragma once
+#include <cooperative_groups.h>
+#include "common.cuh"
+
+namespace csort {
+
+namespace cg = cooperative_groups;
+
+constexpr int THREADS = 256;
+constexpr int WARPS = THREADS / 32;
+constexpr int CLUSTER = 8;
+constexpr int BINS = 256;
+
+struct Args {
+    const int32_t *indices;
+    const int32_t *offsets;
+    const int64_t *row_off;
+    int T, B;
+    int64_t L;
+    u32 *keys_out, *vals_out;       // [L] sorted result
+    u32 *gk[2], *gv[2];             // [L] global staging (tables too large for shared memory)
+    int cap;                        // pairs per block that fit in shared memory
+    int *status;
+};
+
+__device__ __forceinline__ u32 *remote(cg::cluster_group &cluster, u32 *p, unsigned rank)
+{
+    return cluster.map_shared_rank(p, rank);
+}
+
+__global__ void __launch_bounds__(THREADS)
+cluster_sort_kernel(const Args a)
+{
+    extern __shared__ u32 s_dyn[];                 // kbuf[2][cap], vbuf[2][cap]
+    __shared__ u32 s_cnt[WARPS][BINS];
+    __shared__ u32 s_hist[BINS];
+    __shared__ u32 s_scan[WARPS];
+    __shared__ int s_flag;
+
+    cg::cluster_group cluster = cg::this_cluster();
+    const unsigned c = cluster.block_rank();
+    const int t = blockIdx.x / CLUSTER;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const u32 lt = (1u << lane) - 1u;
+
+    int64_t tb0 = __ldg(a.offsets + (int64_t)t * a.B), tb1 = __ldg(a.offsets + (int64_t)(t + 1) * a.B);
+    if (tb0 < 0 || tb1 < tb0 || tb1 > a.L) {
+        if (threadIdx.x == 0 && c == 0) dq_report(a.status, DQRM_ERR_INDEX_RANGE);
+        return;                                    // uniform over the cluster
+    }
+    const int64_t n = tb1 - tb0;
+    if (n == 0) return;
+    const int64_t r0 = __ldg(a.row_off + t);
+    const int64_t nrows = __ldg(a.row_off + t + 1) - r0;
+    const int npc = (int)(((n + CLUSTER - 1) / CLUSTER + 31) / 32 * 32);      // pairs per block
+    const bool in_smem = npc <= a.cap;
+    const int my_n = (int)max((int64_t)0, min((int64_t)npc, n - (int64_t)c * npc));
+
+    // buffers of this block for stage s (shared memory slices, or this block's part of the global staging)
+    u32 *kb[2], *vb[2];
+    if (in_smem) {
+        kb[0] = s_dyn; kb[1] = s_dyn + a.cap; vb[0] = s_dyn + 2 * a.cap; vb[1] = s_dyn + 3 * a.cap;
+    } else {
+        for (int s = 0; s < 2; ++s) { kb[s] = a.gk[s] + tb0 + (int64_t)c * npc; vb[s] = a.gv[s] + tb0 + (int64_t)c * npc; }
+    }
+
+    // ---- are this table's bags all one-index bags in order (offsets = identity)? ----
+    {
+        if (threadIdx.x == 0) s_flag = 1;
+        __syncthreads();
+        int ok = 1;
+        const int per = (a.B + CLUSTER - 1) / CLUSTER;
+        const int b0 = c * per, b1 = min(a.B, b0 + per);
+        if (n != a.B) ok = 0;
+        else
+            for (int i = b0 + threadIdx.x; i < b1; i += THREADS)
+                if ((int64_t)__ldg(a.offsets + (int64_t)t * a.B + i) != tb0 + i) ok = 0;
+        if (!ok) s_flag = 0;
+        __syncthreads();
+    }
+    cluster.sync();
+    bool onehot = true;
+    for (unsigned cc = 0; cc < CLUSTER; ++cc) onehot &= (*cluster.map_shared_rank(&s_flag, cc) != 0);
+
+    // ---- load this block's slice: key = row within the table, payload = row of grad_out ----
+    bool bad = false;
+    for (int i = threadIdx.x; i < my_n; i += THREADS) {
+        const int64_t p = (int64_t)c * npc + i;    // position within the table's lookups
+        int32_t idx = __ldg(a.indices + tb0 + p);
+        bad |= (idx < 0) | (idx >= nrows);
+        idx = (int32_t)min((int64_t)max(idx, 0), nrows - 1);
+        int64_t bag = p;
+        if (!onehot) {                             // largest bag b with offsets[t*B + b] <= tb0 + p
+            int lo = 0, hi = a.B;
+            const int32_t *off = a.offsets + (int64_t)t * a.B;
+            while (hi - lo > 1) {
+                int mid = (lo + hi) >> 1;
+                if ((int64_t)__ldg(off + mid) <= tb0 + p) lo = mid; else hi = mid;
+            }
+            bag = lo;
+        }
+        kb[0][i] = (u32)idx;
+        vb[0][i] = (u32)(bag * a.T + t);
+    }
+    if (bad) dq_report(a.status, DQRM_ERR_INDEX_RANGE);
+
+    int bits = 0;
+    while (((int64_t)1 << bits) < nrows) ++bits;
+    const int passes = (bits + 7) / 8;
+    // the slice of this block is cut into WARPS contiguous parts, walked 32 entries at a time
+    const int wsz = ((my_n + WARPS - 1) / WARPS + 31) / 32 * 32;
+    const int w0 = min(my_n, warp * wsz), w1 = min(my_n, w0 + wsz);
+
+    int s = 0;
+    __syncthreads();
+    for (int pass = 0; pass < passes; ++pass) {
+        const int shift = 8 * pass;
+        for (int i = threadIdx.x; i < WARPS * BINS; i += THREADS) (&s_cnt[0][0])[i] = 0u;
+        __syncthreads();
+        // phase 1: digit counts of this warp's part
+        for (int i0 = w0; i0 < w1; i0 += 32) {
+            const int i = i0 + lane;
+            const bool valid = i < w1;
+            const u32 d = valid ? ((kb[s][i] >> shift) & 255u) : 256u;
+            const u32 peers = __match_any_sync(0xffffffffu, d);
+            if (valid && lane == __ffs(peers) - 1) s_cnt[warp][d] += __popc(peers);
+            __syncwarp();
+        }
+        __syncthreads();
+        {
+            u32 h = 0;
+#pragma unroll
+            for (int w = 0; w < WARPS; ++w) h += s_cnt[w][threadIdx.x];
+            s_hist[threadIdx.x] = h;
+        }
+        cluster.sync();
+        // offsets: digits first, then blocks of the cluster, then warps of this block
+        u32 tot = 0, pre = 0;
+        for (unsigned cc = 0; cc < CLUSTER; ++cc) {
+            const u32 h = *remote(cluster, &s_hist[threadIdx.x], cc);
+            if (cc < c) pre += h;
+            tot += h;
+        }
+        u32 incl = tot;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            u32 v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) s_scan[warp] = incl;
+        __syncthreads();
+        u32 woff = 0;
+        for (int w = 0; w < warp; ++w) woff += s_scan[w];
+        u32 run = woff + incl - tot + pre;          // first destination of (digit, this block)
+#pragma unroll
+        for (int w = 0; w < WARPS; ++w) {
+            const u32 cnt = s_cnt[w][threadIdx.x];
+            s_cnt[w][threadIdx.x] = run;
+            run += cnt;
+        }
+        __syncthreads();
+        // phase 2: rank again and scatter into the owners' buffers of the other stage
+        for (int i0 = w0; i0 < w1; i0 += 32) {
+            const int i = i0 + lane;
+            const bool valid = i < w1;
+            const u32 key = valid ? kb[s][i] : 0u;
+            const u32 val = valid ? vb[s][i] : 0u;
+            const u32 d = valid ? ((key >> shift) & 255u) : 256u;
+            const u32 peers = __match_any_sync(0xffffffffu, d);
+            const int leader = __ffs(peers) - 1;
+            u32 base = 0;
+            if (valid && lane == leader) { base = s_cnt[warp][d]; s_cnt[warp][d] = base + __popc(peers); }
+            base = __shfl_sync(0xffffffffu, base, leader);
+            __syncwarp();
+            if (valid) {
+                const u32 pos = base + __popc(peers & lt);      // position within the table, < n
+                if ((int64_t)pos < n) {
+                    if (in_smem) {
+                        const unsigned owner = pos / npc;
+                        const u32 j = pos - owner * npc;
+                        remote(cluster, kb[s ^ 1], owner)[j] = key;
+                        remote(cluster, vb[s ^ 1], owner)[j] = val;
+                    } else {
+                        a.gk[s ^ 1][tb0 + pos] = key;
+                        a.gv[s ^ 1][tb0 + pos] = val;
+                    }
+                }
+            }
+        }
+        cluster.sync();
+        s ^= 1;
+    }
+    // ---- write the sorted slice: arena row keys ----
+    for (int i = threadIdx.x; i < my_n; i += THREADS) {
+        const int64_t j = tb0 + (int64_t)c * npc + i;
+        a.keys_out[j] = (u32)(r0 + kb[s][i]);
+        a.vals_out[j] = vb[s][i];
+    }
+    cluster.sync();      // nobody leaves while its shared memory may still be read or written
+}
+
+inline size_t smem_bytes(int cap) { return (size_t)4 * cap * sizeof(u32); }
+
+// pairs per block to provision in shared memory for an expected n per table
+inline int choose_cap(int64_t expect_n)
+{
+    int64_t npc = ((expect_n + CLUSTER - 1) / CLUSTER + 31) / 32 * 32;
+    int64_t cap = (npc + npc / 4 + 31) / 32 * 32;         // 25 % head room for uneven tables
+    if (cap < 256) cap = 256;
+    if (cap > 12288) cap = 12288;                         // 192 KB of the 227 KB a block may use
+    return (int)cap;
+}
+
+}  // namespace csort

@@ -19,6 +19,7 @@ struct dqrm_ctx {
     int device = 0;
     int num_sms = 0;
     int key_bits = 1;               // bits of an arena row number
+    int sort_path = 0;              // 0: per-table cluster sort, 1: global radix sort
     // launch accounting and optional per-launch timing (see dqrm_profile_*)
     int64_t launch_count = 0;
     int prof_on = 0, prof_n = 0;
@@ -29,7 +30,7 @@ struct dqrm_ctx {
 enum {
     DQ_K_BEGIN = 0, DQ_K_REFRESH, DQ_K_FWD, DQ_K_MEMSET, DQ_K_PREPARE, DQ_K_SORT_SCAN, DQ_K_SORT_SCATTER,
     DQ_K_SEG_COUNT, DQ_K_SEG_EMIT, DQ_K_SEG_REDUCE, DQ_K_SEG_FIXUP, DQ_K_ABSMAX, DQ_K_QUANT, DQ_K_UPDATE,
-    DQ_K_QUANT_UPDATE, DQ_K_COPY, DQ_K_SEG_FIXUP_BIG, DQ_K_COUNT
+    DQ_K_QUANT_UPDATE, DQ_K_COPY, DQ_K_SEG_FIXUP_BIG, DQ_K_CLUSTER_SORT, DQ_K_COUNT
 };
 constexpr int DQ_PROF_MAX = 4096;
 

@@ -150,3 +150,19 @@ def test_train_step_equals_separate_calls_and_oracle(case, oracle):
         assert bit_equal(d_tables.cpu().numpy(), o_tables)
     else:
         assert_close_fp32(d_tables.cpu().numpy(), o_tables, "updated weights")
+
+
+def test_backward_sort_paths_agree(case, oracle):
+    """The per-table cluster sort (default) and the global radix sort give the same bits."""
+    idx, off, go = case.batch(5)
+    case.ctx.set_sort_path(0)
+    ur0, uo0, gr0 = case.gpu_bwd(idx, off, go)
+    case.ctx.set_sort_path(1)
+    try:
+        ur1, uo1, gr1 = case.gpu_bwd(idx, off, go)
+    finally:
+        case.ctx.set_sort_path(0)
+    assert bit_equal(ur0, ur1) and bit_equal(uo0, uo1) and bit_equal(gr0, gr1)
+    o_ur, o_uo, o_gr = oracle.emb_bwd(go, case.wl.T, case.wl.D, case.wl.B, idx, off)
+    assert bit_equal(ur1, o_ur) and bit_equal(uo1, o_uo)
+    assert_close_fp32(gr1, o_gr)
