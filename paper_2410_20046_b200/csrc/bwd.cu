@@ -37,7 +37,7 @@ struct Layout {
     int passes, digit_bits, nb;
     int64_t num_tiles, num_chunks;
     size_t ghist, absmax, counters, tilehist_a, zero_bytes;   // zeroed at call start: [0, zero_bytes)
-    size_t tilehist_b, keys_a, keys_b, vals_a, vals_b, tile_heads, seg_start, chunk_first, long_list, partials;
+    size_t tilehist_b, keys_a, keys_b, vals_a, vals_b, pairs_a, pairs_b, tile_heads, seg_start, chunk_first, long_list, partials;
     size_t total;
 };
 
@@ -63,6 +63,8 @@ Layout make_layout(const dqrm_ctx *ctx, int64_t L)
     y.keys_b = take(sizeof(u32) * Lc);
     y.vals_a = take(sizeof(u32) * Lc);
     y.vals_b = take(sizeof(u32) * Lc);
+    y.pairs_a = take(sizeof(uint2) * Lc);
+    y.pairs_b = take(sizeof(uint2) * Lc);
     y.tile_heads = take(sizeof(u32) * y.num_tiles);
     y.seg_start = take(sizeof(u32) * (Lc + 1));
     y.chunk_first = take(sizeof(u32) * y.num_chunks);
@@ -409,13 +411,16 @@ int dq_launch_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, 
     u32 *ghist = reinterpret_cast<u32 *>(ws + y.ghist);
     const u32 *skeys = nullptr, *svals = nullptr;
     bool sorted = false;
-    if (ctx->sort_path != 1) {
+    // tables far beyond the shared-memory slices sort faster with the global radix sort
+    const bool fits_cluster = (L + ctx->T - 1) / ctx->T <= (int64_t)csort::CLUSTER * 12288;
+    if (ctx->sort_path != 1 && fits_cluster) {
         // one eight-block cluster per table; falls through to the global radix sort if the launch is refused
         csort::Args ca;
         ca.indices = indices; ca.offsets = offsets; ca.row_off = ctx->d_row_off;
         ca.T = ctx->T; ca.B = B; ca.L = L;
         ca.keys_out = keys[0]; ca.vals_out = vals[0];
-        ca.gk[0] = keys[0]; ca.gk[1] = keys[1]; ca.gv[0] = vals[0]; ca.gv[1] = vals[1];
+        // global staging of (row, payload) pairs, used only by tables too large for shared memory
+        ca.gp[0] = reinterpret_cast<uint2 *>(ws + y.pairs_a); ca.gp[1] = reinterpret_cast<uint2 *>(ws + y.pairs_b);
         ca.cap = csort::choose_cap((L + ctx->T - 1) / ctx->T);
         ca.status = ctx->d_status;
         const size_t smem = csort::smem_bytes(ca.cap);

@@ -6,9 +6,9 @@
 // in shared memory, and a least-significant-digit radix sort (8-bit digits, only as many
 // passes as the table's row count needs) moves the pairs between the blocks' shared
 // memories with distributed-shared-memory stores.  Per pass: per-warp digit counts over
-// the block's slice (match_any, stable), the eight per-block histograms are exchanged
-// through DSMEM, every block derives its scatter offsets, ranks its slice again and
-// scatters.  Cluster barriers separate the phases; no block waits on anything else.
+// the block's slice (shared-memory atomics), the eight per-block histograms are exchanged
+// through DSMEM, every block derives its scatter offsets, ranks its slice in order (warp ballots, stable)
+// and scatters.  Cluster barriers separate the phases; no block waits on anything else.
 // Tables whose lookups do not fit the shared-memory slices use the same algorithm on
 // global staging buffers.  The result - keys (arena rows) ascending, payloads (rows of
 // grad_out) in the original order within equal keys - is written table-major, which is
@@ -17,11 +17,16 @@
 #include <cooperative_groups.h>
 #include "common.cuh"
 
+// phase time stamps for bench-top studies of this kernel; compiled out in the library
+#ifndef CSORT_TS
+#define CSORT_TS(i)
+#endif
+
 namespace csort {
 
 namespace cg = cooperative_groups;
 
-constexpr int THREADS = 256;
+constexpr int THREADS = 512;
 constexpr int WARPS = THREADS / 32;
 constexpr int CLUSTER = 8;
 constexpr int BINS = 256;
@@ -33,7 +38,7 @@ struct Args {
     int T, B;
     int64_t L;
     u32 *keys_out, *vals_out;       // [L] sorted result
-    u32 *gk[2], *gv[2];             // [L] global staging (tables too large for shared memory)
+    uint2 *gp[2];                   // [L] global staging of pairs (tables too large for shared memory)
     int cap;                        // pairs per block that fit in shared memory
     int *status;
 };
@@ -43,13 +48,26 @@ __device__ __forceinline__ u32 *remote(cg::cluster_group &cluster, u32 *p, unsig
     return cluster.map_shared_rank(p, rank);
 }
 
+// lanes of the warp that hold the same 8-bit digit as this lane (ballot per bit: the match
+// instruction costs tens of cycles of a shared unit when all 32 digits differ)
+__device__ __forceinline__ u32 same_digit_lanes(u32 d, bool valid)
+{
+    u32 peers = __ballot_sync(0xffffffffu, valid);
+#pragma unroll
+    for (int b = 0; b < 8; ++b) {
+        const u32 m = __ballot_sync(0xffffffffu, (d >> b) & 1u);
+        peers &= ((d >> b) & 1u) ? m : ~m;
+    }
+    return valid ? peers : 0u;
+}
+
 __global__ void __launch_bounds__(THREADS)
 cluster_sort_kernel(const Args a)
 {
-    extern __shared__ u32 s_dyn[];                 // kbuf[2][cap], vbuf[2][cap]
+    extern __shared__ uint2 s_dyn[];               // pair buffers [2][cap]: (row within table, payload)
     __shared__ u32 s_cnt[WARPS][BINS];
     __shared__ u32 s_hist[BINS];
-    __shared__ u32 s_scan[WARPS];
+    __shared__ u32 s_scan[BINS / 32];
     __shared__ int s_flag;
 
     cg::cluster_group cluster = cg::this_cluster();
@@ -72,13 +90,15 @@ cluster_sort_kernel(const Args a)
     const int my_n = (int)max((int64_t)0, min((int64_t)npc, n - (int64_t)c * npc));
 
     // buffers of this block for stage s (shared memory slices, or this block's part of the global staging)
-    u32 *kb[2], *vb[2];
+    // a pair travels as one 8-byte store: distributed-shared-memory traffic is bound by the number of stores
+    uint2 *pb0, *pb1;
     if (in_smem) {
-        kb[0] = s_dyn; kb[1] = s_dyn + a.cap; vb[0] = s_dyn + 2 * a.cap; vb[1] = s_dyn + 3 * a.cap;
+        pb0 = s_dyn; pb1 = s_dyn + a.cap;
     } else {
-        for (int s = 0; s < 2; ++s) { kb[s] = a.gk[s] + tb0 + (int64_t)c * npc; vb[s] = a.gv[s] + tb0 + (int64_t)c * npc; }
+        pb0 = a.gp[0] + tb0 + (int64_t)c * npc; pb1 = a.gp[1] + tb0 + (int64_t)c * npc;
     }
 
+    CSORT_TS(0)
     // ---- are this table's bags all one-index bags in order (offsets = identity)? ----
     {
         if (threadIdx.x == 0) s_flag = 1;
@@ -97,6 +117,7 @@ cluster_sort_kernel(const Args a)
     bool onehot = true;
     for (unsigned cc = 0; cc < CLUSTER; ++cc) onehot &= (*cluster.map_shared_rank(&s_flag, cc) != 0);
 
+    CSORT_TS(1)
     // ---- load this block's slice: key = row within the table, payload = row of grad_out ----
     bool bad = false;
     for (int i = threadIdx.x; i < my_n; i += THREADS) {
@@ -114,8 +135,7 @@ cluster_sort_kernel(const Args a)
             }
             bag = lo;
         }
-        kb[0][i] = (u32)idx;
-        vb[0][i] = (u32)(bag * a.T + t);
+        pb0[i] = make_uint2((u32)idx, (u32)(bag * a.T + t));
     }
     if (bad) dq_report(a.status, DQRM_ERR_INDEX_RANGE);
 
@@ -128,60 +148,65 @@ cluster_sort_kernel(const Args a)
 
     int s = 0;
     __syncthreads();
+    CSORT_TS(2)
     for (int pass = 0; pass < passes; ++pass) {
         const int shift = 8 * pass;
+        const uint2 *src = s ? pb1 : pb0;                           // this pass reads stage s ...
+        uint2 *dst = s ? pb0 : pb1;                                 // ... and fills the other one
+        uint2 *gdst = s ? a.gp[0] : a.gp[1];
         for (int i = threadIdx.x; i < WARPS * BINS; i += THREADS) (&s_cnt[0][0])[i] = 0u;
         __syncthreads();
+        CSORT_TS(3 + 6 * pass)
         // phase 1: digit counts of this warp's part
-        for (int i0 = w0; i0 < w1; i0 += 32) {
-            const int i = i0 + lane;
-            const bool valid = i < w1;
-            const u32 d = valid ? ((kb[s][i] >> shift) & 255u) : 256u;
-            const u32 peers = __match_any_sync(0xffffffffu, d);
-            if (valid && lane == __ffs(peers) - 1) s_cnt[warp][d] += __popc(peers);
-            __syncwarp();
-        }
+        for (int i = w0 + lane; i < w1; i += 32) atomicAdd(&s_cnt[warp][(src[i].x >> shift) & 255u], 1u);
         __syncthreads();
-        {
+        CSORT_TS(4 + 6 * pass)
+        if (threadIdx.x < BINS) {
             u32 h = 0;
-#pragma unroll
+#pragma unroll 8
             for (int w = 0; w < WARPS; ++w) h += s_cnt[w][threadIdx.x];
             s_hist[threadIdx.x] = h;
         }
         cluster.sync();
+        CSORT_TS(5 + 6 * pass)
         // offsets: digits first, then blocks of the cluster, then warps of this block
-        u32 tot = 0, pre = 0;
-        for (unsigned cc = 0; cc < CLUSTER; ++cc) {
-            const u32 h = *remote(cluster, &s_hist[threadIdx.x], cc);
-            if (cc < c) pre += h;
-            tot += h;
-        }
-        u32 incl = tot;
+        u32 tot = 0, pre = 0, incl = 0;
+        if (threadIdx.x < BINS) {                  // one thread per digit (the first BINS / 32 warps)
+            u32 h[CLUSTER];
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            u32 v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
-        }
-        if (lane == 31) s_scan[warp] = incl;
-        __syncthreads();
-        u32 woff = 0;
-        for (int w = 0; w < warp; ++w) woff += s_scan[w];
-        u32 run = woff + incl - tot + pre;          // first destination of (digit, this block)
+            for (unsigned cc = 0; cc < CLUSTER; ++cc) h[cc] = *remote(cluster, &s_hist[threadIdx.x], cc);
 #pragma unroll
-        for (int w = 0; w < WARPS; ++w) {
-            const u32 cnt = s_cnt[w][threadIdx.x];
-            s_cnt[w][threadIdx.x] = run;
-            run += cnt;
+            for (unsigned cc = 0; cc < CLUSTER; ++cc) { if (cc < c) pre += h[cc]; tot += h[cc]; }
+            incl = tot;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                u32 v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            if (lane == 31) s_scan[warp] = incl;
         }
         __syncthreads();
+        if (threadIdx.x < BINS) {
+            u32 woff = 0;
+            for (int w = 0; w < warp; ++w) woff += s_scan[w];
+            u32 run = woff + incl - tot + pre;      // first destination of (digit, this block)
+#pragma unroll 8
+            for (int w = 0; w < WARPS; ++w) {
+                const u32 cnt = s_cnt[w][threadIdx.x];
+                s_cnt[w][threadIdx.x] = run;
+                run += cnt;
+            }
+        }
+        __syncthreads();
+        CSORT_TS(6 + 6 * pass)
         // phase 2: rank again and scatter into the owners' buffers of the other stage
         for (int i0 = w0; i0 < w1; i0 += 32) {
             const int i = i0 + lane;
             const bool valid = i < w1;
-            const u32 key = valid ? kb[s][i] : 0u;
-            const u32 val = valid ? vb[s][i] : 0u;
-            const u32 d = valid ? ((key >> shift) & 255u) : 256u;
-            const u32 peers = __match_any_sync(0xffffffffu, d);
+            const uint2 pr = valid ? src[i] : make_uint2(0u, 0u);
+            const u32 key = pr.x;
+            const u32 d = (key >> shift) & 255u;
+            const u32 peers = same_digit_lanes(d, valid);
             const int leader = __ffs(peers) - 1;
             u32 base = 0;
             if (valid && lane == leader) { base = s_cnt[warp][d]; s_cnt[warp][d] = base + __popc(peers); }
@@ -193,28 +218,31 @@ cluster_sort_kernel(const Args a)
                     if (in_smem) {
                         const unsigned owner = pos / npc;
                         const u32 j = pos - owner * npc;
-                        remote(cluster, kb[s ^ 1], owner)[j] = key;
-                        remote(cluster, vb[s ^ 1], owner)[j] = val;
+                        cluster.map_shared_rank(dst, owner)[j] = pr;
                     } else {
-                        a.gk[s ^ 1][tb0 + pos] = key;
-                        a.gv[s ^ 1][tb0 + pos] = val;
+                        gdst[tb0 + pos] = pr;
                     }
                 }
             }
         }
+        CSORT_TS(7 + 6 * pass)
         cluster.sync();
+        CSORT_TS(8 + 6 * pass)
         s ^= 1;
     }
+    CSORT_TS(30)
     // ---- write the sorted slice: arena row keys ----
     for (int i = threadIdx.x; i < my_n; i += THREADS) {
         const int64_t j = tb0 + (int64_t)c * npc + i;
-        a.keys_out[j] = (u32)(r0 + kb[s][i]);
-        a.vals_out[j] = vb[s][i];
+        const uint2 pr = (s ? pb1 : pb0)[i];
+        a.keys_out[j] = (u32)(r0 + pr.x);
+        a.vals_out[j] = pr.y;
     }
+    CSORT_TS(31)
     cluster.sync();      // nobody leaves while its shared memory may still be read or written
 }
 
-inline size_t smem_bytes(int cap) { return (size_t)4 * cap * sizeof(u32); }
+inline size_t smem_bytes(int cap) { return (size_t)2 * cap * sizeof(uint2); }
 
 // pairs per block to provision in shared memory for an expected n per table
 inline int choose_cap(int64_t expect_n)
