@@ -199,6 +199,12 @@ int dqrm_grad_quant_int8_static(int T, int D, const float *grad_rows, const int3
  * sort over all tables.  Both give identical outputs; the choice only affects speed. */
 int dqrm_set_sort_path(dqrm_ctx *ctx, int path);
 
+/* dqrm_train_step runs the index sort of its backward on a second stream owned by the
+ * context (created by dqrm_create), beside the forward on the caller's stream, and joins
+ * the two before the gradient is summed; the caller's stream sees one ordered step.
+ * on = 0 keeps every launch on the caller's stream.  Default: 1. */
+int dqrm_set_overlap(dqrm_ctx *ctx, int on);
+
 /* ---- quantiser self-check (no counterpart in the paper) ----------------------------
  * The kernels evaluate Q(x; s, b) without the IEEE division sequence where a scale is
  * shared by many elements, and fall back to the division near rounding ties.  This call

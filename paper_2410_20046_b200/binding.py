@@ -43,6 +43,7 @@ SIGNATURES = {
     "dqrm_grad_quant_int8_static": (_i, [_i, _i, _vp, _vp, _vp, _vp, _vp]),
     "dqrm_selfcheck_quantizer": (_i, [_vp, _f, _i, ctypes.c_uint32, ctypes.c_uint64, _vp, _vp]),
     "dqrm_set_sort_path": (_i, [_vp, _i]),
+    "dqrm_set_overlap": (_i, [_vp, _i]),
     "dqrm_launch_count": (_i64, [_vp]),
     "dqrm_profile_begin": (_i, [_vp, _vp]),
     "dqrm_profile_end": (_i, [_vp, _vp, ctypes.POINTER(_f), ctypes.POINTER(ctypes.c_int32), _i]),
@@ -162,6 +163,9 @@ class Context:
         self._check("dqrm_selfcheck_quantizer", self.lib.dqrm_selfcheck_quantizer(
             self._h, float(scale), int(bits), int(first_bits) & 0xFFFFFFFF, int(count),
             _ptr(mismatches, torch.int64), _stream(stream)))
+
+    def set_overlap(self, on: bool):
+        self._check("dqrm_set_overlap", self.lib.dqrm_set_overlap(self._h, int(bool(on))))
 
     def set_sort_path(self, path: int):
         self._check("dqrm_set_sort_path", self.lib.dqrm_set_sort_path(self._h, int(path)))

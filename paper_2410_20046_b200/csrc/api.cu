@@ -73,6 +73,9 @@ int dqrm_create(dqrm_ctx **out, int T, int D, const int64_t *h_row_off)
     if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, sizeof(int));
     if (e == cudaSuccess) e = cudaMalloc(&ctx->d_done, sizeof(u32));
     if (e == cudaSuccess) e = cudaMallocHost(&ctx->h_status_pinned, sizeof(int));
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaMemcpy(ctx->d_row_off, h_row_off, sizeof(int64_t) * (T + 1), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(ctx->d_done, 0, sizeof(u32));
@@ -93,6 +96,9 @@ int dqrm_destroy(dqrm_ctx *ctx)
     if (ctx->d_status) cudaFree(ctx->d_status);
     if (ctx->d_done) cudaFree(ctx->d_done);
     if (ctx->h_status_pinned) cudaFreeHost(ctx->h_status_pinned);
+    if (ctx->side) cudaStreamDestroy(ctx->side);
+    if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+    if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
     if (ctx->prof_events) {
         for (int i = 0; i < DQ_PROF_MAX; ++i) cudaEventDestroy(ctx->prof_events[i]);
         delete[] ctx->prof_events;
@@ -130,6 +136,13 @@ int dqrm_check_status(dqrm_ctx *ctx, void *stream)
 int dqrm_last_cuda_error(const dqrm_ctx *ctx) { return ctx ? ctx->last_cuda_error : 0; }
 
 int64_t dqrm_launch_count(const dqrm_ctx *ctx) { return ctx ? ctx->launch_count : 0; }
+
+int dqrm_set_overlap(dqrm_ctx *ctx, int on)
+{
+    if (!ctx) return DQRM_ERR_INVALID_ARG;
+    ctx->overlap = on ? 1 : 0;
+    return DQRM_OK;
+}
 
 int dqrm_set_sort_path(dqrm_ctx *ctx, int path)
 {
@@ -253,11 +266,30 @@ int dqrm_train_step(dqrm_ctx *ctx, float *tables, const int32_t *indices, const 
     if (!ws_ok(workspace, workspace_bytes, dq_bwd_ws_bytes(ctx, L, (int64_t)ctx->T * B))) return DQRM_ERR_WORKSPACE;
     cudaStream_t st = as_stream(stream);
     if (ctx->prof_on) dq_mark(ctx, st, DQ_K_BEGIN);
-    int rc = dq_launch_fwd(ctx, tables, indices, offsets, scales, bits, out, nullptr, B, L, st);
-    if (rc != DQRM_OK) return rc;
+    // The sort half of the backward needs only the indices, so it runs on the context's second
+    // stream while the forward runs on the caller's (per-launch profiling keeps one stream,
+    // because its events time consecutive launches).
+    const bool overlap = ctx->overlap && !ctx->prof_on && L > 0;
+    cudaStream_t ss = overlap ? ctx->side : st;
     const u32 *absmax = nullptr;
-    rc = dq_launch_bwd(ctx, grad_out, indices, offsets, unique_rows, uniq_off, grad_rows, B, L, workspace,
-                       workspace_bytes, st, &absmax);
+    if (overlap) {
+        DQRM_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_fork, st));
+        DQRM_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
+    }
+    int rc;
+    if (overlap) {
+        rc = dq_launch_bwd_sort(ctx, indices, offsets, unique_rows, uniq_off, B, L, workspace, workspace_bytes, ss, &absmax);
+        if (rc == DQRM_OK) rc = dq_launch_fwd(ctx, tables, indices, offsets, scales, bits, out, nullptr, B, L, st);
+        // join even after an error so that the caller's stream stays ordered behind the side stream
+        cudaEventRecord(ctx->ev_join, ctx->side);
+        cudaStreamWaitEvent(st, ctx->ev_join, 0);
+    } else {
+        rc = dq_launch_fwd(ctx, tables, indices, offsets, scales, bits, out, nullptr, B, L, st);
+        if (rc == DQRM_OK)
+            rc = dq_launch_bwd_sort(ctx, indices, offsets, unique_rows, uniq_off, B, L, workspace, workspace_bytes, st, &absmax);
+    }
+    if (rc != DQRM_OK) return rc;
+    rc = dq_launch_bwd_reduce(ctx, grad_out, grad_rows, B, L, workspace, workspace_bytes, st);
     if (rc != DQRM_OK) return rc;
     return dq_launch_quant_update(ctx, tables, unique_rows, uniq_off, grad_rows, absmax, codes, grad_scales, lr, st);
 }

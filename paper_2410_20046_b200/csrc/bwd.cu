@@ -390,9 +390,11 @@ size_t dq_bwd_ws_bytes(const dqrm_ctx *ctx, int64_t L, int64_t G)
     return make_layout(ctx, L).total;
 }
 
-int dq_launch_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, const int32_t *offsets,
-                  int32_t *unique_rows, int32_t *uniq_off, float *grad_rows, int B, int64_t L,
-                  void *ws_, size_t ws_bytes, cudaStream_t st, const u32 **absmax_bits_out)
+// first half of the backward: everything that depends only on the indices (sort, unique rows,
+// segment starts).  It needs no upstream gradient, so a training step runs it beside the forward.
+int dq_launch_bwd_sort(dqrm_ctx *ctx, const int32_t *indices, const int32_t *offsets,
+                       int32_t *unique_rows, int32_t *uniq_off, int B, int64_t L,
+                       void *ws_, size_t ws_bytes, cudaStream_t st, const u32 **absmax_bits_out)
 {
     const Layout y = make_layout(ctx, L);
     if (ws_bytes < y.total) return DQRM_ERR_WORKSPACE;
@@ -409,7 +411,7 @@ int dq_launch_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, 
     u32 *vals[2] = {reinterpret_cast<u32 *>(ws + y.vals_a), reinterpret_cast<u32 *>(ws + y.vals_b)};
     u32 *thist[2] = {reinterpret_cast<u32 *>(ws + y.tilehist_a), reinterpret_cast<u32 *>(ws + y.tilehist_b)};
     u32 *ghist = reinterpret_cast<u32 *>(ws + y.ghist);
-    const u32 *skeys = nullptr, *svals = nullptr;
+    const u32 *skeys = nullptr;      // sorted keys; the sorted payloads sit beside them in vals[0]
     bool sorted = false;
     // tables far beyond the shared-memory slices sort faster with the global radix sort
     const bool fits_cluster = (L + ctx->T - 1) / ctx->T <= (int64_t)csort::CLUSTER * 12288;
@@ -445,7 +447,7 @@ int dq_launch_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, 
         }
         if (e == cudaSuccess) {
             dq_mark(ctx, st, DQ_K_CLUSTER_SORT);
-            skeys = keys[0]; svals = vals[0];
+            skeys = keys[0];
             sorted = true;
         } else {
             (void)cudaGetLastError();
@@ -457,7 +459,7 @@ int dq_launch_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, 
         int64_t blocks = (G + 255) / 256;
         int64_t cap = (int64_t)ctx->num_sms * 8;
         int grid = (int)(blocks > cap ? cap : blocks);
-        prepare_kernel<<<grid, 256, 0, st>>>(indices, offsets, ctx->d_row_off, ctx->T, B, G, L, keys[0], vals[0],
+        prepare_kernel<<<grid, 256, 0, st>>>(indices, offsets, ctx->d_row_off, ctx->T, B, G, L, keys[y.passes & 1], vals[y.passes & 1],
                                              ghist, thist[0], y.num_tiles, y.passes, y.digit_bits, ctx->d_status);
         DQRM_CUDA_TRY(ctx, cudaGetLastError());
         dq_mark(ctx, st, DQ_K_PREPARE);
@@ -471,12 +473,13 @@ int dq_launch_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, 
         DQRM_CUDA_TRY(ctx, cudaGetLastError());
         dq_mark(ctx, st, DQ_K_SORT_SCAN);
         sort_scatter_kernel<<<(unsigned)y.num_tiles, ST_THREADS, 0, st>>>(
-            keys[p & 1], vals[p & 1], keys[(p + 1) & 1], vals[(p + 1) & 1], cur, nxt, L, p * y.digit_bits, y.nb,
+            keys[(p + y.passes) & 1], vals[(p + y.passes) & 1], keys[(p + y.passes + 1) & 1], vals[(p + y.passes + 1) & 1],
+            cur, nxt, L, p * y.digit_bits, y.nb,
             (p + 1) * y.digit_bits, y.num_tiles, ctx->d_status);
         DQRM_CUDA_TRY(ctx, cudaGetLastError());
         dq_mark(ctx, st, DQ_K_SORT_SCATTER);
     }
-        skeys = keys[y.passes & 1]; svals = vals[y.passes & 1];
+        skeys = keys[0];                         // the ping-pong starts so that the last pass lands in buffer 0
     }
     seg_count_kernel<<<(unsigned)y.num_tiles, ST_THREADS, 0, st>>>(skeys, L, reinterpret_cast<u32 *>(ws + y.tile_heads));
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
@@ -487,7 +490,20 @@ int dq_launch_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, 
         reinterpret_cast<u32 *>(ws + y.counters));
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
     dq_mark(ctx, st, DQ_K_SEG_EMIT);
+    return DQRM_OK;
+}
 
+// second half: segmented sum of the upstream gradient over the sorted lookups
+int dq_launch_bwd_reduce(dqrm_ctx *ctx, const float *grad_out, float *grad_rows, int B, int64_t L,
+                         void *ws_, size_t ws_bytes, cudaStream_t st)
+{
+    const Layout y = make_layout(ctx, L);
+    if (ws_bytes < y.total) return DQRM_ERR_WORKSPACE;
+    if (L == 0) return DQRM_OK;
+    char *ws = reinterpret_cast<char *>(ws_);
+    const int64_t G = (int64_t)ctx->T * B;
+    // both sort paths leave the sorted pairs in the first key / payload buffers
+    const u32 *skeys = reinterpret_cast<const u32 *>(ws + y.keys_a), *svals = reinterpret_cast<const u32 *>(ws + y.vals_a);
     const int D = ctx->D, d4 = D / 4;
 #define DQ_RED(RL, RV, RC, LPR, CH) \
     return launch_reduce<RL, RV, RC, LPR, CH>(ctx, y, ws, skeys, svals, grad_out, grad_rows, L, G, st)
@@ -501,4 +517,13 @@ int dq_launch_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, 
     if (d4 <= 128) DQ_RED(32, 4, 4, 32, 4);
     DQ_RED(32, 4, 8, 32, 8);
 #undef DQ_RED
+}
+
+int dq_launch_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, const int32_t *offsets,
+                  int32_t *unique_rows, int32_t *uniq_off, float *grad_rows, int B, int64_t L,
+                  void *ws, size_t ws_bytes, cudaStream_t st, const u32 **absmax_bits_out)
+{
+    int rc = dq_launch_bwd_sort(ctx, indices, offsets, unique_rows, uniq_off, B, L, ws, ws_bytes, st, absmax_bits_out);
+    if (rc != DQRM_OK) return rc;
+    return dq_launch_bwd_reduce(ctx, grad_out, grad_rows, B, L, ws, ws_bytes, st);
 }

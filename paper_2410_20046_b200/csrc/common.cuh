@@ -20,6 +20,9 @@ struct dqrm_ctx {
     int num_sms = 0;
     int key_bits = 1;               // bits of an arena row number
     int sort_path = 0;              // 0: per-table cluster sort, 1: global radix sort
+    cudaStream_t side = nullptr;    // second stream: a training step sorts the indices beside its forward
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    int overlap = 1;                // 0: keep everything on the caller's stream
     // launch accounting and optional per-launch timing (see dqrm_profile_*)
     int64_t launch_count = 0;
     int prof_on = 0, prof_n = 0;
@@ -184,6 +187,12 @@ size_t dq_bwd_ws_bytes(const dqrm_ctx *ctx, int64_t L, int64_t G);
 int dq_launch_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, const int32_t *offsets,
                   int32_t *unique_rows, int32_t *uniq_off, float *grad_rows, int B, int64_t L,
                   void *ws, size_t ws_bytes, cudaStream_t st, const u32 **absmax_bits_out);
+
+int dq_launch_bwd_sort(dqrm_ctx *ctx, const int32_t *indices, const int32_t *offsets, int32_t *unique_rows,
+                       int32_t *uniq_off, int B, int64_t L, void *ws, size_t ws_bytes, cudaStream_t st,
+                       const u32 **absmax_bits_out);
+int dq_launch_bwd_reduce(dqrm_ctx *ctx, const float *grad_out, float *grad_rows, int B, int64_t L, void *ws,
+                         size_t ws_bytes, cudaStream_t st);
 
 size_t dq_quant_ws_bytes(const dqrm_ctx *ctx);
 int dq_launch_grad_quant(dqrm_ctx *ctx, const float *grad_rows, const int32_t *uniq_off, int8_t *codes,
