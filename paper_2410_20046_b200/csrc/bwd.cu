@@ -36,8 +36,9 @@ constexpr int SEG_CHUNK = segred::CHUNK;         // sorted entries per reduce wo
 struct Layout {
     int passes, digit_bits, nb;
     int64_t num_tiles, num_chunks;
-    size_t ghist, absmax, counters, tilehist_a, zero_bytes;   // zeroed at call start: [0, zero_bytes)
-    size_t tilehist_b, keys_a, keys_b, vals_a, vals_b, pairs_a, pairs_b, tile_heads, seg_start, chunk_first, long_list, partials;
+    // zeroed at call start: [0, zero_small) always, [0, zero_bytes) by the radix path
+    size_t absmax, counters, tile_heads, zero_small, ghist, tilehist_a, zero_bytes;
+    size_t tilehist_b, keys_a, keys_b, vals_a, vals_b, pairs_a, pairs_b, seg_start, chunk_first, long_list, partials;
     size_t total;
 };
 
@@ -53,9 +54,11 @@ Layout make_layout(const dqrm_ctx *ctx, int64_t L)
     y.num_chunks = (Lc + SEG_CHUNK - 1) / SEG_CHUNK;
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
-    y.ghist = take(sizeof(u32) * MAX_PASSES * NB_MAX);
     y.absmax = take(sizeof(u32) * ctx->T);
     y.counters = take(sizeof(u32) * 8);
+    y.tile_heads = take(sizeof(u32) * y.num_tiles);
+    y.zero_small = o;
+    y.ghist = take(sizeof(u32) * MAX_PASSES * NB_MAX);
     y.tilehist_a = take(sizeof(u32) * y.nb * y.num_tiles);
     y.zero_bytes = o;
     y.tilehist_b = take(sizeof(u32) * y.nb * y.num_tiles);
@@ -65,7 +68,6 @@ Layout make_layout(const dqrm_ctx *ctx, int64_t L)
     y.vals_b = take(sizeof(u32) * Lc);
     y.pairs_a = take(sizeof(uint2) * Lc);
     y.pairs_b = take(sizeof(uint2) * Lc);
-    y.tile_heads = take(sizeof(u32) * y.num_tiles);
     y.seg_start = take(sizeof(u32) * (Lc + 1));
     y.chunk_first = take(sizeof(u32) * y.num_chunks);
     y.long_list = take(sizeof(u32) * y.num_chunks);
@@ -358,27 +360,19 @@ int launch_reduce(dqrm_ctx *ctx, const Layout &y, char *ws, const u32 *keys, con
     dq_mark(ctx, st, DQ_K_SEG_REDUCE);
     int64_t fblocks = (y.num_chunks + 7) / 8;                // at most one cut segment per chunk, a warp each
     int fgrid = (int)(fblocks < (int64_t)ctx->num_sms * 4 ? (fblocks < 1 ? 1 : fblocks) : (int64_t)ctx->num_sms * 4);
-    seg_fixup_kernel<LPR, CH><<<fgrid, 256, smem, st>>>(keys, seg_start, partials, long_list, counters, grad_rows,
-                                                        absmax, ctx->d_row_off, ctx->T, ctx->D);
-    DQRM_CUDA_TRY(ctx, cudaGetLastError());
-    dq_mark(ctx, st, DQ_K_SEG_FIXUP);
-    const size_t big_smem = (size_t)(256 / LPR) * ctx->D * sizeof(double);
-    if (big_smem > 48 * 1024) {
+    const size_t fix_smem = (size_t)(256 / LPR) * ctx->D * sizeof(double) + smem;
+    if (fix_smem > 48 * 1024) {
         static bool raised = false;
         if (!raised) {
-            DQRM_CUDA_TRY(ctx, cudaFuncSetAttribute(seg_fixup_big_kernel<LPR, CH>,
-                                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)big_smem));
+            DQRM_CUDA_TRY(ctx, cudaFuncSetAttribute(seg_fixup_kernel<LPR, CH>,
+                                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fix_smem));
             raised = true;
         }
     }
-    int bgrid = (int)((y.num_chunks + BIG_PIECES - 1) / BIG_PIECES);     // at most this many big segments
-    if (bgrid > ctx->num_sms * 2) bgrid = ctx->num_sms * 2;
-    if (bgrid < 1) bgrid = 1;
-    seg_fixup_big_kernel<LPR, CH><<<bgrid, 256, big_smem, st>>>(keys, seg_start, partials, long_list, counters,
-                                                                 grad_rows, absmax, ctx->d_row_off, ctx->T, ctx->D,
-                                                                 y.num_chunks);
+    seg_fixup_kernel<LPR, CH><<<fgrid, 256, fix_smem, st>>>(keys, seg_start, partials, long_list, counters, grad_rows,
+                                                            absmax, ctx->d_row_off, ctx->T, ctx->D, y.num_chunks);
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
-    dq_mark(ctx, st, DQ_K_SEG_FIXUP_BIG);
+    dq_mark(ctx, st, DQ_K_SEG_FIXUP);
     return DQRM_OK;
 }
 
@@ -401,7 +395,9 @@ int dq_launch_bwd_sort(dqrm_ctx *ctx, const int32_t *indices, const int32_t *off
     char *ws = reinterpret_cast<char *>(ws_);
     const int64_t G = (int64_t)ctx->T * B;
     if (absmax_bits_out) *absmax_bits_out = reinterpret_cast<const u32 *>(ws + y.absmax);
-    DQRM_CUDA_TRY(ctx, cudaMemsetAsync(ws, 0, y.zero_bytes, st));
+    const bool fits_cluster = (L + ctx->T - 1) / ctx->T <= (int64_t)csort::CLUSTER * 12288;
+    const bool try_cluster = ctx->sort_path != 1 && fits_cluster;
+    DQRM_CUDA_TRY(ctx, cudaMemsetAsync(ws, 0, try_cluster ? y.zero_small : y.zero_bytes, st));
     dq_mark(ctx, st, DQ_K_MEMSET);
     if (L == 0) {
         DQRM_CUDA_TRY(ctx, cudaMemsetAsync(uniq_off, 0, sizeof(int32_t) * (ctx->T + 1), st));
@@ -413,9 +409,8 @@ int dq_launch_bwd_sort(dqrm_ctx *ctx, const int32_t *indices, const int32_t *off
     u32 *ghist = reinterpret_cast<u32 *>(ws + y.ghist);
     const u32 *skeys = nullptr;      // sorted keys; the sorted payloads sit beside them in vals[0]
     bool sorted = false;
-    // tables far beyond the shared-memory slices sort faster with the global radix sort
-    const bool fits_cluster = (L + ctx->T - 1) / ctx->T <= (int64_t)csort::CLUSTER * 12288;
-    if (ctx->sort_path != 1 && fits_cluster) {
+    // (tables far beyond the shared-memory slices sort faster with the global radix sort)
+    if (try_cluster) {
         // one eight-block cluster per table; falls through to the global radix sort if the launch is refused
         csort::Args ca;
         ca.indices = indices; ca.offsets = offsets; ca.row_off = ctx->d_row_off;
@@ -425,6 +420,7 @@ int dq_launch_bwd_sort(dqrm_ctx *ctx, const int32_t *indices, const int32_t *off
         ca.gp[0] = reinterpret_cast<uint2 *>(ws + y.pairs_a); ca.gp[1] = reinterpret_cast<uint2 *>(ws + y.pairs_b);
         ca.cap = csort::choose_cap((L + ctx->T - 1) / ctx->T);
         ca.status = ctx->d_status;
+        ca.tile_heads = reinterpret_cast<u32 *>(ws + y.tile_heads);
         const size_t smem = csort::smem_bytes(ca.cap);
         static bool raised = false;
         cudaError_t e = cudaSuccess;
@@ -455,6 +451,8 @@ int dq_launch_bwd_sort(dqrm_ctx *ctx, const int32_t *indices, const int32_t *off
         }
     }
     if (!sorted) {
+        if (try_cluster)      // the cluster launch was refused: zero what the radix sort needs as well
+            DQRM_CUDA_TRY(ctx, cudaMemsetAsync(ws + y.zero_small, 0, y.zero_bytes - y.zero_small, st));
     {
         int64_t blocks = (G + 255) / 256;
         int64_t cap = (int64_t)ctx->num_sms * 8;
@@ -481,9 +479,11 @@ int dq_launch_bwd_sort(dqrm_ctx *ctx, const int32_t *indices, const int32_t *off
     }
         skeys = keys[0];                         // the ping-pong starts so that the last pass lands in buffer 0
     }
-    seg_count_kernel<<<(unsigned)y.num_tiles, ST_THREADS, 0, st>>>(skeys, L, reinterpret_cast<u32 *>(ws + y.tile_heads));
-    DQRM_CUDA_TRY(ctx, cudaGetLastError());
-    dq_mark(ctx, st, DQ_K_SEG_COUNT);
+    if (!sorted) {        // (the cluster sort counts the segment heads of every tile on its way out)
+        seg_count_kernel<<<(unsigned)y.num_tiles, ST_THREADS, 0, st>>>(skeys, L, reinterpret_cast<u32 *>(ws + y.tile_heads));
+        DQRM_CUDA_TRY(ctx, cudaGetLastError());
+        dq_mark(ctx, st, DQ_K_SEG_COUNT);
+    }
     seg_emit_kernel<<<(unsigned)y.num_tiles, ST_THREADS, (size_t)(ctx->T + 1) * sizeof(int64_t), st>>>(
         skeys, L, reinterpret_cast<const u32 *>(ws + y.tile_heads), ctx->d_row_off, ctx->T,
         reinterpret_cast<u32 *>(ws + y.seg_start), reinterpret_cast<u32 *>(ws + y.chunk_first), unique_rows, uniq_off,

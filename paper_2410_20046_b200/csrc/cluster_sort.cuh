@@ -41,6 +41,7 @@ struct Args {
     uint2 *gp[2];                   // [L] global staging of pairs (tables too large for shared memory)
     int cap;                        // pairs per block that fit in shared memory
     int *status;
+    u32 *tile_heads;                // [ceil(L / 2048)] zeroed by the caller: segment heads per tile of the sorted order
 };
 
 __device__ __forceinline__ u32 *remote(cg::cluster_group &cluster, u32 *p, unsigned rank)
@@ -232,11 +233,36 @@ cluster_sort_kernel(const Args a)
     }
     CSORT_TS(30)
     // ---- write the sorted slice: arena row keys ----
-    for (int i = threadIdx.x; i < my_n; i += THREADS) {
-        const int64_t j = tb0 + (int64_t)c * npc + i;
-        const uint2 pr = (s ? pb1 : pb0)[i];
-        a.keys_out[j] = (u32)(r0 + pr.x);
-        a.vals_out[j] = pr.y;
+    // and count, per 2048-entry tile of the sorted order, the entries that start a new row
+    {
+        const uint2 *fin = s ? pb1 : pb0;
+        u32 prev_last = 0xFFFFFFFFu;               // last row of the previous block's slice (full by construction)
+        if (c > 0) {
+            const uint2 *pf = in_smem ? cluster.map_shared_rank(s ? pb1 : pb0, c - 1)
+                                      : (s ? a.gp[1] : a.gp[0]) + tb0 + (int64_t)(c - 1) * npc;
+            prev_last = pf[npc - 1].x;
+        }
+        for (int i0 = warp * 32; i0 < my_n; i0 += THREADS) {
+            const int i = i0 + lane;
+            const bool valid = i < my_n;
+            const int64_t j = tb0 + (int64_t)c * npc + i;
+            bool head = false;
+            if (valid) {
+                const uint2 pr = fin[i];
+                a.keys_out[j] = (u32)(r0 + pr.x);
+                a.vals_out[j] = pr.y;
+                const u32 before = i > 0 ? fin[i - 1].x : prev_last;
+                head = (c == 0 && i == 0) || before != pr.x;
+            }
+            const int64_t tile = j >> 11;
+            const int64_t tile0 = __shfl_sync(0xffffffffu, tile, 0);
+            const u32 m0 = __ballot_sync(0xffffffffu, head && tile == tile0);
+            const u32 m1 = __ballot_sync(0xffffffffu, head && tile != tile0);
+            if (lane == 0) {
+                if (m0) atomicAdd(&a.tile_heads[tile0], __popc(m0));
+                if (m1) atomicAdd(&a.tile_heads[tile0 + 1], __popc(m1));
+            }
+        }
     }
     CSORT_TS(31)
     cluster.sync();      // nobody leaves while its shared memory may still be read or written

@@ -294,16 +294,12 @@ __device__ __forceinline__ void add_pieces(double (&acc)[CH][4], const double *p
 
 // one warp per cut segment of at most BIG_PIECES pieces
 template <int LPR, int CH>
-__global__ void __launch_bounds__(256)
-seg_fixup_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ seg_start,
-                 const double *__restrict__ partials, const u32 *__restrict__ long_list,
-                 const u32 *__restrict__ counters, float *__restrict__ grad_rows, u32 *__restrict__ absmax,
-                 const int64_t *__restrict__ row_off, int T, int D)
+__device__ __forceinline__ void
+fixup_small(const u32 *__restrict__ keys, const u32 *__restrict__ seg_start,
+            const double *__restrict__ partials, const u32 *__restrict__ long_list,
+            const u32 *__restrict__ counters, float *__restrict__ grad_rows, u32 *__restrict__ absmax,
+            const int64_t *s_off, int T, int D)
 {
-    extern __shared__ unsigned char smem_raw[];
-    int64_t *s_off = reinterpret_cast<int64_t *>(smem_raw);
-    for (int t = threadIdx.x; t <= T; t += blockDim.x) s_off[t] = row_off[t];
-    __syncthreads();
     constexpr int SG = 32 / LPR;
     const int d4 = D >> 2;
     const int wl = threadIdx.x & 31;
@@ -335,15 +331,13 @@ seg_fixup_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ seg_start
 
 // one block per cut segment of more than BIG_PIECES pieces (hot rows)
 template <int LPR, int CH>
-__global__ void __launch_bounds__(256)
-seg_fixup_big_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ seg_start,
-                     const double *__restrict__ partials, const u32 *__restrict__ long_list,
-                     const u32 *__restrict__ counters, float *__restrict__ grad_rows, u32 *__restrict__ absmax,
-                     const int64_t *__restrict__ row_off, int T, int D, int64_t num_chunks)
+__device__ __forceinline__ void
+fixup_big(const u32 *__restrict__ keys, const u32 *__restrict__ seg_start,
+          const double *__restrict__ partials, const u32 *__restrict__ long_list,
+          const u32 *__restrict__ counters, float *__restrict__ grad_rows, u32 *__restrict__ absmax,
+          const int64_t *__restrict__ row_off, int T, int D, int64_t num_chunks, double *s_part /*[256/LPR][D]*/)
 {
-    extern __shared__ unsigned char smem_raw[];
     constexpr int NSG = 256 / LPR;
-    double *s_part = reinterpret_cast<double *>(smem_raw);            // [NSG][D]
     const int d4 = D >> 2;
     const int sub = threadIdx.x / LPR, lane = threadIdx.x % LPR;
     const u32 count = counters[CNT_BIG];
@@ -392,6 +386,25 @@ seg_fixup_big_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ seg_s
             }
         }
     }
+}
+
+// both fix-ups in one launch: every block first takes its share of the hot rows, then its
+// warps take the short cut segments
+template <int LPR, int CH>
+__global__ void __launch_bounds__(256)
+seg_fixup_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ seg_start,
+                 const double *__restrict__ partials, const u32 *__restrict__ long_list,
+                 const u32 *__restrict__ counters, float *__restrict__ grad_rows, u32 *__restrict__ absmax,
+                 const int64_t *__restrict__ row_off, int T, int D, int64_t num_chunks)
+{
+    extern __shared__ unsigned char smem_raw[];
+    double *s_part = reinterpret_cast<double *>(smem_raw);                         // [256/LPR][D]
+    int64_t *s_off = reinterpret_cast<int64_t *>(s_part + (size_t)(256 / LPR) * D);  // [T+1]
+    for (int t = threadIdx.x; t <= T; t += blockDim.x) s_off[t] = row_off[t];
+    __syncthreads();
+    fixup_big<LPR, CH>(keys, seg_start, partials, long_list, counters, grad_rows, absmax, row_off, T, D, num_chunks,
+                       s_part);
+    fixup_small<LPR, CH>(keys, seg_start, partials, long_list, counters, grad_rows, absmax, s_off, T, D);
 }
 
 }  // namespace segred
