@@ -166,3 +166,52 @@ def test_backward_sort_paths_agree(case, oracle):
     o_ur, o_uo, o_gr = oracle.emb_bwd(go, case.wl.T, case.wl.D, case.wl.B, idx, off)
     assert bit_equal(ur1, o_ur) and bit_equal(uo1, o_uo)
     assert_close_fp32(gr1, o_gr)
+
+
+def test_tiny_trajectory_100_steps_with_periodic_refresh(oracle):
+    """The Tiny configuration end to end: 100 iterations, scale refresh every 10, GPU and oracle
+    running free (no resynchronisation).  Integer outputs and scales must agree bit for bit at
+    every step; a code may differ only where the oracle's pre-rounding quotient lies within 1e-4
+    of a rounding boundary (a last-bit difference of an FP64-accumulated sum), and none is expected."""
+    import torch
+
+    wl = W.tiny()
+    c = Case(wl)
+    o_tables = W.tables_np(wl)
+    d_tables = c.dev(o_tables)
+    L = wl.T * wl.B
+    out = c.empty((wl.B, wl.T, wl.D), torch.float32)
+    ur = c.empty(L, torch.int32)
+    uo = c.empty(wl.T + 1, torch.int32)
+    gr = c.empty((L, wl.D), torch.float32)
+    codes = c.empty((L, wl.D), torch.int8)
+    gs = c.empty(wl.T, torch.float32)
+    scales = c.empty(wl.T, torch.float32)
+    o_scales = None
+    flips = 0
+    for step in range(wl.iters):
+        if step % wl.period == 0:
+            c.ctx.scale_refresh(d_tables, c.bits, scales)
+            o_scales, _ = oracle.scale_refresh(o_tables, c.row_off, wl.D, c.bits_np)
+            assert bit_equal(scales.cpu().numpy(), o_scales), f"step {step}: scales"
+        idx, off, go = c.batch(step)
+        c.ctx.train_step(d_tables, c.dev(idx), c.dev(off), c.dev(go), scales, c.bits, out, ur, uo, gr, codes, gs,
+                         wl.lr, B=wl.B, L=len(idx))
+        r = oracle.train_step(o_tables, c.row_off, wl.D, wl.B, idx, off, go, o_scales, c.bits_np, wl.lr)
+        U = int(r["uniq_off"][-1])
+        assert bit_equal(uo.cpu().numpy(), r["uniq_off"]), f"step {step}"
+        assert bit_equal(ur.cpu().numpy()[:U], r["unique_rows"]), f"step {step}"
+        assert_close_fp32(out.cpu().numpy(), r["out"], f"step {step}: pooled output")
+        assert_close_fp32(gr.cpu().numpy()[:U], r["grad_rows"], f"step {step}: summed gradients")
+        assert bit_equal(gs.cpu().numpy(), r["grad_scales"]), f"step {step}: gradient scales"
+        diff = codes.cpu().numpy()[:U] != r["codes"]
+        if diff.any():
+            t_of = np.searchsorted(r["uniq_off"], np.nonzero(diff)[0], side="right") - 1
+            q = r["grad_rows"][diff] / r["grad_scales"][t_of]
+            assert (np.abs(np.abs(q - np.floor(q)) - 0.5) < 1e-4).all(), f"step {step}: unexplained code flips"
+            flips += int(diff.sum())
+    c.ctx.raise_on_device_error()
+    assert_close_fp32(d_tables.cpu().numpy(), o_tables, "weights after 100 steps")
+    assert flips == 0, f"{flips} explained code flips (expected none)"
+    assert bit_equal(d_tables.cpu().numpy(), o_tables)
+    c.ctx.close()
