@@ -215,3 +215,110 @@ def test_tiny_trajectory_100_steps_with_periodic_refresh(oracle):
     assert flips == 0, f"{flips} explained code flips (expected none)"
     assert bit_equal(d_tables.cpu().numpy(), o_tables)
     c.ctx.close()
+
+
+# ---------------------------------------------------------------------------
+# edge cases and error paths of the ABI
+# ---------------------------------------------------------------------------
+def _mini():
+    return W.Workload("mini", (50, 7, 300), D=16, B=64, alpha=1.1, bits=4)
+
+
+def test_alternating_empty_and_double_bags_with_L_equal_G(oracle):
+    """L == T*B selects the one-index forward kernel; bags of 0 and 2 indices must still pool right."""
+    wl = _mini()
+    c = Case(wl)
+    tables = W.tables_np(wl)
+    idx, _, go = c.batch(0)                                   # L = T*B indices
+    lens = np.tile(np.array([0, 2], dtype=np.int64), wl.T * wl.B // 2)
+    off = np.zeros(wl.T * wl.B + 1, dtype=np.int32)
+    off[1:] = np.cumsum(lens)
+    o_scales, _ = oracle.scale_refresh(tables, c.row_off, wl.D, c.bits_np)
+    out, _ = c.gpu_fwd(c.dev(tables), idx, off, c.dev(o_scales), want_codes=False)
+    o_out = oracle.emb_fwd(tables, c.row_off, wl.D, wl.B, idx, off, o_scales, c.bits_np)
+    assert bit_equal(out, o_out)
+    ur, uo, gr = c.gpu_bwd(idx, off, go)
+    o_ur, o_uo, o_gr = oracle.emb_bwd(go, wl.T, wl.D, wl.B, idx, off)
+    assert bit_equal(ur, o_ur) and bit_equal(uo, o_uo)
+    assert_close_fp32(gr, o_gr)
+    c.ctx.close()
+
+
+def test_all_bags_empty(oracle):
+    import torch
+
+    wl = _mini()
+    c = Case(wl)
+    tables = W.tables_np(wl)
+    off = np.zeros(wl.T * wl.B + 1, dtype=np.int32)
+    idx = np.zeros(0, dtype=np.int32)
+    go = W.grad_out_np(wl, 0)
+    o_scales, _ = oracle.scale_refresh(tables, c.row_off, wl.D, c.bits_np)
+    out, _ = c.gpu_fwd(c.dev(tables), idx, off, c.dev(o_scales), want_codes=False)
+    assert not out.any()
+    ur, uo, gr = c.gpu_bwd(idx, off, go)
+    assert len(ur) == 0 and not uo.any()
+    d_tables = c.dev(tables)
+    gs = c.empty(wl.T, torch.float32)
+    one = c.empty(1, torch.int32)
+    c.ctx.train_step(d_tables, one, c.dev(off), c.dev(go), c.dev(o_scales), c.bits,
+                     c.empty((wl.B, wl.T, wl.D), torch.float32), one, c.empty(wl.T + 1, torch.int32),
+                     c.empty((1, wl.D), torch.float32), c.empty((1, wl.D), torch.int8), gs, wl.lr, B=wl.B, L=0)
+    c.ctx.raise_on_device_error()
+    assert bit_equal(d_tables.cpu().numpy(), tables)                       # nothing touched, nothing updated
+    assert (gs.cpu().numpy() == oracle.scale_from_absmax(0.0, 8)).all()    # scale of an empty gradient
+    c.ctx.close()
+
+
+def test_out_of_range_index_is_reported_not_trapped(oracle):
+    import paper_2410_20046_b200 as dq
+
+    wl = _mini()
+    c = Case(wl)
+    tables = W.tables_np(wl)
+    idx, off, go = c.batch(0)
+    o_scales, _ = oracle.scale_refresh(tables, c.row_off, wl.D, c.bits_np)
+    bad = idx.copy()
+    bad[3] = wl.rows[0] + 5                   # beyond table 0
+    bad[wl.B + 1] = -2                        # negative, table 1
+    for call in ("fwd", "bwd"):
+        if call == "fwd":
+            with pytest.raises(dq.DqrmError) as e:
+                c.gpu_fwd(c.dev(tables), bad, off, c.dev(o_scales), want_codes=False)
+        else:
+            with pytest.raises(dq.DqrmError) as e:
+                c.gpu_bwd(bad, off, go)
+        assert e.value.status == dq.ERR_INDEX_RANGE
+        assert c.ctx.check_status() == dq.OK                 # the report cleared the status word
+    # the context is still usable and correct
+    out, _ = c.gpu_fwd(c.dev(tables), idx, off, c.dev(o_scales), want_codes=False)
+    assert bit_equal(out, oracle.emb_fwd(tables, c.row_off, wl.D, wl.B, idx, off, o_scales, c.bits_np))
+    c.ctx.close()
+
+
+def test_bad_arguments_are_refused_on_the_host():
+    import ctypes
+    import torch
+    import paper_2410_20046_b200 as dq
+
+    wl = _mini()
+    c = Case(wl)
+    lib = c.ctx.lib
+    t = c.empty((wl.total_rows, wl.D), torch.float32)
+    i32 = c.empty(wl.T * wl.B + 1, torch.int32)
+    f32 = c.empty((wl.B, wl.T, wl.D), torch.float32)
+    st = torch.cuda.current_stream().cuda_stream
+    # null output pointer
+    assert lib.dqrm_emb_fwd(c.ctx._h, t.data_ptr(), i32.data_ptr(), i32.data_ptr(), f32.data_ptr(), c.bits.data_ptr(),
+                            None, None, wl.B, wl.T * wl.B, st) == dq.ERR_INVALID_ARG
+    # negative batch
+    assert lib.dqrm_emb_fwd(c.ctx._h, t.data_ptr(), i32.data_ptr(), i32.data_ptr(), f32.data_ptr(), c.bits.data_ptr(),
+                            f32.data_ptr(), None, -1, 10, st) == dq.ERR_INVALID_ARG
+    # workspace too small / misaligned
+    args = (c.ctx._h, f32.data_ptr(), i32.data_ptr(), i32.data_ptr(), i32.data_ptr(), i32.data_ptr(), f32.data_ptr(),
+            wl.B, wl.T * wl.B)
+    assert lib.dqrm_emb_bwd(*args, c.ctx._ws_ptr, 1024, st) == dq.ERR_WORKSPACE
+    assert lib.dqrm_emb_bwd(*args, c.ctx._ws_ptr + 8, c.ctx.workspace_bytes - 8, st) == dq.ERR_WORKSPACE
+    assert lib.dqrm_emb_bwd(*args, None, c.ctx.workspace_bytes, st) == dq.ERR_WORKSPACE
+    torch.cuda.synchronize()
+    c.ctx.close()
