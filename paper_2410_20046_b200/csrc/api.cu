@@ -73,7 +73,12 @@ int dqrm_create(dqrm_ctx **out, int T, int D, const int64_t *h_row_off)
     if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, sizeof(int));
     if (e == cudaSuccess) e = cudaMalloc(&ctx->d_done, sizeof(u32));
     if (e == cudaSuccess) e = cudaMallocHost(&ctx->h_status_pinned, sizeof(int));
-    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking);
+    if (e == cudaSuccess) {
+        // highest priority: the sort's few blocks should be placed ahead of the forward's many
+        int lo_prio = 0, hi_prio = 0;
+        e = cudaDeviceGetStreamPriorityRange(&lo_prio, &hi_prio);
+        if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&ctx->side, cudaStreamNonBlocking, hi_prio);
+    }
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaMemcpy(ctx->d_row_off, h_row_off, sizeof(int64_t) * (T + 1), cudaMemcpyHostToDevice);
