@@ -62,7 +62,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50",
                  "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
@@ -106,6 +106,14 @@ def algorithmic_bytes(wl, L, G, U):
 
 # kernel -> which algorithmic byte count bounds it (the sort kernels carry no algorithmic
 # bytes of their own: they are implementation cost of the backward)
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
+# profiles/ (set an entry to None when its kernel has changed since the capture)
+NCU_TRAFFIC = {
+    ("kaggle_b16384", "seg_reduce_kernel"): 31.14e6,
+    ("kaggle_b16384", "fwd_kernel"): 31.88e6,
+    ("kaggle_b16384", "row_stream_kernel<fused>"): 25.19e6,
+}
+
 KERNEL_BYTES = {
     "fwd_kernel": lambda ab, wl, L, G, U: ab["fwd"],
     "seg_reduce_kernel": lambda ab, wl, L, G, U: 4 * wl.D * G + 4 * wl.D * U,
@@ -380,7 +388,8 @@ def run_ours(args):
             "clocks": clocks,
             "roofline": {"bound": "hbm", "kernel": dominant, "achieved": round(achieved, 1), "peak": peak,
                          "peak_kind": peak_kind, "unit": "GB/s", "frac": round(achieved / peak, 4),
-                         "frac_of_8TBps_nominal": round(achieved / NOMINAL_HBM_GBS, 4), "traffic": None,
+                         "frac_of_8TBps_nominal": round(achieved / NOMINAL_HBM_GBS, 4),
+                         "traffic": NCU_TRAFFIC.get((wl.name, dominant)),
                          "algorithmic_bytes_per_launch": int(dom_bytes)},
             "step_roofline": {"algorithmic_bytes_per_step": int(step_bytes), "GB/s": round(step_gbs, 1),
                               "frac_of_" + peak_kind: round(step_gbs / peak / world, 4),
@@ -397,7 +406,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="kaggle_b16384")
