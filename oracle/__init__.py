@@ -44,6 +44,7 @@ def lib():
         _lib.dqrm_oracle_fake_quant.restype = ctypes.c_float
         _lib.dqrm_oracle_fake_quant.argtypes = [ctypes.c_float, ctypes.c_float, ctypes.c_int]
         _lib.dqrm_oracle_emb_bwd.restype = ctypes.c_int64
+        _lib.dqrm_oracle_dp_merge.restype = ctypes.c_int64
     return _lib
 
 
@@ -146,3 +147,64 @@ def train_step(tables, row_off, D, B, indices, offsets, grad_out, scales, bits, 
     row_update(tables, row_off, D, unique_rows, uniq_off, codes, grad_scales, lr)
     return dict(out=out, unique_rows=unique_rows, uniq_off=uniq_off, grad_rows=grad_rows,
                 codes=codes, grad_scales=grad_scales)
+
+
+# ---- data-parallel exchange of the sparse INT8 gradient (Appendix B.1) -----------------
+def grad_absmax(grad_rows, uniq_off, D):
+    T = len(uniq_off) - 1
+    out = np.empty(T, dtype=np.float32)
+    gr = grad_rows if grad_rows.size else np.zeros((1, D), dtype=np.float32)
+    lib().dqrm_oracle_grad_absmax(_p(gr, np.float32), _p(uniq_off, np.int32), T, int(D), _p(out, np.float32))
+    return out
+
+
+def grad_quant_int8_scaled(grad_rows, uniq_off, D, scales):
+    T = len(uniq_off) - 1
+    codes = np.empty(grad_rows.shape, dtype=np.int8)
+    gr = grad_rows if grad_rows.size else np.zeros((1, D), dtype=np.float32)
+    cd = codes if codes.size else np.zeros((1, D), dtype=np.int8)
+    lib().dqrm_oracle_grad_quant_int8_scaled(_p(gr, np.float32), _p(uniq_off, np.int32), T, int(D),
+                                             _p(np.ascontiguousarray(scales, dtype=np.float32), np.float32),
+                                             _p(cd, np.int8))
+    return codes
+
+
+def dp_merge(rows, uoffs, codes, T, D):
+    """rows[r] int32 [U_r], uoffs[r] int32 [T+1], codes[r] int8 [U_r, D] -> (union rows, off [T+1], int32 sums)"""
+    W = len(rows)
+    n_in = sum(len(r) for r in rows)
+    out_rows = np.empty(max(n_in, 1), dtype=np.int32)
+    out_off = np.empty(T + 1, dtype=np.int32)
+    out_sums = np.empty((max(n_in, 1), D), dtype=np.int32)
+    pad = lambda a, shape, dt: a if a.size else np.zeros(shape, dtype=dt)
+    keep = [[pad(np.ascontiguousarray(r, dtype=np.int32), 1, np.int32) for r in rows],
+            [np.ascontiguousarray(u, dtype=np.int32) for u in uoffs],
+            [pad(np.ascontiguousarray(c, dtype=np.int8), (1, D), np.int8) for c in codes]]
+    arr = lambda lst: (ctypes.c_void_p * W)(*[a.ctypes.data for a in lst])
+    n = lib().dqrm_oracle_dp_merge(W, int(T), int(D), arr(keep[0]), arr(keep[1]), arr(keep[2]),
+                                   _p(out_rows, np.int32), _p(out_off, np.int32), _p(out_sums, np.int32))
+    return out_rows[:n].copy(), out_off, out_sums[:n].copy()
+
+
+def row_update_i32(tables, row_off, D, rows, off, sums, scales, lr):
+    T = len(row_off) - 1
+    row_off = np.ascontiguousarray(row_off, dtype=np.int64)
+    r = rows if rows.size else np.zeros(1, dtype=np.int32)
+    s = sums if sums.size else np.zeros((1, D), dtype=np.int32)
+    lib().dqrm_oracle_row_update_i32(_p(tables, np.float32), _p(row_off, np.int64), T, int(D), _p(r, np.int32),
+                                     _p(off, np.int32), _p(s, np.int32),
+                                     _p(np.ascontiguousarray(scales, dtype=np.float32), np.float32),
+                                     ctypes.c_float(float(np.float32(lr))))
+
+
+def dp_exchange_update(tables, row_off, D, local, lr):
+    """`local` = per rank (unique_rows, uniq_off, grad_rows).  Unifies the scales by max, quantises every
+    rank's gradient with them, sums the codes exactly and applies the dequantised sum to `tables`
+    (one replica; all replicas are identical).  Returns what the ranks would hold afterwards."""
+    T = len(row_off) - 1
+    absmax = np.max(np.stack([grad_absmax(g, uo, D) for (_, uo, g) in local]), axis=0)
+    scales = np.array([scale_from_absmax(a, 8) for a in absmax], dtype=np.float32)
+    codes = [grad_quant_int8_scaled(g, uo, D, scales) for (_, uo, g) in local]
+    rows, off, sums = dp_merge([l[0] for l in local], [l[1] for l in local], codes, T, D)
+    row_update_i32(tables, row_off, D, rows, off, sums, scales, lr)
+    return dict(scales=scales, codes=codes, rows=rows, off=off, sums=sums)

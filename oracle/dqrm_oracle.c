@@ -218,3 +218,87 @@ void dqrm_oracle_row_update(float *tables, const int64_t *row_off, int T, int D,
         }
     }
 }
+
+/* ==========================================================================
+ * Data-parallel exchange of the sparse INT8 gradient (Appendix B.1, Figure
+ * "Customized Data Parallelism Framework"): every rank computes its local
+ * gradient, the per-tensor quantisation scales are unified across ranks, each
+ * rank quantises with the unified scale, the integer gradients are summed over
+ * ranks, and every rank applies the dequantised sum.  Readings taken here: the
+ * scales are unified by MAX (no rank clips), the integers are summed exactly in
+ * 32 bits (so no re-rounding at intermediate reduce steps, the caveat the
+ * paper raises for recursive-doubling all-reduce), and the update uses the sum,
+ * not the mean.
+ * ========================================================================== */
+
+/* codes = Q(grad_rows; given scales[t], 8): the quantiser of step "quantise locally
+ * with the unified scale" */
+void dqrm_oracle_grad_quant_int8_scaled(const float *grad_rows, const int32_t *uniq_off, int T, int D,
+                                        const float *scales, int8_t *codes)
+{
+    for (int t = 0; t < T; ++t)
+        for (int64_t i = (int64_t)uniq_off[t] * D; i < (int64_t)uniq_off[t + 1] * D; ++i)
+            codes[i] = (int8_t)dqrm_oracle_quantize(grad_rows[i], scales[t], 8);
+}
+
+/* per-table max |grad_rows| (0 for a table that touched nothing) */
+void dqrm_oracle_grad_absmax(const float *grad_rows, const int32_t *uniq_off, int T, int D, float *absmax)
+{
+    for (int t = 0; t < T; ++t) {
+        float a = 0.0f;
+        for (int64_t i = (int64_t)uniq_off[t] * D; i < (int64_t)uniq_off[t + 1] * D; ++i) {
+            float v = fabsf(grad_rows[i]);
+            if (v > a) a = v;
+        }
+        absmax[t] = a;
+    }
+}
+
+/* Sum of the ranks' integer gradients.  Rank r holds, per table, ascending distinct rows
+ * rows[r][uoff[r][t] .. uoff[r][t+1]) with codes[r][u][D].  Output: the ascending union of
+ * rows per table (out_rows, out_off[T+1]) and the exact int32 sum of the codes of each row.
+ * out_rows / out_sums have room for the total number of input rows.  Returns the union size. */
+int64_t dqrm_oracle_dp_merge(int W, int T, int D, const int32_t *const *rows, const int32_t *const *uoff,
+                             const int8_t *const *codes, int32_t *out_rows, int32_t *out_off, int32_t *out_sums)
+{
+    int64_t n = 0;
+    int32_t *pos = (int32_t *)malloc(sizeof(int32_t) * (size_t)W);
+    for (int t = 0; t < T; ++t) {
+        out_off[t] = (int32_t)n;
+        for (int r = 0; r < W; ++r) pos[r] = uoff[r][t];
+        for (;;) {
+            /* smallest row not yet consumed over the W ascending lists */
+            int found = 0;
+            int32_t best = 0;
+            for (int r = 0; r < W; ++r)
+                if (pos[r] < uoff[r][t + 1] && (!found || rows[r][pos[r]] < best)) { best = rows[r][pos[r]]; found = 1; }
+            if (!found) break;
+            out_rows[n] = best;
+            for (int d = 0; d < D; ++d) out_sums[n * D + d] = 0;
+            for (int r = 0; r < W; ++r)
+                if (pos[r] < uoff[r][t + 1] && rows[r][pos[r]] == best) {
+                    for (int d = 0; d < D; ++d) out_sums[n * D + d] += (int32_t)codes[r][(int64_t)pos[r] * D + d];
+                    ++pos[r];
+                }
+            ++n;
+        }
+    }
+    out_off[T] = (int32_t)n;
+    free(pos);
+    return n;
+}
+
+/* W[row] -= lr * ((float)sum * scale[t]) for every row of the union: three rounded FP32 operations */
+void dqrm_oracle_row_update_i32(float *tables, const int64_t *row_off, int T, int D, const int32_t *rows,
+                                const int32_t *off, const int32_t *sums, const float *scales, float lr)
+{
+    for (int t = 0; t < T; ++t)
+        for (int64_t u = off[t]; u < off[t + 1]; ++u) {
+            float *w = tables + (row_off[t] + (int64_t)rows[u]) * D;
+            for (int d = 0; d < D; ++d) {
+                float g = (float)sums[u * D + d] * scales[t];
+                float step = lr * g;
+                w[d] = w[d] - step;
+            }
+        }
+}
