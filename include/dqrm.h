@@ -192,6 +192,36 @@ int dqrm_train_step_host(dqrm_ctx *ctx, float *tables, const int32_t *h_indices,
 int dqrm_grad_quant_int8_static(int T, int D, const float *grad_rows, const int32_t *uniq_off,
                                 int8_t *codes, float *grad_scales, void *stream);
 
+/* ---- data-parallel exchange of the sparse INT8 gradient (Appendix B.1) --------------
+ * The paper's data-parallel step, for every parameter tensor: compute the quantisation
+ * scale locally, unify it across ranks, quantise locally with the unified scale, sum the
+ * integer gradients over the ranks, apply the dequantised sum on every rank.  The three
+ * calls below are the local pieces; the two collectives between them (a MAX all-reduce of
+ * T floats, an all-gather of each rank's rows and codes) are the caller's, e.g. NCCL.
+ * Readings: scales are unified by MAX of the abs-max (no rank clips); the integers are
+ * summed exactly in 32 bits; the update uses the sum over ranks, not the mean.
+ *
+ * dqrm_grad_absmax: absmax[t] = max |grad_rows| over table t's rows (0 if none); [T] floats.
+ * dqrm_grad_quant_int8_unified: grad_scales[t] = scale(unified_absmax[t], 8) and
+ *   codes = Q(grad_rows; grad_scales[t], 8).  With unified_absmax = this rank's own abs-max
+ *   it equals dqrm_grad_quant_int8.
+ * dqrm_dp_merge_update: rank r's sparse gradient sits at rows_cat + r*rank_stride (ascending
+ *   distinct rows per table, uoff_cat + r*(T+1) as in dqrm_emb_bwd) with codes at
+ *   codes_cat + r*rank_stride*D.  n_entries = sum of the ranks' row counts and
+ *   max_table_entries = the largest per-table sum over ranks (both from the host copy of
+ *   uoff_cat).  Writes the ascending union of rows per table to union_rows [>= n_entries] /
+ *   union_off [T+1], optionally the int32 sums to sums_out [>= n_entries][D] (may be NULL),
+ *   and updates W[row] -= lr * ((float)sum * grad_scales[t]) with three rounded operations.
+ *   Workspace: dqrm_dp_workspace_bytes(ctx, max n_entries). */
+int dqrm_grad_absmax(dqrm_ctx *ctx, const float *grad_rows, const int32_t *uniq_off, float *absmax, void *stream);
+int dqrm_grad_quant_int8_unified(dqrm_ctx *ctx, const float *grad_rows, const int32_t *uniq_off,
+                                 const float *unified_absmax, int8_t *codes, float *grad_scales, void *stream);
+size_t dqrm_dp_workspace_bytes(const dqrm_ctx *ctx, int64_t max_entries);
+int dqrm_dp_merge_update(dqrm_ctx *ctx, float *tables, int W, int64_t rank_stride, const int32_t *rows_cat,
+                         const int32_t *uoff_cat, const int8_t *codes_cat, const float *grad_scales, float lr,
+                         int64_t n_entries, int64_t max_table_entries, int32_t *union_rows, int32_t *union_off,
+                         int32_t *sums_out, void *workspace, size_t workspace_bytes, void *stream);
+
 /* ---- choice of the backward's sort (no counterpart in the paper) --------------------
  * dqrm_emb_bwd and dqrm_train_step order the batch's lookups by row before they sum
  * duplicates.  path 0 (default): one thread-block cluster per table sorts that table's

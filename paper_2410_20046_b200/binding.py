@@ -42,6 +42,10 @@ SIGNATURES = {
     "dqrm_train_step_host": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _f, _i, _i64, _vp, _sz, _vp]),
     "dqrm_grad_quant_int8_static": (_i, [_i, _i, _vp, _vp, _vp, _vp, _vp]),
     "dqrm_selfcheck_quantizer": (_i, [_vp, _f, _i, ctypes.c_uint32, ctypes.c_uint64, _vp, _vp]),
+    "dqrm_grad_absmax": (_i, [_vp, _vp, _vp, _vp, _vp]),
+    "dqrm_grad_quant_int8_unified": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "dqrm_dp_workspace_bytes": (_sz, [_vp, _i64]),
+    "dqrm_dp_merge_update": (_i, [_vp, _vp, _i, _i64, _vp, _vp, _vp, _vp, _f, _i64, _i64, _vp, _vp, _vp, _vp, _sz, _vp]),
     "dqrm_set_sort_path": (_i, [_vp, _i]),
     "dqrm_set_overlap": (_i, [_vp, _i]),
     "dqrm_launch_count": (_i64, [_vp]),
@@ -163,6 +167,40 @@ class Context:
         self._check("dqrm_selfcheck_quantizer", self.lib.dqrm_selfcheck_quantizer(
             self._h, float(scale), int(bits), int(first_bits) & 0xFFFFFFFF, int(count),
             _ptr(mismatches, torch.int64), _stream(stream)))
+
+    # ---- data-parallel exchange (local pieces) ----
+    def grad_absmax(self, grad_rows, uniq_off, absmax, stream=None):
+        import torch
+
+        self._check("dqrm_grad_absmax", self.lib.dqrm_grad_absmax(
+            self._h, _ptr(grad_rows, torch.float32), _ptr(uniq_off, torch.int32), _ptr(absmax, torch.float32),
+            _stream(stream)))
+
+    def grad_quant_int8_unified(self, grad_rows, uniq_off, unified_absmax, codes, grad_scales, stream=None):
+        import torch
+
+        self._check("dqrm_grad_quant_int8_unified", self.lib.dqrm_grad_quant_int8_unified(
+            self._h, _ptr(grad_rows, torch.float32), _ptr(uniq_off, torch.int32), _ptr(unified_absmax, torch.float32),
+            _ptr(codes, torch.int8), _ptr(grad_scales, torch.float32), _stream(stream)))
+
+    def dp_workspace(self, max_entries: int):
+        """torch-allocated, 256-byte aligned workspace for dp_merge_update -> (tensor, pointer, bytes)"""
+        import torch
+
+        n = int(self.lib.dqrm_dp_workspace_bytes(self._h, int(max_entries)))
+        buf = torch.empty(n + 256, dtype=torch.uint8, device="cuda")
+        return buf, (buf.data_ptr() + 255) // 256 * 256, n
+
+    def dp_merge_update(self, tables, W, rank_stride, rows_cat, uoff_cat, codes_cat, grad_scales, lr, n_entries,
+                        max_table_entries, union_rows, union_off, sums_out, ws, stream=None):
+        import torch
+
+        _, ws_ptr, ws_bytes = ws
+        self._check("dqrm_dp_merge_update", self.lib.dqrm_dp_merge_update(
+            self._h, _ptr(tables, torch.float32), int(W), int(rank_stride), _ptr(rows_cat, torch.int32),
+            _ptr(uoff_cat, torch.int32), _ptr(codes_cat, torch.int8), _ptr(grad_scales, torch.float32), float(lr),
+            int(n_entries), int(max_table_entries), _ptr(union_rows, torch.int32), _ptr(union_off, torch.int32),
+            _ptr(sums_out, torch.int32), ws_ptr, ws_bytes, _stream(stream)))
 
     def set_overlap(self, on: bool):
         self._check("dqrm_set_overlap", self.lib.dqrm_set_overlap(self._h, int(bool(on))))

@@ -195,7 +195,7 @@ const char *dqrm_kernel_name(int kernel_id)
         "begin", "refresh_kernel", "fwd_kernel", "memset", "prepare_kernel", "sort_scan_kernel",
         "sort_scatter_kernel", "seg_count_kernel", "seg_emit_kernel", "seg_reduce_kernel", "seg_fixup_kernel",
         "absmax_kernel", "row_stream_kernel<quant>", "row_stream_kernel<update>", "row_stream_kernel<fused>",
-        "copy", "seg_fixup_big_kernel", "cluster_sort_kernel"};
+        "copy", "seg_fixup_big_kernel", "cluster_sort_kernel", "dp_pack_kernel", "dp_sum_update_kernel"};
     return (kernel_id >= 0 && kernel_id < DQ_K_COUNT) ? names[kernel_id] : "?";
 }
 
@@ -297,6 +297,41 @@ int dqrm_train_step(dqrm_ctx *ctx, float *tables, const int32_t *indices, const 
     rc = dq_launch_bwd_reduce(ctx, grad_out, grad_rows, B, L, workspace, workspace_bytes, st);
     if (rc != DQRM_OK) return rc;
     return dq_launch_quant_update(ctx, tables, unique_rows, uniq_off, grad_rows, absmax, codes, grad_scales, lr, st);
+}
+
+int dqrm_grad_absmax(dqrm_ctx *ctx, const float *grad_rows, const int32_t *uniq_off, float *absmax, void *stream)
+{
+    if (!ctx || !grad_rows || !uniq_off || !absmax) return DQRM_ERR_INVALID_ARG;
+    return dq_launch_grad_absmax(ctx, grad_rows, uniq_off, absmax, as_stream(stream));
+}
+
+int dqrm_grad_quant_int8_unified(dqrm_ctx *ctx, const float *grad_rows, const int32_t *uniq_off,
+                                 const float *unified_absmax, int8_t *codes, float *grad_scales, void *stream)
+{
+    if (!ctx || !grad_rows || !uniq_off || !unified_absmax || !codes || !grad_scales) return DQRM_ERR_INVALID_ARG;
+    return dq_launch_grad_quant_unified(ctx, grad_rows, uniq_off, unified_absmax, codes, grad_scales, as_stream(stream));
+}
+
+size_t dqrm_dp_workspace_bytes(const dqrm_ctx *ctx, int64_t max_entries)
+{
+    if (!ctx || max_entries < 0) return 0;
+    return dq_dp_ws_bytes(ctx, max_entries);
+}
+
+int dqrm_dp_merge_update(dqrm_ctx *ctx, float *tables, int W, int64_t rank_stride, const int32_t *rows_cat,
+                         const int32_t *uoff_cat, const int8_t *codes_cat, const float *grad_scales, float lr,
+                         int64_t n_entries, int64_t max_table_entries, int32_t *union_rows, int32_t *union_off,
+                         int32_t *sums_out, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!ctx || !tables || W < 1 || rank_stride < 0 || !uoff_cat || !grad_scales || !union_off || n_entries < 0 ||
+        n_entries > (int64_t)W * rank_stride || max_table_entries < 0 || max_table_entries > n_entries ||
+        n_entries >= ((int64_t)1 << 31))
+        return DQRM_ERR_INVALID_ARG;
+    if (n_entries > 0 && (!rows_cat || !codes_cat || !union_rows)) return DQRM_ERR_INVALID_ARG;
+    if (!ws_ok(workspace, workspace_bytes, 1)) return DQRM_ERR_WORKSPACE;
+    return dq_launch_dp_merge_update(ctx, tables, W, rank_stride, rows_cat, uoff_cat, codes_cat, grad_scales, lr,
+                                     n_entries, max_table_entries, union_rows, union_off, sums_out, workspace,
+                                     workspace_bytes, as_stream(stream));
 }
 
 size_t dqrm_host_step_workspace_bytes(const dqrm_ctx *ctx, int64_t max_lookups, int64_t max_bags)

@@ -85,7 +85,7 @@ prepare_kernel(const int32_t *__restrict__ indices, const int32_t *__restrict__ 
                const int64_t *__restrict__ row_off, int T, int B, int64_t G, int64_t L,
                u32 *__restrict__ keys, u32 *__restrict__ vals, u32 *__restrict__ ghist,
                u32 *__restrict__ tilehist0, int64_t num_tiles, int passes, int digit_bits,
-               int *__restrict__ status)
+               int payload_position, int *__restrict__ status)
 {
     __shared__ u32 sh[MAX_PASSES * NB_MAX];
     for (int i = threadIdx.x; i < MAX_PASSES * NB_MAX; i += blockDim.x) sh[i] = 0;
@@ -109,7 +109,7 @@ prepare_kernel(const int32_t *__restrict__ indices, const int32_t *__restrict__ 
             }
             const u32 key = (u32)(r0 + idx);
             keys[j] = key;
-            vals[j] = payload;
+            vals[j] = payload_position ? (u32)j : payload;
             for (int p = 0; p < passes; ++p) atomicAdd(&sh[p * NB_MAX + ((key >> (p * digit_bits)) & mask)], 1u);
             atomicAdd(&tilehist0[(size_t)(key & mask) * num_tiles + j / ST_TILE], 1u);
         }
@@ -378,6 +378,13 @@ int launch_reduce(dqrm_ctx *ctx, const Layout &y, char *ws, const u32 *keys, con
 
 }  // namespace
 
+void dq_bwd_ws_views(const dqrm_ctx *ctx, int64_t L, char *ws, const u32 **sorted_vals, const u32 **seg_start)
+{
+    const Layout y = make_layout(ctx, L);
+    *sorted_vals = reinterpret_cast<const u32 *>(ws + y.vals_a);
+    *seg_start = reinterpret_cast<const u32 *>(ws + y.seg_start);
+}
+
 size_t dq_bwd_ws_bytes(const dqrm_ctx *ctx, int64_t L, int64_t G)
 {
     (void)G;
@@ -420,6 +427,7 @@ int dq_launch_bwd_sort(dqrm_ctx *ctx, const int32_t *indices, const int32_t *off
         ca.gp[0] = reinterpret_cast<uint2 *>(ws + y.pairs_a); ca.gp[1] = reinterpret_cast<uint2 *>(ws + y.pairs_b);
         ca.cap = csort::choose_cap((L + ctx->T - 1) / ctx->T);
         ca.status = ctx->d_status;
+        ca.payload_position = ctx->payload_position;
         ca.tile_heads = reinterpret_cast<u32 *>(ws + y.tile_heads);
         const size_t smem = csort::smem_bytes(ca.cap);
         static bool raised = false;
@@ -458,7 +466,7 @@ int dq_launch_bwd_sort(dqrm_ctx *ctx, const int32_t *indices, const int32_t *off
         int64_t cap = (int64_t)ctx->num_sms * 8;
         int grid = (int)(blocks > cap ? cap : blocks);
         prepare_kernel<<<grid, 256, 0, st>>>(indices, offsets, ctx->d_row_off, ctx->T, B, G, L, keys[y.passes & 1], vals[y.passes & 1],
-                                             ghist, thist[0], y.num_tiles, y.passes, y.digit_bits, ctx->d_status);
+                                             ghist, thist[0], y.num_tiles, y.passes, y.digit_bits, ctx->payload_position, ctx->d_status);
         DQRM_CUDA_TRY(ctx, cudaGetLastError());
         dq_mark(ctx, st, DQ_K_PREPARE);
     }

@@ -40,6 +40,7 @@ struct Args {
     u32 *keys_out, *vals_out;       // [L] sorted result
     uint2 *gp[2];                   // [L] global staging of pairs (tables too large for shared memory)
     int cap;                        // pairs per block that fit in shared memory
+    int payload_position;           // 0: payload = row of grad_out [B][T][D]; 1: payload = position of the lookup in indices
     int *status;
     u32 *tile_heads;                // [ceil(L / 2048)] zeroed by the caller: segment heads per tile of the sorted order
 };
@@ -136,7 +137,7 @@ cluster_sort_kernel(const Args a)
             }
             bag = lo;
         }
-        pb0[i] = make_uint2((u32)idx, (u32)(bag * a.T + t));
+        pb0[i] = make_uint2((u32)idx, a.payload_position ? (u32)(tb0 + p) : (u32)(bag * a.T + t));
     }
     if (bad) dq_report(a.status, DQRM_ERR_INDEX_RANGE);
 

@@ -23,6 +23,7 @@ struct dqrm_ctx {
     cudaStream_t side = nullptr;    // second stream: a training step sorts the indices beside its forward
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     int overlap = 1;                // 0: keep everything on the caller's stream
+    int payload_position = 0;       // sort payload: 0 = row of grad_out, 1 = position of the lookup (set by the merge)
     // launch accounting and optional per-launch timing (see dqrm_profile_*)
     int64_t launch_count = 0;
     int prof_on = 0, prof_n = 0;
@@ -33,7 +34,7 @@ struct dqrm_ctx {
 enum {
     DQ_K_BEGIN = 0, DQ_K_REFRESH, DQ_K_FWD, DQ_K_MEMSET, DQ_K_PREPARE, DQ_K_SORT_SCAN, DQ_K_SORT_SCATTER,
     DQ_K_SEG_COUNT, DQ_K_SEG_EMIT, DQ_K_SEG_REDUCE, DQ_K_SEG_FIXUP, DQ_K_ABSMAX, DQ_K_QUANT, DQ_K_UPDATE,
-    DQ_K_QUANT_UPDATE, DQ_K_COPY, DQ_K_SEG_FIXUP_BIG, DQ_K_CLUSTER_SORT, DQ_K_COUNT
+    DQ_K_QUANT_UPDATE, DQ_K_COPY, DQ_K_SEG_FIXUP_BIG, DQ_K_CLUSTER_SORT, DQ_K_DP_PACK, DQ_K_DP_SUM_UPDATE, DQ_K_COUNT
 };
 constexpr int DQ_PROF_MAX = 4096;
 
@@ -195,6 +196,15 @@ int dq_launch_bwd_reduce(dqrm_ctx *ctx, const float *grad_out, float *grad_rows,
                          size_t ws_bytes, cudaStream_t st);
 
 size_t dq_quant_ws_bytes(const dqrm_ctx *ctx);
+int dq_launch_grad_absmax(dqrm_ctx *ctx, const float *grad_rows, const int32_t *uniq_off, float *absmax,
+                          cudaStream_t st);
+int dq_launch_grad_quant_unified(dqrm_ctx *ctx, const float *grad_rows, const int32_t *uniq_off,
+                                 const float *unified_absmax, int8_t *codes, float *grad_scales, cudaStream_t st);
+size_t dq_dp_ws_bytes(const dqrm_ctx *ctx, int64_t max_entries);
+int dq_launch_dp_merge_update(dqrm_ctx *ctx, float *tables, int W, int64_t rank_stride, const int32_t *rows_cat,
+                              const int32_t *uoff_cat, const int8_t *codes_cat, const float *grad_scales, float lr,
+                              int64_t n_entries, int64_t max_table_entries, int32_t *union_rows, int32_t *union_off,
+                              int32_t *sums_out, void *ws, size_t ws_bytes, cudaStream_t st);
 int dq_launch_grad_quant(dqrm_ctx *ctx, const float *grad_rows, const int32_t *uniq_off, int8_t *codes,
                          float *grad_scales, void *ws, size_t ws_bytes, cudaStream_t st);
 int dq_launch_row_update(dqrm_ctx *ctx, float *tables, const int32_t *unique_rows, const int32_t *uniq_off,

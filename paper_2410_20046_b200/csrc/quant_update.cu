@@ -195,6 +195,28 @@ int dq_launch_grad_quant(dqrm_ctx *ctx, const float *grad_rows, const int32_t *u
     return dispatch<MODE_QUANT>(ctx, nullptr, nullptr, uniq_off, grad_rows, absmax, codes, grad_scales, 0.f, st);
 }
 
+// per-table max |grad_rows| as floats (the bit pattern of a non-negative float orders like the uint the kernel maximises)
+int dq_launch_grad_absmax(dqrm_ctx *ctx, const float *grad_rows, const int32_t *uniq_off, float *absmax,
+                          cudaStream_t st)
+{
+    DQRM_CUDA_TRY(ctx, cudaMemsetAsync(absmax, 0, sizeof(float) * ctx->T, st));
+    dq_mark(ctx, st, DQ_K_MEMSET);
+    const size_t smem = (size_t)(ctx->T + 1) * sizeof(int32_t) + (size_t)ctx->T * sizeof(u32);
+    absmax_kernel<<<ctx->num_sms * 8, QU_THREADS, smem, st>>>(grad_rows, uniq_off, ctx->T, ctx->D,
+                                                              reinterpret_cast<u32 *>(absmax));
+    DQRM_CUDA_TRY(ctx, cudaGetLastError());
+    dq_mark(ctx, st, DQ_K_ABSMAX);
+    return DQRM_OK;
+}
+
+// quantise with scales derived from abs-max values that were unified across ranks
+int dq_launch_grad_quant_unified(dqrm_ctx *ctx, const float *grad_rows, const int32_t *uniq_off,
+                                 const float *unified_absmax, int8_t *codes, float *grad_scales, cudaStream_t st)
+{
+    return dispatch<MODE_QUANT>(ctx, nullptr, nullptr, uniq_off, grad_rows, reinterpret_cast<const u32 *>(unified_absmax),
+                                codes, grad_scales, 0.f, st);
+}
+
 int dq_launch_row_update(dqrm_ctx *ctx, float *tables, const int32_t *unique_rows, const int32_t *uniq_off,
                          const int8_t *codes, const float *grad_scales, float lr, cudaStream_t st)
 {
