@@ -257,9 +257,16 @@ def run_ours(args):
 
     # The step is a fixed sequence of launches on fixed buffers, so each pre-staged batch's step is
     # captured once into a CUDA graph and replayed (the launches themselves are unchanged).
+    dp_step = None
+    if args.dp_exchange and world > 1:
+        from paper_2410_20046_b200 import dp
+        dp_step = dp.DataParallelStep(ctx, wl.B, Lmax, world)
+
+        def launch_step(b):      # noqa: F811  (the exchange has host-side size reads, so no graph capture)
+            dp_step.step(tables, b["idx"], b["off"], b["go"], scales, bits, wl.lr, b["L"])
     graphs = None
     launches_per_step = 0
-    if not args.no_graph:
+    if not args.no_graph and dp_step is None:
         try:
             for b in batches[:2]:
                 launch_step(b)                       # first use outside capture (function attributes, caches)
@@ -379,7 +386,8 @@ def run_ours(args):
                        "lookups_per_step_per_gpu": Lavg, "unique_rows_per_step": Uavg, "unique_fraction": Uavg / Lavg,
                        "bits": wl.bits, "grad_bits": 8, "refresh_period": wl.period, "table_bytes": wl.table_bytes(),
                        "launch": "CUDA graph replay per step" if graphs is not None else "direct launches",
-                       "parallelism": f"{world} replica(s), batch sharded by sample, no exchange",
+                       "parallelism": (f"{world} ranks, sparse INT8 gradient exchange every step" if dp_step is not None
+                                       else f"{world} replica(s), batch sharded by sample, no exchange"),
                        "l2": f"{N_BATCHES} distinct pre-staged batches cycled; their rows, gradients and outputs "
                              f"exceed the 126 MB L2 and the table is {wl.table_bytes() / 1e9:.2f} GB"},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -412,6 +420,9 @@ def main():
     ap.add_argument("--workload", default="kaggle_b16384")
     ap.add_argument("--e2e-steps", type=int, default=50)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--dp-exchange", action="store_true",
+                    help="with --gpus N > 1: exchange the sparse INT8 gradient every step (paper's data parallelism) "
+                         "instead of running independent replicas")
     ap.add_argument("--no-graph", action="store_true", help="launch every step directly instead of replaying CUDA graphs")
     ap.add_argument("--no-overlap", action="store_true", help="keep the index sort on the caller's stream")
     ap.add_argument("--sort-path", type=int, default=0, help="0: per-table cluster sort, 1: global radix sort")
