@@ -208,3 +208,27 @@ def dp_exchange_update(tables, row_off, D, local, lr):
     rows, off, sums = dp_merge([l[0] for l in local], [l[1] for l in local], codes, T, D)
     row_update_i32(tables, row_off, D, rows, off, sums, scales, lr)
     return dict(scales=scales, codes=codes, rows=rows, off=off, sums=sums)
+
+
+# ---- bit-packed export and inference (Appendix C) ---------------------------------------
+def pack_tables(tables, row_off, D, scales, bits):
+    """-> uint8 [sum R_t, D*bits/8]"""
+    T = len(row_off) - 1
+    assert bits in (2, 4, 8) and (D * bits) % 8 == 0
+    row_off = np.ascontiguousarray(row_off, dtype=np.int64)
+    packed = np.empty((tables.shape[0], D * bits // 8), dtype=np.uint8)
+    lib().dqrm_oracle_pack_tables(_p(tables, np.float32), _p(row_off, np.int64), T, int(D),
+                                  _p(np.ascontiguousarray(scales, dtype=np.float32), np.float32), int(bits),
+                                  _p(packed, np.uint8))
+    return packed
+
+
+def packed_fwd(packed, row_off, D, B, indices, offsets, scales, bits):
+    T = len(row_off) - 1
+    row_off = np.ascontiguousarray(row_off, dtype=np.int64)
+    out = np.empty((B, T, D), dtype=np.float32)
+    lib().dqrm_oracle_packed_fwd(_p(packed, np.uint8), _p(row_off, np.int64), T, int(D), int(B),
+                                 _p(indices, np.int32), _p(offsets, np.int32),
+                                 _p(np.ascontiguousarray(scales, dtype=np.float32), np.float32), int(bits),
+                                 _p(out, np.float32))
+    return out

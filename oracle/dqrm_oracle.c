@@ -302,3 +302,56 @@ void dqrm_oracle_row_update_i32(float *tables, const int64_t *row_off, int T, in
             }
         }
 }
+
+/* ==========================================================================
+ * Bit-packed export of the quantised tables and inference from them (Appendix C:
+ * the INT4 embedding vectors are bit-packed into bytes to realise the 8x smaller
+ * model; Table "res_tab": 2.161 GB -> 0.270 GB, 12.575 GB -> 1.572 GB).  The paper
+ * gives no layout; here element d of a row sits in byte (d*b)/8 at bit offset
+ * (d*b)%8, lowest bits first, as a b-bit two's-complement code, b in {2, 4, 8},
+ * and a row takes D*b/8 bytes.
+ * ========================================================================== */
+
+void dqrm_oracle_pack_tables(const float *tables, const int64_t *row_off, int T, int D,
+                             const float *scales, int bits, uint8_t *packed /* [sum R_t][D*bits/8] */)
+{
+    const int row_bytes = D * bits / 8;
+    const uint32_t mask = (1u << bits) - 1u;
+    for (int t = 0; t < T; ++t)
+        for (int64_t r = row_off[t]; r < row_off[t + 1]; ++r) {
+            uint8_t *dst = packed + r * row_bytes;
+            memset(dst, 0, (size_t)row_bytes);
+            for (int d = 0; d < D; ++d) {
+                int32_t q = dqrm_oracle_quantize(tables[r * D + d], scales[t], bits);
+                dst[(d * bits) / 8] |= (uint8_t)(((uint32_t)q & mask) << ((d * bits) % 8));
+            }
+        }
+}
+
+static int32_t unpack_code(const uint8_t *row, int d, int bits)
+{
+    uint32_t v = (row[(d * bits) / 8] >> ((d * bits) % 8)) & ((1u << bits) - 1u);
+    if (v & (1u << (bits - 1))) v |= ~((1u << bits) - 1u); /* sign-extend */
+    return (int32_t)v;
+}
+
+/* inference lookup from the packed tables: out[i][t][:] = sum over the bag of code * scale[t] */
+void dqrm_oracle_packed_fwd(const uint8_t *packed, const int64_t *row_off, int T, int D, int B,
+                            const int32_t *indices, const int32_t *offsets, const float *scales, int bits,
+                            float *out)
+{
+    const int row_bytes = D * bits / 8;
+    double *acc = (double *)malloc(sizeof(double) * (size_t)D);
+    for (int t = 0; t < T; ++t)
+        for (int i = 0; i < B; ++i) {
+            int64_t g = (int64_t)t * B + i;
+            for (int d = 0; d < D; ++d) acc[d] = 0.0;
+            for (int32_t j = offsets[g]; j < offsets[g + 1]; ++j) {
+                const uint8_t *row = packed + (row_off[t] + (int64_t)indices[j]) * row_bytes;
+                for (int d = 0; d < D; ++d) acc[d] += (double)dqrm_oracle_dequantize(unpack_code(row, d, bits), scales[t]);
+            }
+            float *o = out + ((int64_t)i * T + t) * D;
+            for (int d = 0; d < D; ++d) o[d] = (float)acc[d];
+        }
+    free(acc);
+}
