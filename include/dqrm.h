@@ -222,6 +222,21 @@ int dqrm_dp_merge_update(dqrm_ctx *ctx, float *tables, int W, int64_t rank_strid
                          int64_t n_entries, int64_t max_table_entries, int32_t *union_rows, int32_t *union_off,
                          int32_t *sums_out, void *workspace, size_t workspace_bytes, void *stream);
 
+/* ---- bit-packed export and inference (Appendix C) ----------------------------------
+ * The deployed model stores the embedding codes bit-packed (Appendix C; Table "res_tab":
+ * 2.161 GB -> 0.270 GB at 4 bits).  The paper gives no layout; here element d of a row sits
+ * in byte (d*bits)/8 at bit offset (d*bits)%8, lowest bits first, as a two's-complement code;
+ * a row takes D*bits/8 bytes and rows follow the arena order.  bits is 2, 4 or 8 for all tables.
+ * dqrm_packed_bytes: size of the packed arena (0 for an unsupported width).
+ * dqrm_pack_tables: packed = Q(tables; scales[t], bits), one pass over the arena.
+ * dqrm_packed_fwd: out[i][t][:] = sum over bag (t,i) of code * scales[t] (bag order, FP64
+ *   accumulator, rounded once) - equal, bit for bit, to dqrm_emb_fwd on the weights and
+ *   scales the tables were packed from. */
+size_t dqrm_packed_bytes(const dqrm_ctx *ctx, int bits);
+int dqrm_pack_tables(dqrm_ctx *ctx, const float *tables, const float *scales, int bits, uint8_t *packed, void *stream);
+int dqrm_packed_fwd(dqrm_ctx *ctx, const uint8_t *packed, const int32_t *indices, const int32_t *offsets,
+                    const float *scales, int bits, float *out, int B, int64_t L, void *stream);
+
 /* ---- choice of the backward's sort (no counterpart in the paper) --------------------
  * dqrm_emb_bwd and dqrm_train_step order the batch's lookups by row before they sum
  * duplicates.  path 0 (default): one thread-block cluster per table sorts that table's

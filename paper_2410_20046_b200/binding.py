@@ -46,6 +46,9 @@ SIGNATURES = {
     "dqrm_grad_quant_int8_unified": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "dqrm_dp_workspace_bytes": (_sz, [_vp, _i64]),
     "dqrm_dp_merge_update": (_i, [_vp, _vp, _i, _i64, _vp, _vp, _vp, _vp, _f, _i64, _i64, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "dqrm_packed_bytes": (_sz, [_vp, _i]),
+    "dqrm_pack_tables": (_i, [_vp, _vp, _vp, _i, _vp, _vp]),
+    "dqrm_packed_fwd": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _vp, _i, _i64, _vp]),
     "dqrm_set_sort_path": (_i, [_vp, _i]),
     "dqrm_set_overlap": (_i, [_vp, _i]),
     "dqrm_launch_count": (_i64, [_vp]),
@@ -201,6 +204,24 @@ class Context:
             _ptr(uoff_cat, torch.int32), _ptr(codes_cat, torch.int8), _ptr(grad_scales, torch.float32), float(lr),
             int(n_entries), int(max_table_entries), _ptr(union_rows, torch.int32), _ptr(union_off, torch.int32),
             _ptr(sums_out, torch.int32), ws_ptr, ws_bytes, _stream(stream)))
+
+    # ---- bit-packed export and inference ----
+    def packed_bytes(self, bits: int) -> int:
+        return int(self.lib.dqrm_packed_bytes(self._h, int(bits)))
+
+    def pack_tables(self, tables, scales, bits, packed, stream=None):
+        import torch
+
+        self._check("dqrm_pack_tables", self.lib.dqrm_pack_tables(
+            self._h, _ptr(tables, torch.float32), _ptr(scales, torch.float32), int(bits), _ptr(packed, torch.uint8),
+            _stream(stream)))
+
+    def packed_fwd(self, packed, indices, offsets, scales, bits, out, *, B, L, stream=None):
+        import torch
+
+        self._check("dqrm_packed_fwd", self.lib.dqrm_packed_fwd(
+            self._h, _ptr(packed, torch.uint8), _ptr(indices, torch.int32), _ptr(offsets, torch.int32),
+            _ptr(scales, torch.float32), int(bits), _ptr(out, torch.float32), int(B), int(L), _stream(stream)))
 
     def set_overlap(self, on: bool):
         self._check("dqrm_set_overlap", self.lib.dqrm_set_overlap(self._h, int(bool(on))))

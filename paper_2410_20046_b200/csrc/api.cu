@@ -195,7 +195,7 @@ const char *dqrm_kernel_name(int kernel_id)
         "begin", "refresh_kernel", "fwd_kernel", "memset", "prepare_kernel", "sort_scan_kernel",
         "sort_scatter_kernel", "seg_count_kernel", "seg_emit_kernel", "seg_reduce_kernel", "seg_fixup_kernel",
         "absmax_kernel", "row_stream_kernel<quant>", "row_stream_kernel<update>", "row_stream_kernel<fused>",
-        "copy", "seg_fixup_big_kernel", "cluster_sort_kernel", "dp_pack_kernel", "dp_sum_update_kernel"};
+        "copy", "seg_fixup_big_kernel", "cluster_sort_kernel", "dp_pack_kernel", "dp_sum_update_kernel", "pack_kernel", "packed_fwd_kernel"};
     return (kernel_id >= 0 && kernel_id < DQ_K_COUNT) ? names[kernel_id] : "?";
 }
 
@@ -332,6 +332,27 @@ int dqrm_dp_merge_update(dqrm_ctx *ctx, float *tables, int W, int64_t rank_strid
     return dq_launch_dp_merge_update(ctx, tables, W, rank_stride, rows_cat, uoff_cat, codes_cat, grad_scales, lr,
                                      n_entries, max_table_entries, union_rows, union_off, sums_out, workspace,
                                      workspace_bytes, as_stream(stream));
+}
+
+size_t dqrm_packed_bytes(const dqrm_ctx *ctx, int bits)
+{
+    if (!ctx || (bits != 2 && bits != 4 && bits != 8)) return 0;
+    return (size_t)ctx->total_rows * (size_t)(ctx->D * bits / 8);
+}
+
+int dqrm_pack_tables(dqrm_ctx *ctx, const float *tables, const float *scales, int bits, uint8_t *packed, void *stream)
+{
+    if (!ctx || !tables || !scales || !packed || (bits != 2 && bits != 4 && bits != 8)) return DQRM_ERR_INVALID_ARG;
+    return dq_launch_pack(ctx, tables, scales, bits, packed, as_stream(stream));
+}
+
+int dqrm_packed_fwd(dqrm_ctx *ctx, const uint8_t *packed, const int32_t *indices, const int32_t *offsets,
+                    const float *scales, int bits, float *out, int B, int64_t L, void *stream)
+{
+    if (!batch_ok(ctx, B, L) || !packed || !offsets || !scales || !out || (bits != 2 && bits != 4 && bits != 8))
+        return DQRM_ERR_INVALID_ARG;
+    if (L > 0 && !indices) return DQRM_ERR_INVALID_ARG;
+    return dq_launch_packed_fwd(ctx, packed, indices, offsets, scales, bits, out, B, L, as_stream(stream));
 }
 
 size_t dqrm_host_step_workspace_bytes(const dqrm_ctx *ctx, int64_t max_lookups, int64_t max_bags)
