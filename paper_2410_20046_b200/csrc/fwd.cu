@@ -10,10 +10,10 @@
 // constants.  A group of LPR lanes owns one row: a feature-16 row is one 64-byte request
 // of four lanes, a feature-64 row one 256-byte request of sixteen.
 //   * fwd_onehot_kernel (launched when L == T*B and no codes are asked for, the Criteo-shaped
-//     training case): a lane group
-//     has NB rows of NB different one-index bags in flight; the pooled value is the
-//     fake-quantised row itself.  A bag that turns out not to hold exactly one index is
-//     pooled by a plain loop.
+//     training case): a warp owns 32 consecutive bags, does their bookkeeping one bag per
+//     lane, then fetches the rows 32/LPR per step with NB steps in flight; the pooled value
+//     is the fake-quantised row itself.  A bag that turns out not to hold exactly one index
+//     is pooled by a plain loop.
 //   * fwd_bags_kernel (any other batch): a lane group walks one bag at a time, NB of its
 //     rows per batch, and sums them in bag order in FP64, rounded once, so the result
 //     does not depend on the launch shape.
@@ -97,67 +97,82 @@ __device__ __forceinline__ void pool_bag_plain(const FwdArgs &a, const TableCtx 
     }
 }
 
+// A warp takes 32 consecutive bags of its table.  The bookkeeping of a bag (its offsets, its index,
+// the range checks) is done once, by the one lane that owns the bag; the rows are then fetched
+// 32/LPR at a time by all lanes, each step reading its bag's index from the owner lane by shuffle.
+// Measured on B200 the kernel is bound by instruction issue, not by HBM, at 256-byte rows, which
+// is why the per-bag work is kept off the per-row path.
 template <int LPR, int CH, bool EXACT>
-__global__ void __launch_bounds__(FW_THREADS, 6)
+__global__ void __launch_bounds__(FW_THREADS, 5)
 fwd_onehot_kernel(const FwdArgs a)
 {
-    constexpr int NB = NBOf<LPR, CH>::v;
-    constexpr int GPB = FW_THREADS / LPR;
+    constexpr int NB = NBOf<LPR, CH>::v;      // row steps in flight
+    constexpr int RPW = 32 / LPR;             // rows one warp instruction covers
+    constexpr int WPB = FW_THREADS / 32;
     const int D = EXACT ? 4 * LPR * CH : a.D;
     const int d4 = D >> 2;
     const int t = blockIdx.y;
-    const int lane = threadIdx.x % LPR;
-    const int grp = threadIdx.x / LPR;
+    const int wlane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = wlane % LPR, grp = wlane / LPR;
     const TableCtx tc = table_ctx(a, t, D);
+    const float4 *tbl_lane = reinterpret_cast<const float4 *>(tc.tbl) + lane;
+    const int TD4 = a.T * d4;                 // 128-bit vectors between the output rows of bags i and i+1
     bool bad = false;
 
-    for (int ib = blockIdx.x * (GPB * NB); ib < a.B; ib += gridDim.x * (GPB * NB)) {
-        int32_t lo[NB], idx[NB];
-        unsigned one = 0;                 // bit b: bag b holds exactly one index
-        unsigned rare = 0;                // bit b: bag b exists but is not a one-index bag
-#pragma unroll
-        for (int b = 0; b < NB; ++b) {
-            const int i = ib + b * GPB + grp;
-            lo[b] = 0; idx[b] = 0;
-            if (i < a.B) {
-                lo[b] = __ldg(a.offsets + tc.g0 + i);
-                const int32_t hi = __ldg(a.offsets + tc.g0 + i + 1);
-                idx[b] = __ldg(a.indices + tc.g0 + i);      // right when offsets are the identity (L == T*B)
-                if (hi - lo[b] == 1 && lo[b] >= 0 && (int64_t)hi <= a.L) one |= 1u << b; else rare |= 1u << b;
+    for (int i0 = (blockIdx.x * WPB + warp) * 32; i0 < a.B; i0 += gridDim.x * (WPB * 32)) {
+        // ---- lane-per-bag bookkeeping
+        const int i = i0 + wlane;
+        int32_t idx = 0;
+        bool single = false;
+        if (i < a.B) {
+            const int32_t lo = __ldg(a.offsets + tc.g0 + i), hi = __ldg(a.offsets + tc.g0 + i + 1);
+            idx = __ldg(a.indices + tc.g0 + i);            // right when the offsets are the identity (L == T*B)
+            single = (hi - lo == 1) & (lo >= 0) & ((int64_t)hi <= a.L);
+            if (single) {
+                if ((int64_t)lo != tc.g0 + i) idx = __ldg(a.indices + lo);
+                idx = clamp_index(idx, tc.nrows, bad);
             }
         }
-#pragma unroll
-        for (int b = 0; b < NB; ++b) {
-            const int i = ib + b * GPB + grp;
-            if (((one >> b) & 1u) && (int64_t)lo[b] != tc.g0 + i) idx[b] = __ldg(a.indices + lo[b]);
-            idx[b] = clamp_index(idx[b], tc.nrows, bad);
-        }
-#pragma unroll
-        for (int c = 0; c < CH; ++c) {
-            const int c4 = c * LPR + lane;
-            float4 v[NB];
-#pragma unroll
-            for (int b = 0; b < NB; ++b)
-                if (((one >> b) & 1u) && (EXACT || c4 < d4))
-                    v[b] = __ldg(reinterpret_cast<const float4 *>(tc.tbl + (int64_t)idx[b] * D) + c4);
-#pragma unroll
-            for (int b = 0; b < NB; ++b) {
-                if (((one >> b) & 1u) && (EXACT || c4 < d4)) {
-                    const int i = ib + b * GPB + grp;
-                    float4 cd, f;
-                    dq_fq4(v[b], tc.qs, cd, f);
-                    reinterpret_cast<float4 *>(a.out + ((int64_t)i * a.T + t) * D)[c4] = f;
-                }
-            }
-        }
-        if (rare) {
+        const unsigned one = __ballot_sync(0xffffffffu, single);
+        unsigned rare = __ballot_sync(0xffffffffu, (i < a.B) && !single);
+        float4 *out_lane = reinterpret_cast<float4 *>(a.out) + ((int64_t)i0 * a.T + t) * d4 + lane;
+
+        // ---- rows, RPW per step, NB steps in flight
 #pragma unroll 1
-            for (int b = 0; b < NB; ++b) {
-                if ((rare >> b) & 1u) {
-                    const int i = ib + b * GPB + grp;
-                    const int32_t l = __ldg(a.offsets + tc.g0 + i), h = __ldg(a.offsets + tc.g0 + i + 1);
-                    pool_bag_plain<LPR, CH>(a, tc, D, d4, l, h, a.out + ((int64_t)i * a.T + t) * D, lane, bad);
+        for (int k0 = 0; k0 < 32; k0 += RPW * NB) {
+            if ((one >> k0) == 0u) break;
+            int32_t ib[NB];
+#pragma unroll
+            for (int b = 0; b < NB; ++b) ib[b] = __shfl_sync(0xffffffffu, idx, (k0 + b * RPW + grp) & 31);
+#pragma unroll
+            for (int c = 0; c < CH; ++c) {
+                const int c4 = c * LPR + lane;
+                float4 v[NB];
+#pragma unroll
+                for (int b = 0; b < NB; ++b) {
+                    const int bag = k0 + b * RPW + grp;
+                    if (bag < 32 && ((one >> bag) & 1u) && (EXACT || c4 < d4))
+                        v[b] = __ldg(tbl_lane + (int64_t)ib[b] * d4 + c * LPR);
                 }
+#pragma unroll
+                for (int b = 0; b < NB; ++b) {
+                    const int bag = k0 + b * RPW + grp;
+                    if (bag < 32 && ((one >> bag) & 1u) && (EXACT || c4 < d4)) {
+                        float4 cd, f;
+                        dq_fq4(v[b], tc.qs, cd, f);
+                        out_lane[(int64_t)bag * TD4 + c * LPR] = f;
+                    }
+                }
+            }
+        }
+        // ---- bags that do not hold exactly one index: pooled by the first lane group, one at a time
+        while (rare) {
+            const int bag = __ffs(rare) - 1;
+            rare &= rare - 1;
+            const int ii = i0 + bag;
+            if (grp == 0) {
+                const int32_t l = __ldg(a.offsets + tc.g0 + ii), h = __ldg(a.offsets + tc.g0 + ii + 1);
+                pool_bag_plain<LPR, CH>(a, tc, D, d4, l, h, a.out + ((int64_t)ii * a.T + t) * D, lane, bad);
             }
         }
     }
@@ -227,7 +242,7 @@ int launch2(dqrm_ctx *ctx, const FwdArgs &a, cudaStream_t st)
     constexpr int GPB = FW_THREADS / LPR;
     // the one-index kernel does not emit codes; a caller that asks for them gets the general kernel
     const bool onehot = a.L == (int64_t)a.T * a.B && a.codes_out == nullptr;
-    const int per_block = onehot ? GPB * NBOf<LPR, CH>::v : GPB;
+    const int per_block = onehot ? FW_THREADS : GPB;
     int bx = (a.B + per_block - 1) / per_block;
     const int cap = (ctx->num_sms * 32 + ctx->T - 1) / ctx->T;     // a few waves over all tables
     if (bx > cap) bx = cap;

@@ -57,86 +57,195 @@ pack_kernel(const float4 *__restrict__ arena4, const int64_t *__restrict__ row_o
     }
 }
 
-template <int BITS>
-__device__ __forceinline__ float4 unpack4(u32 v)
+// ---- packed lookups -------------------------------------------------------------------
+// A lane owns EPL consecutive elements of a row (8 when the feature size allows, else 4): one
+// load of EPL*BITS/8 bytes, EPL/4 128-bit stores.
+template <int BITS, int EPL>
+struct Unit {
+    static constexpr int BYTES = BITS * EPL / 8;
+    u32 w[2];
+    __device__ __forceinline__ void load(const uint8_t *__restrict__ p, int64_t u)
+    {
+        w[1] = 0;
+        if constexpr (BYTES == 1) w[0] = __ldg(p + u);
+        else if constexpr (BYTES == 2) w[0] = __ldg(reinterpret_cast<const uint16_t *>(p) + u);
+        else if constexpr (BYTES == 4) w[0] = __ldg(reinterpret_cast<const u32 *>(p) + u);
+        else { const uint2 v = __ldg(reinterpret_cast<const uint2 *>(p) + u); w[0] = v.x; w[1] = v.y; }
+    }
+    // element k as a float: sign-extended BITS-wide field
+    template <int K>
+    __device__ __forceinline__ float get() const
+    {
+        constexpr int bit = K * BITS, word = bit / 32, off = bit % 32;
+        return (float)((int)(w[word] << (32 - BITS - off)) >> (32 - BITS));
+    }
+    template <int Q>
+    __device__ __forceinline__ float4 quad() const
+    {
+        return make_float4(get<4 * Q>(), get<4 * Q + 1>(), get<4 * Q + 2>(), get<4 * Q + 3>());
+    }
+};
+
+__device__ __forceinline__ float4 scale4(const float4 &q, float s)
 {
-    // sign-extend each BITS-wide field
-    const int sh = 32 - BITS;
-    return make_float4((float)((int)(v << sh) >> sh), (float)((int)(v << (sh - BITS)) >> sh),
-                       (float)((int)(v << (sh - 2 * BITS)) >> sh), (float)((int)(v << (sh - 3 * BITS)) >> sh));
+    const float2 s2 = make_float2(s, s);
+    const float2 a = __fmul2_rn(make_float2(q.x, q.y), s2), b = __fmul2_rn(make_float2(q.z, q.w), s2);
+    return make_float4(a.x, a.y, b.x, b.y);
 }
 
-template <int BITS>
-__device__ __forceinline__ u32 load_packed(const uint8_t *src, int64_t v4)
-{
-    if constexpr (BITS == 2) return src[v4];
-    else if constexpr (BITS == 4) return reinterpret_cast<const uint16_t *>(src)[v4];
-    else return reinterpret_cast<const u32 *>(src)[v4];
-}
+struct PfArgs {
+    const uint8_t *packed;
+    const int64_t *row_off;
+    const int32_t *indices;
+    const int32_t *offsets;
+    const float *scales;
+    float *out;
+    int T, D, B;
+    int64_t L;
+    int *status;
+};
 
-template <int BITS, int LPR, int CH>
-__global__ void __launch_bounds__(PK_THREADS)
-packed_fwd_kernel(const uint8_t *__restrict__ packed, const int64_t *__restrict__ row_off,
-                  const int32_t *__restrict__ indices, const int32_t *__restrict__ offsets,
-                  const float *__restrict__ scales, float *__restrict__ out, int T, int D, int B, int64_t L,
-                  int *__restrict__ status)
+// pools one bag in bag order in FP64 and rounds once (any bag length, zero included)
+template <int BITS, int EPL, int LPR, int CH>
+__device__ __forceinline__ void pool_bag(const PfArgs &a, int64_t r0, int32_t nrows, float s, int units, int32_t lo,
+                                         int32_t hi, float *out_row, int lane, bool &bad)
 {
-    constexpr int GPB = PK_THREADS / LPR;
     constexpr int NB = 4;
-    const int d4 = D >> 2;
-    const int t = blockIdx.y;
-    const int lane = threadIdx.x % LPR, grp = threadIdx.x / LPR;
-    const float s = __ldg(scales + t);
-    const int64_t r0 = __ldg(row_off + t);
-    const int32_t nrows = (int32_t)(__ldg(row_off + t + 1) - r0);
-    const int64_t g0 = (int64_t)t * B;
-    bool bad = false;
-    for (int i = blockIdx.x * GPB + grp; i < B; i += gridDim.x * GPB) {
-        int32_t lo = __ldg(offsets + g0 + i), hi = __ldg(offsets + g0 + i + 1);
-        if (lo < 0 || hi < lo || (int64_t)hi > L) { bad = true; hi = lo = 0; }
-        double acc[CH][4];
+    if (lo < 0 || hi < lo || (int64_t)hi > a.L) { bad = true; hi = lo = 0; }
+    double acc[CH][EPL];
 #pragma unroll
-        for (int c = 0; c < CH; ++c) acc[c][0] = acc[c][1] = acc[c][2] = acc[c][3] = 0.0;
-        for (int32_t j0 = lo; j0 < hi; j0 += NB) {
-            u32 v[NB][CH];
+    for (int c = 0; c < CH; ++c)
 #pragma unroll
-            for (int b = 0; b < NB; ++b) {
-                if (j0 + b < hi) {
-                    int32_t idx = __ldg(indices + j0 + b);
-                    bad |= (idx < 0) | (idx >= nrows);
-                    idx = min(max(idx, 0), nrows - 1);
+        for (int k = 0; k < EPL; ++k) acc[c][k] = 0.0;
+    for (int32_t j0 = lo; j0 < hi; j0 += NB) {
+        Unit<BITS, EPL> v[NB][CH];
 #pragma unroll
-                    for (int c = 0; c < CH; ++c) {
-                        const int c4 = c * LPR + lane;
-                        if (c4 < d4) v[b][c] = load_packed<BITS>(packed, (r0 + idx) * d4 + c4);
-                    }
+        for (int b = 0; b < NB; ++b) {
+            if (j0 + b < hi) {
+                int32_t idx = __ldg(a.indices + j0 + b);
+                bad |= (idx < 0) | (idx >= nrows);
+                idx = min(max(idx, 0), nrows - 1);
+#pragma unroll
+                for (int c = 0; c < CH; ++c) {
+                    const int u = c * LPR + lane;
+                    if (u < units) v[b][c].load(a.packed, (r0 + idx) * units + u);
                 }
             }
+        }
 #pragma unroll
-            for (int b = 0; b < NB; ++b) {
-                if (j0 + b < hi) {
+        for (int b = 0; b < NB; ++b) {
+            if (j0 + b < hi) {
 #pragma unroll
-                    for (int c = 0; c < CH; ++c) {
-                        const int c4 = c * LPR + lane;
-                        if (c4 < d4) {
-                            const float4 q = unpack4<BITS>(v[b][c]);
-                            acc[c][0] += (double)__fmul_rn(q.x, s);
-                            acc[c][1] += (double)__fmul_rn(q.y, s);
-                            acc[c][2] += (double)__fmul_rn(q.z, s);
-                            acc[c][3] += (double)__fmul_rn(q.w, s);
+                for (int c = 0; c < CH; ++c) {
+                    if (c * LPR + lane < units) {
+                        const float4 f0 = scale4(v[b][c].template quad<0>(), s);
+                        acc[c][0] += (double)f0.x; acc[c][1] += (double)f0.y;
+                        acc[c][2] += (double)f0.z; acc[c][3] += (double)f0.w;
+                        if constexpr (EPL == 8) {
+                            const float4 f1 = scale4(v[b][c].template quad<1>(), s);
+                            acc[c][4] += (double)f1.x; acc[c][5] += (double)f1.y;
+                            acc[c][6] += (double)f1.z; acc[c][7] += (double)f1.w;
                         }
                     }
                 }
             }
         }
-        float4 *o = reinterpret_cast<float4 *>(out + ((int64_t)i * T + t) * D);
+    }
+    float4 *o = reinterpret_cast<float4 *>(out_row);
 #pragma unroll
-        for (int c = 0; c < CH; ++c) {
-            const int c4 = c * LPR + lane;
-            if (c4 < d4) o[c4] = make_float4((float)acc[c][0], (float)acc[c][1], (float)acc[c][2], (float)acc[c][3]);
+    for (int c = 0; c < CH; ++c) {
+        const int u = c * LPR + lane;
+        if (u < units) {
+            o[u * (EPL / 4)] = make_float4((float)acc[c][0], (float)acc[c][1], (float)acc[c][2], (float)acc[c][3]);
+            if constexpr (EPL == 8)
+                o[u * 2 + 1] = make_float4((float)acc[c][4], (float)acc[c][5], (float)acc[c][6], (float)acc[c][7]);
         }
     }
-    if (bad) dq_report(status, DQRM_ERR_INDEX_RANGE);
+}
+
+template <int BITS, int EPL, int LPR, int CH>
+__global__ void __launch_bounds__(PK_THREADS)
+packed_fwd_kernel(const PfArgs a)
+{
+    constexpr int GPB = PK_THREADS / LPR;
+    const int units = a.D / EPL;
+    const int t = blockIdx.y;
+    const int lane = threadIdx.x % LPR, grp = threadIdx.x / LPR;
+    const float s = __ldg(a.scales + t);
+    const int64_t r0 = __ldg(a.row_off + t);
+    const int32_t nrows = (int32_t)(__ldg(a.row_off + t + 1) - r0);
+    const int64_t g0 = (int64_t)t * a.B;
+    bool bad = false;
+    for (int i = blockIdx.x * GPB + grp; i < a.B; i += gridDim.x * GPB)
+        pool_bag<BITS, EPL, LPR, CH>(a, r0, nrows, s, units, __ldg(a.offsets + g0 + i), __ldg(a.offsets + g0 + i + 1),
+                                     a.out + ((int64_t)i * a.T + t) * a.D, lane, bad);
+    if (bad) dq_report(a.status, DQRM_ERR_INDEX_RANGE);
+}
+
+// One index per bag (L == T*B, the Criteo shape): a lane group keeps NB rows of NB different bags
+// in flight; the pooled value of a one-index bag is code * scale itself.  A bag that turns out
+// not to hold exactly one index goes through pool_bag.
+template <int BITS, int EPL, int LPR, int CH>
+__global__ void __launch_bounds__(PK_THREADS)
+packed_fwd_onehot_kernel(const PfArgs a)
+{
+    constexpr int NB = CH >= 2 ? 1 : 4;
+    constexpr int GPB = PK_THREADS / LPR;
+    const int units = a.D / EPL;
+    const int t = blockIdx.y;
+    const int lane = threadIdx.x % LPR, grp = threadIdx.x / LPR;
+    const float s = __ldg(a.scales + t);
+    const int64_t r0 = __ldg(a.row_off + t);
+    const int32_t nrows = (int32_t)(__ldg(a.row_off + t + 1) - r0);
+    const int64_t g0 = (int64_t)t * a.B;
+    bool bad = false;
+    for (int ib = blockIdx.x * (GPB * NB); ib < a.B; ib += gridDim.x * (GPB * NB)) {
+        int32_t idx[NB];
+        unsigned one = 0, rare = 0;
+#pragma unroll
+        for (int b = 0; b < NB; ++b) {
+            const int i = ib + b * GPB + grp;
+            idx[b] = 0;
+            if (i < a.B) {
+                const int32_t lo = __ldg(a.offsets + g0 + i), hi = __ldg(a.offsets + g0 + i + 1);
+                if (hi - lo == 1 && lo >= 0 && (int64_t)hi <= a.L) {
+                    one |= 1u << b;
+                    idx[b] = __ldg(a.indices + lo);
+                    bad |= (idx[b] < 0) | (idx[b] >= nrows);
+                    idx[b] = min(max(idx[b], 0), nrows - 1);
+                } else rare |= 1u << b;
+            }
+        }
+#pragma unroll
+        for (int c = 0; c < CH; ++c) {
+            const int u = c * LPR + lane;
+            Unit<BITS, EPL> v[NB];
+#pragma unroll
+            for (int b = 0; b < NB; ++b)
+                if (((one >> b) & 1u) && u < units) v[b].load(a.packed, (r0 + idx[b]) * units + u);
+#pragma unroll
+            for (int b = 0; b < NB; ++b) {
+                if (((one >> b) & 1u) && u < units) {
+                    const int i = ib + b * GPB + grp;
+                    float4 *o = reinterpret_cast<float4 *>(a.out + ((int64_t)i * a.T + t) * a.D) + u * (EPL / 4);
+                    __stcs(o, scale4(v[b].template quad<0>(), s));
+                    if constexpr (EPL == 8) __stcs(o + 1, scale4(v[b].template quad<1>(), s));
+                }
+            }
+        }
+        if (rare) {
+#pragma unroll 1
+            for (int b = 0; b < NB; ++b) {
+                if ((rare >> b) & 1u) {
+                    const int i = ib + b * GPB + grp;
+                    pool_bag<BITS, EPL, LPR, CH>(a, r0, nrows, s, units, __ldg(a.offsets + g0 + i),
+                                                 __ldg(a.offsets + g0 + i + 1), a.out + ((int64_t)i * a.T + t) * a.D,
+                                                 lane, bad);
+                }
+            }
+        }
+    }
+    if (bad) dq_report(a.status, DQRM_ERR_INDEX_RANGE);
 }
 
 template <int BITS>
@@ -151,39 +260,46 @@ int launch_pack(dqrm_ctx *ctx, const float *tables, const float *scales, uint8_t
     return DQRM_OK;
 }
 
-template <int BITS, int LPR, int CH>
-int launch_pfwd(dqrm_ctx *ctx, const uint8_t *packed, const int32_t *indices, const int32_t *offsets,
-                const float *scales, float *out, int B, int64_t L, cudaStream_t st)
+template <int BITS, int EPL, int LPR, int CH>
+int launch_pfwd(dqrm_ctx *ctx, const PfArgs &a, cudaStream_t st)
 {
     constexpr int GPB = PK_THREADS / LPR;
-    int bx = (B + GPB - 1) / GPB;
+    const bool onehot = a.L == (int64_t)a.T * a.B;
+    const int per_block = onehot ? GPB * (CH >= 2 ? 1 : 4) : GPB;
+    int bx = (a.B + per_block - 1) / per_block;
     const int cap = (ctx->num_sms * 32 + ctx->T - 1) / ctx->T;
     if (bx > cap) bx = cap;
     if (bx < 1) bx = 1;
     dim3 grid((unsigned)bx, (unsigned)ctx->T);
-    packed_fwd_kernel<BITS, LPR, CH><<<grid, PK_THREADS, 0, st>>>(packed, ctx->d_row_off, indices, offsets, scales, out,
-                                                                  ctx->T, ctx->D, B, L, ctx->d_status);
+    if (onehot) packed_fwd_onehot_kernel<BITS, EPL, LPR, CH><<<grid, PK_THREADS, 0, st>>>(a);
+    else packed_fwd_kernel<BITS, EPL, LPR, CH><<<grid, PK_THREADS, 0, st>>>(a);
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
     dq_mark(ctx, st, DQ_K_PACKED_FWD);
     return DQRM_OK;
 }
 
-template <int BITS>
-int dispatch_pfwd(dqrm_ctx *ctx, const uint8_t *packed, const int32_t *indices, const int32_t *offsets,
-                  const float *scales, float *out, int B, int64_t L, cudaStream_t st)
+template <int BITS, int EPL>
+int dispatch_pfwd2(dqrm_ctx *ctx, const PfArgs &a, cudaStream_t st)
 {
-    const int d4 = ctx->D / 4;
-#define DQ_PF(LPR, CH) return launch_pfwd<BITS, LPR, CH>(ctx, packed, indices, offsets, scales, out, B, L, st)
-    if (d4 <= 1) DQ_PF(1, 1);
-    if (d4 <= 2) DQ_PF(2, 1);
-    if (d4 <= 4) DQ_PF(4, 1);
-    if (d4 <= 8) DQ_PF(8, 1);
-    if (d4 <= 16) DQ_PF(16, 1);
-    if (d4 <= 32) DQ_PF(32, 1);
-    if (d4 <= 64) DQ_PF(32, 2);
-    if (d4 <= 128) DQ_PF(32, 4);
+    const int units = a.D / EPL;
+#define DQ_PF(LPR, CH) return launch_pfwd<BITS, EPL, LPR, CH>(ctx, a, st)
+    if (units <= 1) DQ_PF(1, 1);
+    if (units <= 2) DQ_PF(2, 1);
+    if (units <= 4) DQ_PF(4, 1);
+    if (units <= 8) DQ_PF(8, 1);
+    if (units <= 16) DQ_PF(16, 1);
+    if (units <= 32) DQ_PF(32, 1);
+    if (units <= 64) DQ_PF(32, 2);
+    if (units <= 128) DQ_PF(32, 4);
     DQ_PF(32, 8);
 #undef DQ_PF
+}
+
+template <int BITS>
+int dispatch_pfwd(dqrm_ctx *ctx, const PfArgs &a, cudaStream_t st)
+{
+    if (a.D % 8 == 0) return dispatch_pfwd2<BITS, 8>(ctx, a, st);
+    return dispatch_pfwd2<BITS, 4>(ctx, a, st);
 }
 
 }  // namespace
@@ -198,7 +314,8 @@ int dq_launch_pack(dqrm_ctx *ctx, const float *tables, const float *scales, int 
 int dq_launch_packed_fwd(dqrm_ctx *ctx, const uint8_t *packed, const int32_t *indices, const int32_t *offsets,
                          const float *scales, int bits, float *out, int B, int64_t L, cudaStream_t st)
 {
-    if (bits == 2) return dispatch_pfwd<2>(ctx, packed, indices, offsets, scales, out, B, L, st);
-    if (bits == 4) return dispatch_pfwd<4>(ctx, packed, indices, offsets, scales, out, B, L, st);
-    return dispatch_pfwd<8>(ctx, packed, indices, offsets, scales, out, B, L, st);
+    const PfArgs a{packed, ctx->d_row_off, indices, offsets, scales, out, ctx->T, ctx->D, B, L, ctx->d_status};
+    if (bits == 2) return dispatch_pfwd<2>(ctx, a, st);
+    if (bits == 4) return dispatch_pfwd<4>(ctx, a, st);
+    return dispatch_pfwd<8>(ctx, a, st);
 }

@@ -104,3 +104,29 @@ def test_pack_rejects_unsupported_width():
         c.ctx.pack_tables(c.empty((c.wl.total_rows, c.wl.D), t.float32), c.empty(c.wl.T, t.float32), 3,
                           c.empty(16, t.uint8))
     c.ctx.close()
+
+
+def test_packed_lookup_uneven_bags_with_one_index_per_bag_on_average(oracle):
+    # L == T*B sends the call down the one-index path; bags of zero and two indices must still pool right
+    wl = W.scaled_down(W.kaggle(), total_rows=20_000, B=200, name="uneven")
+    c = Case(wl)
+    t = c.torch
+    tables = W.tables_np(wl)
+    scales, _ = oracle.scale_refresh(tables, c.row_off, wl.D, np.full(wl.T, 4, dtype=np.int32))
+    idx, off, _ = c.batch(0)
+    assert len(idx) == wl.T * wl.B
+    off = off.copy()
+    rng = np.random.default_rng(3)
+    for g in rng.choice(np.arange(1, wl.T * wl.B - 1), size=150, replace=False):
+        if g % wl.B:                       # keep each table's range: only move boundaries inside a table
+            off[g] += 1 if off[g + 1] - off[g] >= 1 and g % 2 else 0
+    off = np.minimum.accumulate(off[::-1])[::-1].astype(np.int32)
+    packed = oracle.pack_tables(tables, c.row_off, wl.D, scales, 4)
+    want = oracle.packed_fwd(packed, c.row_off, wl.D, wl.B, idx, off, scales, 4)
+    lens = np.diff(off)
+    assert (lens == 0).any() and (lens == 2).any()
+    out = c.empty((wl.B, wl.T, wl.D), t.float32)
+    c.ctx.packed_fwd(c.dev(packed), c.dev(idx), c.dev(off), c.dev(scales), 4, out, B=wl.B, L=len(idx))
+    c.ctx.raise_on_device_error()
+    assert bit_equal(out.cpu().numpy(), want)
+    c.ctx.close()
