@@ -26,7 +26,7 @@ constexpr int FW_THREADS = 256;
 // bytes, two for 256- and 512-byte rows (more resident warps beat deeper unrolling), one
 // when a lane already holds several 128-bit pieces of every row
 template <int LPR, int CH>
-struct NBOf { static constexpr int v = CH >= 2 ? 1 : (LPR >= 16 ? 2 : 4); };
+struct NBOf { static constexpr int v = CH >= 2 ? 1 : 4; };
 
 struct FwdArgs {
     const float *tables;
