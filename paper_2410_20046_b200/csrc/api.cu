@@ -294,7 +294,7 @@ int dqrm_train_step(dqrm_ctx *ctx, float *tables, const int32_t *indices, const 
             rc = dq_launch_bwd_sort(ctx, indices, offsets, unique_rows, uniq_off, B, L, workspace, workspace_bytes, st, &absmax);
     }
     if (rc != DQRM_OK) return rc;
-    rc = dq_launch_bwd_reduce(ctx, grad_out, grad_rows, B, L, workspace, workspace_bytes, st);
+    rc = dq_launch_bwd_reduce(ctx, grad_out, uniq_off, grad_rows, B, L, workspace, workspace_bytes, st);
     if (rc != DQRM_OK) return rc;
     return dq_launch_quant_update(ctx, tables, unique_rows, uniq_off, grad_rows, absmax, codes, grad_scales, lr, st);
 }

@@ -339,7 +339,7 @@ seg_emit_kernel(const u32 *__restrict__ keys, int64_t L, const u32 *__restrict__
 // RL/RV/RC: lanes per row, floats per lane vector and vectors per lane of the reduce kernel;
 // LPR/CH: the same for the fix-up kernels (always 128-bit vectors)
 template <int RL, int RV, int RC, int LPR, int CH>
-int launch_reduce(dqrm_ctx *ctx, const Layout &y, char *ws, const u32 *keys, const u32 *vals,
+int launch_reduce(dqrm_ctx *ctx, const Layout &y, char *ws, const u32 *keys, const u32 *vals, const int32_t *uniq_off,
                   const float *grad_out, float *grad_rows, int64_t L, int64_t G, cudaStream_t st)
 {
     using namespace segred;
@@ -353,9 +353,10 @@ int launch_reduce(dqrm_ctx *ctx, const Layout &y, char *ws, const u32 *keys, con
     const u32 *seg_start = reinterpret_cast<const u32 *>(ws + y.seg_start);
     double *partials = reinterpret_cast<double *>(ws + y.partials);
     u32 *long_list = reinterpret_cast<u32 *>(ws + y.long_list);
-    seg_reduce_kernel<RL, RV, RC><<<grid, 256, smem, st>>>(
-        keys, vals, seg_start, reinterpret_cast<const u32 *>(ws + y.chunk_first), grad_out, grad_rows, partials,
-        long_list, counters, absmax, ctx->d_row_off, ctx->T, ctx->D, L, G, y.num_chunks, ctx->d_status);
+    const size_t red_smem = (size_t)(ctx->T + 1) * sizeof(u32) + (size_t)gpb * SEG_CHUNK * sizeof(u32);
+    seg_reduce_kernel<RL, RV, RC><<<grid, 256, red_smem, st>>>(
+        keys, vals, seg_start, reinterpret_cast<const u32 *>(ws + y.chunk_first), uniq_off, grad_out, grad_rows,
+        partials, long_list, counters, absmax, ctx->T, ctx->D, L, G, y.num_chunks, ctx->d_status);
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
     dq_mark(ctx, st, DQ_K_SEG_REDUCE);
     int64_t fblocks = (y.num_chunks + 7) / 8;                // at most one cut segment per chunk, a warp each
@@ -502,7 +503,7 @@ int dq_launch_bwd_sort(dqrm_ctx *ctx, const int32_t *indices, const int32_t *off
 }
 
 // second half: segmented sum of the upstream gradient over the sorted lookups
-int dq_launch_bwd_reduce(dqrm_ctx *ctx, const float *grad_out, float *grad_rows, int B, int64_t L,
+int dq_launch_bwd_reduce(dqrm_ctx *ctx, const float *grad_out, const int32_t *uniq_off, float *grad_rows, int B, int64_t L,
                          void *ws_, size_t ws_bytes, cudaStream_t st)
 {
     const Layout y = make_layout(ctx, L);
@@ -514,10 +515,10 @@ int dq_launch_bwd_reduce(dqrm_ctx *ctx, const float *grad_out, float *grad_rows,
     const u32 *skeys = reinterpret_cast<const u32 *>(ws + y.keys_a), *svals = reinterpret_cast<const u32 *>(ws + y.vals_a);
     const int D = ctx->D, d4 = D / 4;
 #define DQ_RED(RL, RV, RC, LPR, CH) \
-    return launch_reduce<RL, RV, RC, LPR, CH>(ctx, y, ws, skeys, svals, grad_out, grad_rows, L, G, st)
+    return launch_reduce<RL, RV, RC, LPR, CH>(ctx, y, ws, skeys, svals, uniq_off, grad_out, grad_rows, L, G, st)
     if (D <= 4) DQ_RED(4, 1, 1, 1, 1);
     if (D <= 8) DQ_RED(8, 1, 1, 2, 1);
-    if (D <= 16) DQ_RED(16, 1, 1, 4, 1);
+    if (D <= 16) DQ_RED(4, 4, 1, 4, 1);
     if (D <= 32) DQ_RED(16, 2, 1, 8, 1);
     if (D <= 64) DQ_RED(16, 4, 1, 16, 1);
     if (d4 <= 32) DQ_RED(32, 4, 1, 32, 1);
@@ -533,5 +534,5 @@ int dq_launch_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, 
 {
     int rc = dq_launch_bwd_sort(ctx, indices, offsets, unique_rows, uniq_off, B, L, ws, ws_bytes, st, absmax_bits_out);
     if (rc != DQRM_OK) return rc;
-    return dq_launch_bwd_reduce(ctx, grad_out, grad_rows, B, L, ws, ws_bytes, st);
+    return dq_launch_bwd_reduce(ctx, grad_out, uniq_off, grad_rows, B, L, ws, ws_bytes, st);
 }

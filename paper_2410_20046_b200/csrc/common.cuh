@@ -192,7 +192,8 @@ int dq_launch_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, 
 int dq_launch_bwd_sort(dqrm_ctx *ctx, const int32_t *indices, const int32_t *offsets, int32_t *unique_rows,
                        int32_t *uniq_off, int B, int64_t L, void *ws, size_t ws_bytes, cudaStream_t st,
                        const u32 **absmax_bits_out);
-int dq_launch_bwd_reduce(dqrm_ctx *ctx, const float *grad_out, float *grad_rows, int B, int64_t L, void *ws,
+int dq_launch_bwd_reduce(dqrm_ctx *ctx, const float *grad_out, const int32_t *uniq_off, float *grad_rows, int B,
+                         int64_t L, void *ws,
                          size_t ws_bytes, cudaStream_t st);
 
 size_t dq_quant_ws_bytes(const dqrm_ctx *ctx);

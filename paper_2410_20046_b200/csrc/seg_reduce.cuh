@@ -38,10 +38,10 @@ __device__ __forceinline__ float group_max(float m)
     return m;
 }
 
-// running abs-max of one table at a time (keys only ascend along a lane group's work)
+// running abs-max of one table at a time (segment numbers only ascend along a lane group's work)
 struct AbsmaxTracker {
     int t = -1;
-    int64_t t_end = -1;
+    u32 u_end = 0;          // first segment past table t
     float m = 0.f;
 };
 
@@ -53,14 +53,19 @@ __device__ __forceinline__ void absmax_push(AbsmaxTracker &tr, u32 *absmax)
     tr.m = 0.f;
 }
 
+// s_uoff[t] = first segment (unique row) of table t, s_uoff[T] = number of segments
 template <int LPR>
-__device__ __forceinline__ void absmax_note(AbsmaxTracker &tr, u32 key, float m, const int64_t *s_off, int T,
-                                            u32 *absmax)
+__device__ __forceinline__ void absmax_note(AbsmaxTracker &tr, u32 u, float m, const u32 *s_uoff, int T, u32 *absmax)
 {
-    if ((int64_t)key >= tr.t_end) {
+    if (u >= tr.u_end) {
         absmax_push<LPR>(tr, absmax);
-        tr.t = dq_table_of(s_off, T, (int64_t)key);
-        tr.t_end = s_off[tr.t + 1];
+        int lo = 0, hi = T;              // invariant: s_uoff[lo] <= u < s_uoff[hi]
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (s_uoff[mid] <= u) lo = mid; else hi = mid;
+        }
+        tr.t = lo;
+        tr.u_end = s_uoff[lo + 1];
     }
     tr.m = fmaxf(tr.m, m);
 }
@@ -97,29 +102,34 @@ __device__ __forceinline__ void vec_add(double (&acc)[VEC], const typename Vec<V
 
 // One lane group (LPR lanes) owns one chunk of 32 sorted entries and walks it in order,
 // NB upstream-gradient rows in flight at a time.  Lane `lane` holds, for ch < CH, the VEC
-// consecutive features starting at (ch*LPR + lane)*VEC; narrow rows use VEC = 1 or 2 so
-// that a row is still spread over 16 lanes and small feature sizes keep enough threads.
+// consecutive features starting at (ch*LPR + lane)*VEC.  Per chunk, one lane per entry compares
+// neighbouring keys once; the resulting bit mask of segment heads and the payloads (parked in
+// shared memory) are all the walk needs, so an entry costs one shared load, one address, one
+// 128-bit load, a bit test and the FP64 adds.
 template <int LPR, int VEC, int CH>
 __global__ void __launch_bounds__(256)
 seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
                   const u32 *__restrict__ seg_start, const u32 *__restrict__ chunk_first,
+                  const int32_t *__restrict__ uniq_off,
                   const float *__restrict__ grad_out, float *__restrict__ grad_rows,
                   double *__restrict__ partials, u32 *__restrict__ long_list, u32 *__restrict__ counters,
-                  u32 *__restrict__ absmax, const int64_t *__restrict__ row_off, int T, int D,
+                  u32 *__restrict__ absmax, int T, int D,
                   int64_t L, int64_t G, int64_t num_chunks, int *__restrict__ status)
 {
     extern __shared__ unsigned char smem_raw[];
-    int64_t *s_off = reinterpret_cast<int64_t *>(smem_raw);
-    for (int t = threadIdx.x; t <= T; t += blockDim.x) s_off[t] = row_off[t];
+    u32 *s_uoff = reinterpret_cast<u32 *>(smem_raw);                                     // [T+1]
+    u32 *s_vals = s_uoff + (T + 1) + (size_t)(threadIdx.x / LPR) * CHUNK;                // this group's [CHUNK]
+    for (int t = threadIdx.x; t <= T; t += blockDim.x) s_uoff[t] = (u32)uniq_off[t];
     __syncthreads();
 
     typedef typename Vec<VEC>::type vec_t;
-    constexpr int NB = VEC == 4 ? 4 : 8;          // rows in flight per lane
-    constexpr int EPL = CHUNK / LPR;              // chunk entries whose key and payload a lane holds
+    constexpr int NB = (VEC == 4 && LPR > 4) ? 4 : 8;   // rows in flight per lane
+    constexpr int EPL = CHUNK / LPR;              // chunk entries one lane looks at
     const int dv = D / VEC;                       // vectors per row
     const int lane = threadIdx.x % LPR;
     const u32 gmask = group_mask<LPR>();
     const int gbase = (threadIdx.x & 31) / LPR * LPR;
+    const vec_t *g_lane = reinterpret_cast<const vec_t *>(grad_out) + lane;
     const int64_t group = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / LPR;
     const int64_t n_groups = (int64_t)gridDim.x * blockDim.x / LPR;
     AbsmaxTracker tr;
@@ -127,38 +137,41 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
 
     for (int64_t c = group; c < num_chunks; c += n_groups) {
         const int64_t i0 = c * CHUNK;
-        const int64_t i1 = min(i0 + (int64_t)CHUNK, L);
-        // the chunk's keys and payloads: one coalesced load, then broadcast by shuffles
-        u32 kreg[EPL], vreg[EPL];
+        const int n = (int)(min(i0 + (int64_t)CHUNK, L) - i0);
+        // heads: entry e starts a segment when its key differs from the key before it
+        u32 heads = 0;
+        __syncwarp(gmask);                        // the previous chunk's payloads are no longer read
 #pragma unroll
         for (int j = 0; j < EPL; ++j) {
-            const int64_t i = i0 + j * LPR + lane;
-            kreg[j] = i < i1 ? keys[i] : 0xFFFFFFFFu;
-            vreg[j] = i < i1 ? vals[i] : 0u;
-            if (i < i1 && (int64_t)vreg[j] >= G) { bad = true; vreg[j] = 0u; }
+            const int e = j * LPR + lane;
+            bool head = false;
+            if (e < n) {
+                const int64_t i = i0 + e;
+                u32 v = vals[i];
+                if ((int64_t)v >= G) { bad = true; v = 0u; }
+                s_vals[e] = v;
+                head = (i == 0) || (keys[i] != keys[i - 1]);
+            }
+            const u32 bits = (__ballot_sync(gmask, head) >> gbase) & (LPR >= 32 ? 0xffffffffu : ((1u << LPR) - 1u));
+            heads |= bits << (j * LPR);
         }
-        auto bcast = [&](const u32 (&reg)[EPL], int e) {     // entry e of the chunk, e uniform in the group
-            u32 r = reg[0];
-#pragma unroll
-            for (int j = 1; j < EPL; ++j) if (e / LPR == j) r = reg[j];
-            return __shfl_sync(gmask, r, gbase + (e % LPR));
-        };
-        // does the chunk's first run begin here, does its last run end here?  (neighbouring keys)
-        const bool first_begins = (i0 == 0) || (keys[i0 - 1] != bcast(kreg, 0));
-        const bool last_ends = (i1 == L) || (keys[i1] != bcast(kreg, (int)(i1 - i0) - 1));
+        __syncwarp(gmask);
+        // does the chunk's first run begin here, does its last run end here?
+        const bool first_begins = heads & 1u;
+        const bool last_ends = (i0 + n == L) || (keys[i0 + n] != keys[i0 + n - 1]);
+        heads &= ~1u;                             // the walk starts a run at entry 0 either way
         u32 u = chunk_first[c];
-        u32 cur_key = bcast(kreg, 0);
-        int64_t run_start = i0;
+        int run_start = 0;
         double acc[CH][VEC];
 #pragma unroll
         for (int ch = 0; ch < CH; ++ch)
 #pragma unroll
             for (int q = 0; q < VEC; ++q) acc[ch][q] = 0.0;
 
-        // closes run [a, b) of segment u; runs strictly inside the chunk are whole segments
-        auto flush = [&](int64_t a, int64_t b) {
-            const bool begins = (a != i0) || first_begins;
-            const bool ends = (b != i1) || last_ends;
+        // closes run [a, b) (chunk-relative) of segment u; runs strictly inside the chunk are whole segments
+        auto flush = [&](int a, int b) {
+            const bool begins = (a != 0) || first_begins;
+            const bool ends = (b != n) || last_ends;
             if (begins && ends) {
                 float m = 0.f;
 #pragma unroll
@@ -178,7 +191,7 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
                         }
                     }
                 }
-                absmax_note<LPR>(tr, cur_key, m, s_off, T, absmax);
+                absmax_note<LPR>(tr, u, m, s_uoff, T, absmax);
             } else {
                 double *pdst = partials + ((size_t)c * 2 + (begins ? 1 : 0)) * D;
 #pragma unroll
@@ -200,48 +213,37 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
             }
         };
 
-        for (int64_t ib = i0; ib < i1; ib += NB) {
-            u32 k[NB], v[NB];
-#pragma unroll
-            for (int e = 0; e < NB; ++e) {
-                const int ec = (int)(ib - i0) + e;           // < CHUNK because NB divides CHUNK
-                k[e] = bcast(kreg, ec);
-                v[e] = bcast(vreg, ec);
-            }
+        for (int eb = 0; eb < n; eb += NB) {
             vec_t r[NB][CH];
 #pragma unroll
             for (int e = 0; e < NB; ++e) {
-                if (ib + e < i1) {
-                    const vec_t *src = reinterpret_cast<const vec_t *>(grad_out + (int64_t)v[e] * D);
+                if (eb + e < n) {
+                    const vec_t *src = g_lane + (int64_t)s_vals[eb + e] * dv;
 #pragma unroll
-                    for (int ch = 0; ch < CH; ++ch) {
-                        const int cv = ch * LPR + lane;
-                        if (cv < dv) r[e][ch] = __ldg(src + cv);
-                    }
+                    for (int ch = 0; ch < CH; ++ch)
+                        if (ch * LPR + lane < dv) r[e][ch] = __ldg(src + ch * LPR);
                 }
             }
+            const u32 hb = heads >> eb;
 #pragma unroll
             for (int e = 0; e < NB; ++e) {
-                if (ib + e < i1) {
-                    if (k[e] != cur_key) {
-                        flush(run_start, ib + e);
+                if (eb + e < n) {
+                    if ((hb >> e) & 1u) {
+                        flush(run_start, eb + e);
                         u += 1;
-                        cur_key = k[e];
-                        run_start = ib + e;
+                        run_start = eb + e;
 #pragma unroll
                         for (int ch = 0; ch < CH; ++ch)
 #pragma unroll
                             for (int q = 0; q < VEC; ++q) acc[ch][q] = 0.0;
                     }
 #pragma unroll
-                    for (int ch = 0; ch < CH; ++ch) {
-                        const int cv = ch * LPR + lane;
-                        if (cv < dv) vec_add<VEC>(acc[ch], r[e][ch]);
-                    }
+                    for (int ch = 0; ch < CH; ++ch)
+                        if (ch * LPR + lane < dv) vec_add<VEC>(acc[ch], r[e][ch]);
                 }
             }
         }
-        flush(run_start, i1);
+        flush(run_start, n);
     }
     absmax_push<LPR>(tr, absmax);      // group-uniform: all lanes of a group walk the same chunks
     if (bad) dq_report(status, DQRM_ERR_INDEX_RANGE);
