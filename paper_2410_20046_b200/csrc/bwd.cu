@@ -306,6 +306,13 @@ seg_emit_kernel(const u32 *__restrict__ keys, int64_t L, const u32 *__restrict__
     for (int w = 0; w < warp; ++w) woff += wsum[w];
     u32 heads_before = tile_prefix + woff + incl - c;   // heads strictly before entry i0
 
+    // tables of the keys: found once for the key before this thread's entries, then only advanced
+    // (keys ascend), so a head costs a comparison instead of two searches
+    int t_prev = -1, t = 0;
+    if (n > 0) {
+        if (i0 > 0) t_prev = dq_table_of(s_off, T, (int64_t)prev0);
+        t = t_prev < 0 ? 0 : t_prev;
+    }
     u32 prev = prev0;
 #pragma unroll
     for (int e = 0; e < ST_ITEMS; ++e) {
@@ -316,18 +323,17 @@ seg_emit_kernel(const u32 *__restrict__ keys, int64_t L, const u32 *__restrict__
                 const u32 u = heads_before;
                 heads_before += 1;
                 seg_start[u] = (u32)i;
-                const int t = dq_table_of(s_off, T, (int64_t)k[e]);
+                while ((int64_t)k[e] >= s_off[t + 1]) ++t;        // ends: every key lies below s_off[T]
                 unique_rows[u] = (int32_t)((int64_t)k[e] - s_off[t]);
-                const int t_prev = (i == 0) ? -1 : dq_table_of(s_off, T, (int64_t)prev);
                 for (int tt = t_prev + 1; tt <= t; ++tt) uniq_off[tt] = (int32_t)u;
+                t_prev = t;
             }
             const u32 u_of_i = heads_before - 1;
             if ((i % SEG_CHUNK) == 0) chunk_first[i / SEG_CHUNK] = u_of_i;
             if (i == L - 1) {
                 const u32 U = u_of_i + 1;
                 seg_start[U] = (u32)L;
-                const int t = dq_table_of(s_off, T, (int64_t)k[e]);
-                for (int tt = t + 1; tt <= T; ++tt) uniq_off[tt] = (int32_t)U;
+                for (int tt = t_prev + 1; tt <= T; ++tt) uniq_off[tt] = (int32_t)U;
                 counters[CNT_U] = U;
             }
         }
