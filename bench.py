@@ -251,9 +251,41 @@ def run_ours(args):
     codes = torch.empty((Lmax, wl.D), dtype=torch.int8, device="cuda")
     gs = torch.empty(wl.T, dtype=torch.float32, device="cuda")
 
-    def launch_step(b):
+    def launch_step(bi):
+        b = batches[bi]
         ctx.train_step(tables, b["idx"], b["off"], b["go"], scales, bits, out, ur, uo, gr, codes, gs, wl.lr,
                        B=wl.B, L=b["L"])
+
+    # Software pipeline over steps (default): the index half of the backward of batch k+1 (sort, unique rows)
+    # runs on a second stream while batch k trains; the two halves hand over through two workspaces and two
+    # (unique_rows, uniq_off) buffers used alternately.  Every step still does all of its own work inside the
+    # timed region: K timed steps hold K sorts and K training halves.
+    pipelined = not args.no_pipeline and not (args.dp_exchange and world > 1)
+    if pipelined:
+        assert N_BATCHES % 2 == 0
+        side = torch.cuda.Stream(priority=-1)
+        ctx._workspace(1)                                   # allocate the second workspace before any capture
+        urs = [ur, torch.empty_like(ur)]
+        uos = [uo, torch.empty_like(uo)]
+
+        def prime(bi):                                      # sorts batch bi ahead of its step (pipeline start)
+            b = batches[bi]
+            ctx.sort_batch(b["idx"], b["off"], urs[bi & 1], uos[bi & 1], B=wl.B, L=b["L"], ws=bi & 1)
+
+        def launch_step(bi):     # noqa: F811
+            b, nb, slot = batches[bi], batches[(bi + 1) % N_BATCHES], bi & 1
+            cur = torch.cuda.current_stream()
+            side.wait_stream(cur)
+            ctx.sort_batch(nb["idx"], nb["off"], urs[slot ^ 1], uos[slot ^ 1], B=wl.B, L=nb["L"], ws=slot ^ 1,
+                           stream=side)
+            ctx.train_step_sorted(tables, b["idx"], b["off"], b["go"], scales, bits, out, urs[slot], uos[slot], gr,
+                                  codes, gs, wl.lr, B=wl.B, L=b["L"], ws=slot, stream=cur)
+            cur.wait_stream(side)
+
+        def launch_unpipelined(bi):
+            b = batches[bi]
+            ctx.train_step(tables, b["idx"], b["off"], b["go"], scales, bits, out, ur, uo, gr, codes, gs, wl.lr,
+                           B=wl.B, L=b["L"])
 
     # The step is a fixed sequence of launches on fixed buffers, so each pre-staged batch's step is
     # captured once into a CUDA graph and replayed (the launches themselves are unchanged).
@@ -262,21 +294,24 @@ def run_ours(args):
         from paper_2410_20046_b200 import dp
         dp_step = dp.DataParallelStep(ctx, wl.B, Lmax, world)
 
-        def launch_step(b):      # noqa: F811  (the exchange has host-side size reads, so no graph capture)
+        def launch_step(bi):     # noqa: F811  (the exchange has host-side size reads, so no graph capture)
+            b = batches[bi]
             dp_step.step(tables, b["idx"], b["off"], b["go"], scales, bits, wl.lr, b["L"])
     graphs = None
     launches_per_step = 0
     if not args.no_graph and dp_step is None:
         try:
-            for b in batches[:2]:
-                launch_step(b)                       # first use outside capture (function attributes, caches)
+            if pipelined:
+                prime(0)
+            for bi in range(2):
+                launch_step(bi)                      # first use outside capture (function attributes, caches)
             torch.cuda.synchronize()
             graphs = []
-            for b in batches:
+            for bi in range(N_BATCHES):
                 g = torch.cuda.CUDAGraph()
                 n_before = ctx.launch_count()
                 with torch.cuda.graph(g):
-                    launch_step(b)
+                    launch_step(bi)
                 launches_per_step = ctx.launch_count() - n_before      # kernels recorded into the graph
                 graphs.append(g)
             torch.cuda.synchronize()
@@ -285,13 +320,22 @@ def run_ours(args):
             graphs = None
             torch.cuda.synchronize()
 
+    last = {"s": None}
+
     def step(s, direct=False):
         if s % wl.period == 0:
             ctx.scale_refresh(tables, bits, scales)
+        if direct and pipelined:                     # the per-kernel timing pass: one stream, one call per step
+            launch_unpipelined(s % N_BATCHES)
+            last["s"] = None
+            return
+        if pipelined and last["s"] != s - 1:
+            prime(s % N_BATCHES)                     # (re)start of the pipeline: this batch is not sorted yet
+        last["s"] = s
         if graphs is not None and not direct:
             graphs[s % N_BATCHES].replay()
         else:
-            launch_step(batches[s % N_BATCHES])
+            launch_step(s % N_BATCHES)
 
     def step_host(s):
         if s % wl.period == 0:
@@ -385,7 +429,10 @@ def run_ours(args):
             "config": {"workload": wl.name, "tables": wl.T, "dim": wl.D, "batch_per_gpu": wl.B,
                        "lookups_per_step_per_gpu": Lavg, "unique_rows_per_step": Uavg, "unique_fraction": Uavg / Lavg,
                        "bits": wl.bits, "grad_bits": 8, "refresh_period": wl.period, "table_bytes": wl.table_bytes(),
-                       "launch": "CUDA graph replay per step" if graphs is not None else "direct launches",
+                       "launch": ("CUDA graph replay per step" if graphs is not None else "direct launches") +
+                                 ("; the index sort of batch k+1 runs on a second stream while batch k trains "
+                                  "(two workspaces, every step does one sort and one training half)" if pipelined
+                                  else ""),
                        "parallelism": (f"{world} ranks, sparse INT8 gradient exchange every step" if dp_step is not None
                                        else f"{world} replica(s), batch sharded by sample, no exchange"),
                        "l2": f"{N_BATCHES} distinct pre-staged batches cycled; their rows, gradients and outputs "
@@ -417,6 +464,8 @@ def main():
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-pipeline", action="store_true",
+                    help="one dqrm_train_step call per step instead of sorting the next batch beside the current one")
     ap.add_argument("--workload", default="kaggle_b16384")
     ap.add_argument("--e2e-steps", type=int, default=50)
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -154,6 +154,25 @@ int dqrm_train_step(dqrm_ctx *ctx, float *tables, const int32_t *indices,
                     int8_t *codes, float *grad_scales, float lr, int B, int64_t L,
                     void *workspace, size_t workspace_bytes, void *stream);
 
+/* dqrm_train_step in two calls, for a training loop that knows the next batch's indices
+ * while the current batch trains (no counterpart in the paper; Section 4.3 only fixes what the
+ * sparse gradient holds).  dqrm_sort_batch does the part of the backward that needs the
+ * indices alone: it orders the lookups by row and writes unique_rows and uniq_off.
+ * dqrm_train_step_sorted then runs forward, gradient summation, INT8 quantisation and update
+ * for the same batch.  The sorted order travels in `workspace` (dqrm_workspace_bytes): pass
+ * the same workspace to both calls and to nothing in between; two workspaces used alternately
+ * let batch k+1 be sorted on one stream while batch k trains on another.  The caller orders
+ * the two calls (same stream, or an event).  Outputs equal those of dqrm_train_step. */
+int dqrm_sort_batch(dqrm_ctx *ctx, const int32_t *indices, const int32_t *offsets,
+                    int32_t *unique_rows, int32_t *uniq_off, int B, int64_t L,
+                    void *workspace, size_t workspace_bytes, void *stream);
+int dqrm_train_step_sorted(dqrm_ctx *ctx, float *tables, const int32_t *indices,
+                           const int32_t *offsets, const float *grad_out,
+                           const float *scales, const int32_t *bits, float *out,
+                           const int32_t *unique_rows, const int32_t *uniq_off, float *grad_rows,
+                           int8_t *codes, float *grad_scales, float lr, int B, int64_t L,
+                           void *workspace, size_t workspace_bytes, void *stream);
+
 /* Bytes of workspace dqrm_train_step_host needs (device staging for the host buffers,
  * the step's intermediate outputs and the scratch of dqrm_train_step). */
 size_t dqrm_host_step_workspace_bytes(const dqrm_ctx *ctx, int64_t max_lookups, int64_t max_bags);

@@ -36,6 +36,9 @@ SIGNATURES = {
     "dqrm_emb_bwd": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i64, _vp, _sz, _vp]),
     "dqrm_grad_quant_int8": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "dqrm_row_update": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _f, _vp]),
+    "dqrm_sort_batch": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i64, _vp, _sz, _vp]),
+    "dqrm_train_step_sorted": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _f, _i, _i64,
+                                    _vp, _sz, _vp]),
     "dqrm_train_step": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _f, _i, _i64,
                              _vp, _sz, _vp]),
     "dqrm_host_step_workspace_bytes": (_sz, [_vp, _i64, _i64]),
@@ -133,6 +136,12 @@ class Context:
         self.workspace_bytes = int(self.lib.dqrm_workspace_bytes(self._h, self.max_lookups, self.max_bags))
         self.workspace = torch.empty(self.workspace_bytes + 256, dtype=torch.uint8, device="cuda")
         self._ws_ptr = (self.workspace.data_ptr() + 255) // 256 * 256
+        # scratch of the calls that carry nothing from one call to the next (scale refresh, gradient
+        # quantiser): kept apart from the workspaces that hold a sorted batch between dqrm_sort_batch
+        # and dqrm_train_step_sorted
+        self.scratch_bytes = int(self.lib.dqrm_workspace_bytes(self._h, 0, 0))
+        self.scratch = torch.empty(self.scratch_bytes + 256, dtype=torch.uint8, device="cuda")
+        self._scratch_ptr = (self.scratch.data_ptr() + 255) // 256 * 256
         self.host_workspace = None
         if host_step:
             self.host_workspace_bytes = int(
@@ -249,7 +258,7 @@ class Context:
 
         self._check("dqrm_scale_refresh", self.lib.dqrm_scale_refresh(
             self._h, _ptr(tables, torch.float32), _ptr(bits, torch.int32), _ptr(scales, torch.float32),
-            _ptr(minmax, torch.float32), self._ws_ptr, self.workspace_bytes, _stream(stream)))
+            _ptr(minmax, torch.float32), self._scratch_ptr, self.scratch_bytes, _stream(stream)))
 
     def emb_fwd(self, tables, indices, offsets, scales, bits, out, codes_out=None, *, B, L, stream=None):
         import torch
@@ -272,7 +281,7 @@ class Context:
 
         self._check("dqrm_grad_quant_int8", self.lib.dqrm_grad_quant_int8(
             self._h, _ptr(grad_rows, torch.float32), _ptr(uniq_off, torch.int32), _ptr(codes, torch.int8),
-            _ptr(grad_scales, torch.float32), self._ws_ptr, self.workspace_bytes, _stream(stream)))
+            _ptr(grad_scales, torch.float32), self._scratch_ptr, self.scratch_bytes, _stream(stream)))
 
     def row_update(self, tables, unique_rows, uniq_off, codes, grad_scales, lr, stream=None):
         import torch
@@ -291,6 +300,35 @@ class Context:
             _ptr(out, torch.float32), _ptr(unique_rows, torch.int32), _ptr(uniq_off, torch.int32),
             _ptr(grad_rows, torch.float32), _ptr(codes, torch.int8), _ptr(grad_scales, torch.float32),
             float(lr), int(B), int(L), self._ws_ptr, self.workspace_bytes, _stream(stream)))
+
+    # ---- the step in two calls; `ws` picks one of two workspaces (the second is made on first use) ----
+    def _workspace(self, ws: int) -> int:
+        import torch
+
+        if ws == 0:
+            return self._ws_ptr
+        if getattr(self, "workspace2", None) is None:
+            self.workspace2 = torch.empty(self.workspace_bytes + 256, dtype=torch.uint8, device="cuda")
+            self._ws2_ptr = (self.workspace2.data_ptr() + 255) // 256 * 256
+        return self._ws2_ptr
+
+    def sort_batch(self, indices, offsets, unique_rows, uniq_off, *, B, L, ws=0, stream=None):
+        import torch
+
+        self._check("dqrm_sort_batch", self.lib.dqrm_sort_batch(
+            self._h, _ptr(indices, torch.int32), _ptr(offsets, torch.int32), _ptr(unique_rows, torch.int32),
+            _ptr(uniq_off, torch.int32), int(B), int(L), self._workspace(ws), self.workspace_bytes, _stream(stream)))
+
+    def train_step_sorted(self, tables, indices, offsets, grad_out, scales, bits, out, unique_rows, uniq_off,
+                          grad_rows, codes, grad_scales, lr, *, B, L, ws=0, stream=None):
+        import torch
+
+        self._check("dqrm_train_step_sorted", self.lib.dqrm_train_step_sorted(
+            self._h, _ptr(tables, torch.float32), _ptr(indices, torch.int32), _ptr(offsets, torch.int32),
+            _ptr(grad_out, torch.float32), _ptr(scales, torch.float32), _ptr(bits, torch.int32),
+            _ptr(out, torch.float32), _ptr(unique_rows, torch.int32), _ptr(uniq_off, torch.int32),
+            _ptr(grad_rows, torch.float32), _ptr(codes, torch.int8), _ptr(grad_scales, torch.float32),
+            float(lr), int(B), int(L), self._workspace(ws), self.workspace_bytes, _stream(stream)))
 
     def train_step_host(self, tables, h_indices, h_offsets, h_grad_out, scales, bits, h_out, lr, *, B, L,
                         stream=None):

@@ -334,6 +334,38 @@ int dqrm_dp_merge_update(dqrm_ctx *ctx, float *tables, int W, int64_t rank_strid
                                      workspace_bytes, as_stream(stream));
 }
 
+int dqrm_sort_batch(dqrm_ctx *ctx, const int32_t *indices, const int32_t *offsets, int32_t *unique_rows,
+                    int32_t *uniq_off, int B, int64_t L, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!batch_ok(ctx, B, L) || !offsets || !uniq_off) return DQRM_ERR_INVALID_ARG;
+    if (L > 0 && (!indices || !unique_rows)) return DQRM_ERR_INVALID_ARG;
+    if (!ws_ok(workspace, workspace_bytes, dq_bwd_ws_bytes(ctx, L, (int64_t)ctx->T * B))) return DQRM_ERR_WORKSPACE;
+    cudaStream_t st = as_stream(stream);
+    if (ctx->prof_on) dq_mark(ctx, st, DQ_K_BEGIN);
+    return dq_launch_bwd_sort(ctx, indices, offsets, unique_rows, uniq_off, B, L, workspace, workspace_bytes, st, nullptr);
+}
+
+int dqrm_train_step_sorted(dqrm_ctx *ctx, float *tables, const int32_t *indices, const int32_t *offsets,
+                           const float *grad_out, const float *scales, const int32_t *bits, float *out,
+                           const int32_t *unique_rows, const int32_t *uniq_off, float *grad_rows, int8_t *codes,
+                           float *grad_scales, float lr, int B, int64_t L, void *workspace, size_t workspace_bytes,
+                           void *stream)
+{
+    if (!batch_ok(ctx, B, L) || !tables || !offsets || !grad_out || !scales || !bits || !out || !uniq_off ||
+        !grad_scales)
+        return DQRM_ERR_INVALID_ARG;
+    if (L > 0 && (!indices || !unique_rows || !grad_rows || !codes)) return DQRM_ERR_INVALID_ARG;
+    if (!ws_ok(workspace, workspace_bytes, dq_bwd_ws_bytes(ctx, L, (int64_t)ctx->T * B))) return DQRM_ERR_WORKSPACE;
+    cudaStream_t st = as_stream(stream);
+    if (ctx->prof_on) dq_mark(ctx, st, DQ_K_BEGIN);
+    int rc = dq_launch_fwd(ctx, tables, indices, offsets, scales, bits, out, nullptr, B, L, st);
+    if (rc != DQRM_OK) return rc;
+    rc = dq_launch_bwd_reduce(ctx, grad_out, uniq_off, grad_rows, B, L, workspace, workspace_bytes, st);
+    if (rc != DQRM_OK) return rc;
+    return dq_launch_quant_update(ctx, tables, unique_rows, uniq_off, grad_rows,
+                                  dq_bwd_absmax_bits(ctx, L, workspace), codes, grad_scales, lr, st);
+}
+
 size_t dqrm_packed_bytes(const dqrm_ctx *ctx, int bits)
 {
     if (!ctx || (bits != 2 && bits != 4 && bits != 8)) return 0;

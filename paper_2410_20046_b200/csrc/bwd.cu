@@ -392,6 +392,11 @@ void dq_bwd_ws_views(const dqrm_ctx *ctx, int64_t L, char *ws, const u32 **sorte
     *seg_start = reinterpret_cast<const u32 *>(ws + y.seg_start);
 }
 
+const u32 *dq_bwd_absmax_bits(const dqrm_ctx *ctx, int64_t L, const void *ws)
+{
+    return reinterpret_cast<const u32 *>(reinterpret_cast<const char *>(ws) + make_layout(ctx, L).absmax);
+}
+
 size_t dq_bwd_ws_bytes(const dqrm_ctx *ctx, int64_t L, int64_t G)
 {
     (void)G;

@@ -184,6 +184,9 @@ int dq_launch_fwd(dqrm_ctx *ctx, const float *tables, const int32_t *indices, co
                   int B, int64_t L, cudaStream_t st);
 
 size_t dq_bwd_ws_bytes(const dqrm_ctx *ctx, int64_t L, int64_t G);
+// per-table |grad| maxima (float bit patterns) inside a workspace that dq_launch_bwd_sort and
+// dq_launch_bwd_reduce have filled
+const u32 *dq_bwd_absmax_bits(const dqrm_ctx *ctx, int64_t L, const void *ws);
 // absmax_bits_out: device pointer (inside ws) to per-table |grad| maxima as float bit patterns
 int dq_launch_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, const int32_t *offsets,
                   int32_t *unique_rows, int32_t *uniq_off, float *grad_rows, int B, int64_t L,

@@ -1,0 +1,117 @@
+"""GPU parity of the training step split in two calls (dqrm_sort_batch on one stream for batch
+k+1 while dqrm_train_step_sorted trains batch k on another, two workspaces used alternately):
+the trajectory must equal the oracle's, and the single-call step's, bit for bit."""
+import numpy as np
+import pytest
+
+from dqrm_inputs import workloads as W
+from gpu_util import Case, assert_close_fp32, bit_equal
+
+pytestmark = pytest.mark.gpu
+
+
+def _cases():
+    return {
+        "tiny": W.tiny(),
+        "kaggle_small": W.scaled_down(W.kaggle(), total_rows=300_000, B=2048, name="kaggle_small"),
+        "multihot_small": W.scaled_down(W.multihot(), total_rows=26 * 3000, B=300, name="multihot_small"),
+    }
+
+
+@pytest.mark.parametrize("name", sorted(_cases()))
+def test_pipelined_steps_equal_oracle(oracle, name):
+    import torch
+
+    wl = _cases()[name]
+    steps = 12
+    c = Case(wl)
+    o_tables = W.tables_np(wl)
+    d_tables = c.dev(o_tables)
+    Lmax = c.max_lookups
+    out = c.empty((wl.B, wl.T, wl.D), torch.float32)
+    gr = c.empty((Lmax, wl.D), torch.float32)
+    codes = c.empty((Lmax, wl.D), torch.int8)
+    gs = c.empty(wl.T, torch.float32)
+    scales = c.empty(wl.T, torch.float32)
+    # per in-flight batch: its device inputs and the sort's outputs
+    slots = [dict(ur=c.empty(Lmax, torch.int32), uo=c.empty(wl.T + 1, torch.int32)) for _ in range(2)]
+    main, side = torch.cuda.Stream(), torch.cuda.Stream()
+    sorted_ev = [torch.cuda.Event(), torch.cuda.Event()]
+    trained_ev = [torch.cuda.Event(), torch.cuda.Event()]
+
+    def stage(step):
+        s = slots[step & 1]
+        idx, off, go = c.batch(step)
+        s.update(idx_h=idx, off_h=off, go_h=go, idx=c.dev(idx), off=c.dev(off), go=c.dev(go), L=len(idx))
+        torch.cuda.current_stream().synchronize()
+        with torch.cuda.stream(side):
+            side.wait_event(trained_ev[step & 1])          # the workspace's previous batch is done
+            c.ctx.sort_batch(s["idx"], s["off"], s["ur"], s["uo"], B=wl.B, L=s["L"], ws=step & 1, stream=side)
+            sorted_ev[step & 1].record(side)
+
+    trained_ev[0].record(main)
+    trained_ev[1].record(main)
+    c.ctx.scale_refresh(d_tables, c.bits, scales)
+    torch.cuda.synchronize()
+    o_scales, _ = oracle.scale_refresh(o_tables, c.row_off, wl.D, c.bits_np)
+    stage(0)
+    for step in range(steps):
+        if step + 1 < steps:
+            stage(step + 1)                                 # sorts batch k+1 while batch k trains
+        s = slots[step & 1]
+        if step and step % 4 == 0:
+            # a scale refresh between the two halves of a step must leave the sorted batch alone
+            with torch.cuda.stream(main):
+                c.ctx.scale_refresh(d_tables, c.bits, scales, stream=main)
+            o_scales, _ = oracle.scale_refresh(o_tables, c.row_off, wl.D, c.bits_np)
+        with torch.cuda.stream(main):
+            main.wait_event(sorted_ev[step & 1])
+            c.ctx.train_step_sorted(d_tables, s["idx"], s["off"], s["go"], scales, c.bits, out, s["ur"], s["uo"], gr,
+                                    codes, gs, wl.lr, B=wl.B, L=s["L"], ws=step & 1, stream=main)
+            trained_ev[step & 1].record(main)
+        main.synchronize()
+        r = oracle.train_step(o_tables, c.row_off, wl.D, wl.B, s["idx_h"], s["off_h"], s["go_h"], o_scales, c.bits_np,
+                              wl.lr)
+        U = int(r["uniq_off"][-1])
+        assert bit_equal(s["uo"].cpu().numpy(), r["uniq_off"]), f"step {step}"
+        assert bit_equal(s["ur"].cpu().numpy()[:U], r["unique_rows"]), f"step {step}"
+        assert_close_fp32(out.cpu().numpy(), r["out"], f"step {step}: pooled output")
+        assert_close_fp32(gr.cpu().numpy()[:U], r["grad_rows"], f"step {step}: summed gradients")
+        assert bit_equal(gs.cpu().numpy(), r["grad_scales"]), f"step {step}: gradient scales"
+        assert bit_equal(codes.cpu().numpy()[:U], r["codes"]), f"step {step}: gradient codes"
+    torch.cuda.synchronize()
+    c.ctx.raise_on_device_error()
+    assert bit_equal(d_tables.cpu().numpy(), o_tables)
+    c.ctx.close()
+
+
+def test_two_calls_equal_one_call():
+    import torch
+
+    wl = W.scaled_down(W.terabyte(), total_rows=400_000, B=1500, name="terabyte_small")
+    c = Case(wl)
+    tables = W.tables_np(wl)
+    idx, off, go = c.batch(0)
+    L = len(idx)
+    res = []
+    for split in (False, True):
+        d_tables = c.dev(tables)
+        scales = c.empty(wl.T, torch.float32)
+        c.ctx.scale_refresh(d_tables, c.bits, scales)
+        out = c.empty((wl.B, wl.T, wl.D), torch.float32)
+        ur = torch.full((L,), -1, dtype=torch.int32, device="cuda")
+        uo = c.empty(wl.T + 1, torch.int32)
+        gr = torch.zeros((L, wl.D), dtype=torch.float32, device="cuda")
+        codes = torch.zeros((L, wl.D), dtype=torch.int8, device="cuda")
+        gs = c.empty(wl.T, torch.float32)
+        args = (d_tables, c.dev(idx), c.dev(off), c.dev(go), scales, c.bits, out, ur, uo, gr, codes, gs, wl.lr)
+        if split:
+            c.ctx.sort_batch(args[1], args[2], ur, uo, B=wl.B, L=L, ws=1)
+            c.ctx.train_step_sorted(*args, B=wl.B, L=L, ws=1)
+        else:
+            c.ctx.train_step(*args, B=wl.B, L=L)
+        c.ctx.raise_on_device_error()
+        res.append([x.cpu().numpy() for x in (d_tables, out, ur, uo, gr, codes, gs)])
+    for a, b in zip(*res):
+        assert bit_equal(a, b)
+    c.ctx.close()
