@@ -5,8 +5,9 @@
 //
 // Three variants of one row-streaming kernel share the addressing: quantise only,
 // update only (from stored codes), and quantise + update fused (the training step).
-// A group of LPR lanes owns one unique row; rows are distinct, so the read-modify-write
-// of the master rows needs no atomics.  All streams are 128-bit per lane.
+// A group of LPR lanes owns a contiguous range of unique rows and keeps a few of them in flight;
+// rows are distinct, so the read-modify-write of the master rows needs no atomics.  All
+// streams are 128-bit per lane.
 #include "common.cuh"
 
 namespace {
@@ -67,6 +68,9 @@ absmax_kernel(const float *__restrict__ grad_rows, const int32_t *__restrict__ u
         if (s_max[t]) atomicMax(&absmax[t], s_max[t]);
 }
 
+// rows in flight per lane group: fewer when a lane already holds several vectors of every row
+template <int CH> struct RowsInFlight { static constexpr int v = CH >= 4 ? 1 : (CH == 2 ? 2 : 4); };
+
 template <int MODE, int LPR, int CH>
 __global__ void __launch_bounds__(QU_THREADS)
 row_stream_kernel(float *__restrict__ tables, const int64_t *__restrict__ row_off,
@@ -74,71 +78,94 @@ row_stream_kernel(float *__restrict__ tables, const int64_t *__restrict__ row_of
                   const float *__restrict__ grad_rows, const u32 *__restrict__ absmax,
                   int8_t *__restrict__ codes, float *__restrict__ grad_scales, float lr, int T, int D)
 {
+    constexpr int NB = RowsInFlight<CH>::v;
     extern __shared__ unsigned char smem_raw[];
     int32_t *s_uoff = reinterpret_cast<int32_t *>(smem_raw);      // [T+1]
+    float *s_scale = reinterpret_cast<float *>(s_uoff + (T + 1)); // [T] gradient scale of every table
     for (int t = threadIdx.x; t <= T; t += QU_THREADS) s_uoff[t] = uniq_off[t];
-    __syncthreads();
-    if (MODE != MODE_UPDATE && blockIdx.x == 0) {
-        for (int t = threadIdx.x; t < T; t += QU_THREADS)
-            grad_scales[t] = dq_scale_from_absmax(__uint_as_float(absmax[t]), 8);
+    for (int t = threadIdx.x; t < T; t += QU_THREADS) {
+        const float sc = (MODE == MODE_UPDATE) ? grad_scales[t] : dq_scale_from_absmax(__uint_as_float(absmax[t]), 8);
+        s_scale[t] = sc;
+        if (MODE != MODE_UPDATE && blockIdx.x == 0) grad_scales[t] = sc;
     }
+    __syncthreads();
     const int d4 = D >> 2;
     const int64_t U = s_uoff[T];
     const int lane = threadIdx.x % LPR;
     const int64_t group = ((int64_t)blockIdx.x * QU_THREADS + threadIdx.x) / LPR;
     const int64_t n_groups = (int64_t)gridDim.x * QU_THREADS / LPR;
+    // a lane group owns a contiguous range of unique rows: its rows mostly share a table, and its reads
+    // of the gradient rows and writes of the codes are sequential
+    int64_t per = (U + n_groups - 1) / n_groups;
+    if (per < NB) per = NB;             // few rows: fewer groups, each with a full set of rows in flight
+    const int64_t u_begin = group * per, u_end = min(U, u_begin + per);
     int cur_t = -1;
     int64_t cur_end = -1, r0 = 0;
     float s = 1.f;
     QuantScale qs = dq_make_scale(1.f, 8);
-    for (int64_t u = group; u < U; u += n_groups) {
+    for (int64_t u = u_begin; u < u_end;) {
         if (u >= cur_end) {
             cur_t = table_of_row(s_uoff, T, u);
             cur_end = s_uoff[cur_t + 1];
             if (MODE != MODE_QUANT) r0 = __ldg(row_off + cur_t);
-            s = (MODE == MODE_UPDATE) ? __ldg(grad_scales + cur_t)
-                                      : dq_scale_from_absmax(__uint_as_float(__ldg(absmax + cur_t)), 8);
+            s = s_scale[cur_t];
             qs = dq_make_scale(s, 8);
         }
-        float4 *wrow = nullptr;
-        if (MODE != MODE_QUANT) wrow = reinterpret_cast<float4 *>(tables + (r0 + __ldg(unique_rows + u)) * D);
-        float q[CH][4];            // integer codes held as floats
-        float4 w[CH];
+        // up to NB rows of the current table at once
+        const int nb = (int)min((int64_t)NB, min(u_end, cur_end) - u);
+        float4 *wrow[NB];
+        float4 g[NB][CH], w[NB][CH];
+        char4 cin[NB][CH];
 #pragma unroll
-        for (int ch = 0; ch < CH; ++ch) {
-            int c4 = ch * LPR + lane;
-            if (c4 < d4) {
-                if (MODE == MODE_UPDATE) {
-                    char4 c = *reinterpret_cast<const char4 *>(codes + u * D + 4 * c4);
-                    q[ch][0] = c.x; q[ch][1] = c.y; q[ch][2] = c.z; q[ch][3] = c.w;
-                } else {
-                    float4 g = __ldg(reinterpret_cast<const float4 *>(grad_rows + u * D) + c4);
-                    float4 cd, dq_unused;
-                    dq_fq4(g, qs, cd, dq_unused);
-                    q[ch][0] = cd.x; q[ch][1] = cd.y; q[ch][2] = cd.z; q[ch][3] = cd.w;
+        for (int b = 0; b < NB; ++b) {
+            wrow[b] = nullptr;
+            if (b < nb && MODE != MODE_QUANT)
+                wrow[b] = reinterpret_cast<float4 *>(tables + (r0 + __ldg(unique_rows + u + b)) * D);
+        }
+#pragma unroll
+        for (int b = 0; b < NB; ++b) {
+            if (b < nb) {
+#pragma unroll
+                for (int ch = 0; ch < CH; ++ch) {
+                    const int c4 = ch * LPR + lane;
+                    if (c4 < d4) {
+                        if (MODE == MODE_UPDATE) cin[b][ch] = *reinterpret_cast<const char4 *>(codes + (u + b) * D + 4 * c4);
+                        else g[b][ch] = __ldg(reinterpret_cast<const float4 *>(grad_rows + (u + b) * D) + c4);
+                        if (MODE != MODE_QUANT) w[b][ch] = wrow[b][c4];
+                    }
                 }
-                if (MODE != MODE_QUANT) w[ch] = wrow[c4];
             }
         }
 #pragma unroll
-        for (int ch = 0; ch < CH; ++ch) {
-            int c4 = ch * LPR + lane;
-            if (c4 < d4) {
-                if (MODE != MODE_UPDATE) {
-                    char4 c = make_char4((signed char)(int)q[ch][0], (signed char)(int)q[ch][1],
-                                         (signed char)(int)q[ch][2], (signed char)(int)q[ch][3]);
-                    *reinterpret_cast<char4 *>(codes + u * D + 4 * c4) = c;
-                }
-                if (MODE != MODE_QUANT) {
-                    float4 x = w[ch];
-                    x.x = __fsub_rn(x.x, __fmul_rn(lr, __fmul_rn(q[ch][0], s)));
-                    x.y = __fsub_rn(x.y, __fmul_rn(lr, __fmul_rn(q[ch][1], s)));
-                    x.z = __fsub_rn(x.z, __fmul_rn(lr, __fmul_rn(q[ch][2], s)));
-                    x.w = __fsub_rn(x.w, __fmul_rn(lr, __fmul_rn(q[ch][3], s)));
-                    wrow[c4] = x;
+        for (int b = 0; b < NB; ++b) {
+            if (b < nb) {
+#pragma unroll
+                for (int ch = 0; ch < CH; ++ch) {
+                    const int c4 = ch * LPR + lane;
+                    if (c4 < d4) {
+                        float4 q;                      // integer codes held as floats
+                        if (MODE == MODE_UPDATE) {
+                            q = make_float4((float)cin[b][ch].x, (float)cin[b][ch].y, (float)cin[b][ch].z, (float)cin[b][ch].w);
+                        } else {
+                            float4 dq_unused;
+                            dq_fq4(g[b][ch], qs, q, dq_unused);
+                            *reinterpret_cast<char4 *>(codes + (u + b) * D + 4 * c4) =
+                                make_char4((signed char)(int)q.x, (signed char)(int)q.y, (signed char)(int)q.z,
+                                           (signed char)(int)q.w);
+                        }
+                        if (MODE != MODE_QUANT) {
+                            float4 x = w[b][ch];
+                            x.x = __fsub_rn(x.x, __fmul_rn(lr, __fmul_rn(q.x, s)));
+                            x.y = __fsub_rn(x.y, __fmul_rn(lr, __fmul_rn(q.y, s)));
+                            x.z = __fsub_rn(x.z, __fmul_rn(lr, __fmul_rn(q.z, s)));
+                            x.w = __fsub_rn(x.w, __fmul_rn(lr, __fmul_rn(q.w, s)));
+                            wrow[b][c4] = x;
+                        }
+                    }
                 }
             }
         }
+        u += nb;
     }
 }
 
@@ -147,8 +174,8 @@ int launch_rows(dqrm_ctx *ctx, float *tables, const int32_t *unique_rows, const 
                 const float *grad_rows, const u32 *absmax, int8_t *codes, float *grad_scales, float lr,
                 cudaStream_t st)
 {
-    const size_t smem = (size_t)(ctx->T + 1) * sizeof(int32_t);
-    int grid = ctx->num_sms * 8;      // U lives on the device: persistent grid-stride
+    const size_t smem = (size_t)(ctx->T + 1) * sizeof(int32_t) + (size_t)ctx->T * sizeof(float);
+    int grid = ctx->num_sms * 8;      // U lives on the device: a fixed grid splits the rows evenly
     row_stream_kernel<MODE, LPR, CH><<<grid, QU_THREADS, smem, st>>>(tables, ctx->d_row_off, unique_rows, uniq_off,
                                                                      grad_rows, absmax, codes, grad_scales, lr,
                                                                      ctx->T, ctx->D);
