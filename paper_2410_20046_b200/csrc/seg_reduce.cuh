@@ -138,29 +138,48 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
     for (int64_t c = group; c < num_chunks; c += n_groups) {
         const int64_t i0 = c * CHUNK;
         const int n = (int)(min(i0 + (int64_t)CHUNK, L) - i0);
-        // heads: entry e starts a segment when its key differs from the key before it
+        // heads: entry e starts a segment when its key differs from the key before it.  All loads are
+        // issued before the first vote so that they are in flight together.
         u32 heads = 0;
+        u32 kc[EPL], kp[EPL], vv[EPL];
+#pragma unroll
+        for (int j = 0; j < EPL; ++j) {
+            const int e = j * LPR + lane;
+            const int64_t i = i0 + e;
+            kc[j] = kp[j] = vv[j] = 0u;
+            if (e < n) {
+                vv[j] = vals[i];
+                kc[j] = keys[i];
+                kp[j] = i > 0 ? keys[i - 1] : ~kc[j];
+            }
+        }
+        const u32 k_after = (i0 + n == L) ? 0u : keys[i0 + n];
+        const u32 u_first = chunk_first[c];
         __syncwarp(gmask);                        // the previous chunk's payloads are no longer read
 #pragma unroll
         for (int j = 0; j < EPL; ++j) {
             const int e = j * LPR + lane;
-            bool head = false;
             if (e < n) {
-                const int64_t i = i0 + e;
-                u32 v = vals[i];
+                u32 v = vv[j];
                 if ((int64_t)v >= G) { bad = true; v = 0u; }
                 s_vals[e] = v;
-                head = (i == 0) || (keys[i] != keys[i - 1]);
             }
+            const bool head = (e < n) && (kc[j] != kp[j]);
             const u32 bits = (__ballot_sync(gmask, head) >> gbase) & (LPR >= 32 ? 0xffffffffu : ((1u << LPR) - 1u));
             heads |= bits << (j * LPR);
         }
+        // the chunk's last key sits in lane (n-1) % LPR, register (n-1) / LPR
+        u32 k_last = 0u;
+#pragma unroll
+        for (int j = 0; j < EPL; ++j)
+            if ((n - 1) / LPR == j) k_last = kc[j];
+        k_last = __shfl_sync(gmask, k_last, gbase + (n - 1) % LPR);
         __syncwarp(gmask);
         // does the chunk's first run begin here, does its last run end here?
         const bool first_begins = heads & 1u;
-        const bool last_ends = (i0 + n == L) || (keys[i0 + n] != keys[i0 + n - 1]);
+        const bool last_ends = (i0 + n == L) || (k_after != k_last);
         heads &= ~1u;                             // the walk starts a run at entry 0 either way
-        u32 u = chunk_first[c];
+        u32 u = u_first;
         int run_start = 0;
         double acc[CH][VEC];
 #pragma unroll
