@@ -182,67 +182,78 @@ packed_fwd_kernel(const PfArgs a)
     if (bad) dq_report(a.status, DQRM_ERR_INDEX_RANGE);
 }
 
-// One index per bag (L == T*B, the Criteo shape): a lane group keeps NB rows of NB different bags
-// in flight; the pooled value of a one-index bag is code * scale itself.  A bag that turns out
-// not to hold exactly one index goes through pool_bag.
+// One index per bag (L == T*B, the Criteo shape): a warp takes 32 consecutive bags, one lane per
+// bag does the bag's bookkeeping once, then the rows are fetched 32/LPR per step (the bag's index
+// broadcast by shuffle), NB steps in flight; the pooled value of a one-index bag is code * scale
+// itself.  A bag that turns out not to hold exactly one index goes through pool_bag.
 template <int BITS, int EPL, int LPR, int CH>
 __global__ void __launch_bounds__(PK_THREADS)
 packed_fwd_onehot_kernel(const PfArgs a)
 {
     constexpr int NB = CH >= 2 ? 1 : 4;
-    constexpr int GPB = PK_THREADS / LPR;
+    constexpr int RPW = 32 / LPR;
+    constexpr int WPB = PK_THREADS / 32;
     const int units = a.D / EPL;
     const int t = blockIdx.y;
-    const int lane = threadIdx.x % LPR, grp = threadIdx.x / LPR;
+    const int wlane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = wlane % LPR, grp = wlane / LPR;
     const float s = __ldg(a.scales + t);
     const int64_t r0 = __ldg(a.row_off + t);
     const int32_t nrows = (int32_t)(__ldg(a.row_off + t + 1) - r0);
     const int64_t g0 = (int64_t)t * a.B;
+    const int TD4 = a.T * (a.D >> 2);            // 128-bit vectors between the output rows of bags i and i+1
     bool bad = false;
-    for (int ib = blockIdx.x * (GPB * NB); ib < a.B; ib += gridDim.x * (GPB * NB)) {
-        int32_t idx[NB];
-        unsigned one = 0, rare = 0;
-#pragma unroll
-        for (int b = 0; b < NB; ++b) {
-            const int i = ib + b * GPB + grp;
-            idx[b] = 0;
-            if (i < a.B) {
-                const int32_t lo = __ldg(a.offsets + g0 + i), hi = __ldg(a.offsets + g0 + i + 1);
-                if (hi - lo == 1 && lo >= 0 && (int64_t)hi <= a.L) {
-                    one |= 1u << b;
-                    idx[b] = __ldg(a.indices + lo);
-                    bad |= (idx[b] < 0) | (idx[b] >= nrows);
-                    idx[b] = min(max(idx[b], 0), nrows - 1);
-                } else rare |= 1u << b;
+    for (int i0 = (blockIdx.x * WPB + warp) * 32; i0 < a.B; i0 += gridDim.x * (WPB * 32)) {
+        const int i = i0 + wlane;
+        int32_t idx = 0;
+        bool single = false;
+        if (i < a.B) {
+            const int32_t lo = __ldg(a.offsets + g0 + i), hi = __ldg(a.offsets + g0 + i + 1);
+            idx = __ldg(a.indices + g0 + i);            // right when the offsets are the identity (L == T*B)
+            single = (hi - lo == 1) & (lo >= 0) & ((int64_t)hi <= a.L);
+            if (single) {
+                if ((int64_t)lo != g0 + i) idx = __ldg(a.indices + lo);
+                bad |= (idx < 0) | (idx >= nrows);
+                idx = min(max(idx, 0), nrows - 1);
             }
         }
-#pragma unroll
-        for (int c = 0; c < CH; ++c) {
-            const int u = c * LPR + lane;
-            Unit<BITS, EPL> v[NB];
-#pragma unroll
-            for (int b = 0; b < NB; ++b)
-                if (((one >> b) & 1u) && u < units) v[b].load(a.packed, (r0 + idx[b]) * units + u);
-#pragma unroll
-            for (int b = 0; b < NB; ++b) {
-                if (((one >> b) & 1u) && u < units) {
-                    const int i = ib + b * GPB + grp;
-                    float4 *o = reinterpret_cast<float4 *>(a.out + ((int64_t)i * a.T + t) * a.D) + u * (EPL / 4);
-                    __stcs(o, scale4(v[b].template quad<0>(), s));
-                    if constexpr (EPL == 8) __stcs(o + 1, scale4(v[b].template quad<1>(), s));
-                }
-            }
-        }
-        if (rare) {
+        const unsigned one = __ballot_sync(0xffffffffu, single);
+        unsigned rare = __ballot_sync(0xffffffffu, (i < a.B) && !single);
+        float4 *out_lane = reinterpret_cast<float4 *>(a.out) + ((int64_t)i0 * a.T + t) * (a.D >> 2) + lane * (EPL / 4);
 #pragma unroll 1
-            for (int b = 0; b < NB; ++b) {
-                if ((rare >> b) & 1u) {
-                    const int i = ib + b * GPB + grp;
-                    pool_bag<BITS, EPL, LPR, CH>(a, r0, nrows, s, units, __ldg(a.offsets + g0 + i),
-                                                 __ldg(a.offsets + g0 + i + 1), a.out + ((int64_t)i * a.T + t) * a.D,
-                                                 lane, bad);
+        for (int k0 = 0; k0 < 32; k0 += RPW * NB) {
+            if ((one >> k0) == 0u) break;
+            int32_t ib[NB];
+#pragma unroll
+            for (int b = 0; b < NB; ++b) ib[b] = __shfl_sync(0xffffffffu, idx, (k0 + b * RPW + grp) & 31);
+#pragma unroll
+            for (int c = 0; c < CH; ++c) {
+                const int u = c * LPR + lane;
+                Unit<BITS, EPL> v[NB];
+#pragma unroll
+                for (int b = 0; b < NB; ++b) {
+                    const int bag = k0 + b * RPW + grp;
+                    if (bag < 32 && ((one >> bag) & 1u) && u < units) v[b].load(a.packed, (r0 + ib[b]) * units + u);
+                }
+#pragma unroll
+                for (int b = 0; b < NB; ++b) {
+                    const int bag = k0 + b * RPW + grp;
+                    if (bag < 32 && ((one >> bag) & 1u) && u < units) {
+                        float4 *o = out_lane + (int64_t)bag * TD4 + c * LPR * (EPL / 4);
+                        o[0] = scale4(v[b].template quad<0>(), s);
+                        if constexpr (EPL == 8) o[1] = scale4(v[b].template quad<1>(), s);
+                    }
                 }
             }
+        }
+        while (rare) {
+            const int bag = __ffs(rare) - 1;
+            rare &= rare - 1;
+            const int ii = i0 + bag;
+            if (grp == 0)
+                pool_bag<BITS, EPL, LPR, CH>(a, r0, nrows, s, units, __ldg(a.offsets + g0 + ii),
+                                             __ldg(a.offsets + g0 + ii + 1), a.out + ((int64_t)ii * a.T + t) * a.D, lane,
+                                             bad);
         }
     }
     if (bad) dq_report(a.status, DQRM_ERR_INDEX_RANGE);
@@ -265,7 +276,7 @@ int launch_pfwd(dqrm_ctx *ctx, const PfArgs &a, cudaStream_t st)
 {
     constexpr int GPB = PK_THREADS / LPR;
     const bool onehot = a.L == (int64_t)a.T * a.B;
-    const int per_block = onehot ? GPB * (CH >= 2 ? 1 : 4) : GPB;
+    const int per_block = onehot ? PK_THREADS : GPB;
     int bx = (a.B + per_block - 1) / per_block;
     const int cap = (ctx->num_sms * 32 + ctx->T - 1) / ctx->T;
     if (bx > cap) bx = cap;
