@@ -1,5 +1,6 @@
-"""Parity at the full sizes of the benchmark configurations, through the timed entry point
-(dqrm_train_step) in the launch configuration bench.py uses.
+"""Parity at the full sizes of the benchmark configurations, through the timed entry points
+(dqrm_train_step, and the two-call form dqrm_sort_batch + dqrm_train_step_sorted with the next
+batch being sorted on a second stream meanwhile) in the launch configuration bench.py uses.
 
 The tables (2.2 GB / 12.5 GB) are generated on the device by the shared counter-based
 generator.  The oracle cannot hold them, but it does not need to: every row a batch
@@ -36,11 +37,13 @@ def _workload(name):
 
 @pytest.mark.parametrize("name", ["kaggle_b16384", "terabyte_b32768", "multihot_b16384", "kaggle_b128",
                                   "terabyte_b2048", "sweep_d16_b2_uniform", "sweep_d32_b4_zipf",
-                                  "sweep_d64_b8_zipf", "sweep_d128_b8_uniform"])
+                                  "sweep_d64_b8_zipf", "sweep_d128_b8_uniform",
+                                  "kaggle_b16384+two_calls", "terabyte_b32768+two_calls", "multihot_b16384+two_calls"])
 def test_full_size_step_matches_oracle(name, oracle):
     import torch
     import paper_2410_20046_b200 as dq
 
+    name, _, form = name.partition("+")
     wl = _workload(name)
     off_rows = wl.row_off()
     tables = W.tables_torch(wl, "cuda")
@@ -78,8 +81,24 @@ def test_full_size_step_matches_oracle(name, oracle):
     gr = torch.empty((L, wl.D), dtype=torch.float32, device="cuda")
     codes = torch.empty((L, wl.D), dtype=torch.int8, device="cuda")
     gs = torch.empty(wl.T, dtype=torch.float32, device="cuda")
-    ctx.train_step(tables, torch.from_numpy(idx).cuda(), torch.from_numpy(off).cuda(), torch.from_numpy(go).cuda(),
-                   scales, bits, out, ur, uo, gr, codes, gs, wl.lr, B=wl.B, L=L)
+    d_idx, d_off, d_go = torch.from_numpy(idx).cuda(), torch.from_numpy(off).cuda(), torch.from_numpy(go).cuda()
+    if form == "two_calls":
+        # what a pipelined loop does: this batch was sorted ahead into one workspace; while it trains, the
+        # next batch is sorted on a second stream into the other workspace
+        nidx, noff = W.make_batch(wl, 1, samplers)
+        d_nidx, d_noff = torch.from_numpy(nidx).cuda(), torch.from_numpy(noff).cuda()
+        ur2, uo2 = torch.empty(len(nidx), dtype=torch.int32, device="cuda"), torch.empty_like(uo)
+        ctx2 = ctx if len(nidx) <= L else None
+        ctx.sort_batch(d_idx, d_off, ur, uo, B=wl.B, L=L, ws=1)
+        cur, side = torch.cuda.current_stream(), torch.cuda.Stream(priority=-1)
+        side.wait_stream(cur)
+        if ctx2 is not None:
+            ctx.sort_batch(d_nidx, d_noff, ur2, uo2, B=wl.B, L=len(nidx), ws=0, stream=side)
+        ctx.train_step_sorted(tables, d_idx, d_off, d_go, scales, bits, out, ur, uo, gr, codes, gs, wl.lr, B=wl.B,
+                              L=L, ws=1)
+        cur.wait_stream(side)
+    else:
+        ctx.train_step(tables, d_idx, d_off, d_go, scales, bits, out, ur, uo, gr, codes, gs, wl.lr, B=wl.B, L=L)
     ctx.raise_on_device_error()
 
     # the oracle on the compact problem: only the touched rows, regenerated on the host
