@@ -8,6 +8,9 @@ Prints ONE JSON line.  `value` is whole-job lookups/s with inputs resident in HB
 `e2e` the same through the host-buffer entry point (copies inside the timed region),
 `roofline` the dominant kernel against the measured HBM copy rate, `cpu_baseline` the
 CPU oracle timed on the host cores.  With --impl reference the oracle itself is timed.
+By default consecutive steps are software-pipelined: the index sort of batch k+1 runs on a
+second stream while batch k trains (--no-pipeline: one call per step).  --packed times the
+bit-packed export and the packed inference lookup instead of the training step.
 """
 from __future__ import annotations
 
