@@ -360,9 +360,14 @@ int launch_reduce(dqrm_ctx *ctx, const Layout &y, char *ws, const u32 *keys, con
     double *partials = reinterpret_cast<double *>(ws + y.partials);
     u32 *long_list = reinterpret_cast<u32 *>(ws + y.long_list);
     const size_t red_smem = (size_t)(ctx->T + 1) * sizeof(u32) + (size_t)gpb * SEG_CHUNK * sizeof(u32);
-    seg_reduce_kernel<RL, RV, RC><<<grid, 256, red_smem, st>>>(
-        keys, vals, seg_start, reinterpret_cast<const u32 *>(ws + y.chunk_first), uniq_off, grad_out, grad_rows,
-        partials, long_list, counters, absmax, ctx->T, ctx->D, L, G, y.num_chunks, ctx->d_status);
+    if (ctx->D == RL * RV * RC)
+        seg_reduce_kernel<RL, RV, RC, true><<<grid, 256, red_smem, st>>>(
+            keys, vals, seg_start, reinterpret_cast<const u32 *>(ws + y.chunk_first), uniq_off, grad_out, grad_rows,
+            partials, long_list, counters, absmax, ctx->T, ctx->D, L, G, y.num_chunks, ctx->d_status);
+    else
+        seg_reduce_kernel<RL, RV, RC, false><<<grid, 256, red_smem, st>>>(
+            keys, vals, seg_start, reinterpret_cast<const u32 *>(ws + y.chunk_first), uniq_off, grad_out, grad_rows,
+            partials, long_list, counters, absmax, ctx->T, ctx->D, L, G, y.num_chunks, ctx->d_status);
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
     dq_mark(ctx, st, DQ_K_SEG_REDUCE);
     int64_t fblocks = (y.num_chunks + 7) / 8;                // at most one cut segment per chunk, a warp each

@@ -10,6 +10,7 @@
 // segment is finished by one of the fix-up kernels (a warp for up to 32 pieces, a block
 // beyond that).  The per-table abs-max of the rounded sums is collected on the way.
 #pragma once
+#include <type_traits>
 #include "common.cuh"
 
 namespace segred {
@@ -106,16 +107,20 @@ __device__ __forceinline__ void vec_add(double (&acc)[VEC], const typename Vec<V
 // neighbouring keys once; the resulting bit mask of segment heads and the payloads (parked in
 // shared memory) are all the walk needs, so an entry costs one shared load, one address, one
 // 128-bit load, a bit test and the FP64 adds.
-template <int LPR, int VEC, int CH>
-__global__ void __launch_bounds__(256)
+// (256-byte rows want four resident blocks per SM: that caps the kernel at 64 registers)
+template <int LPR, int VEC, int CH, bool EXACT>
+__global__ void __launch_bounds__(256, (LPR == 16 && VEC == 4 && CH == 1) ? 4 : 1)
 seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
                   const u32 *__restrict__ seg_start, const u32 *__restrict__ chunk_first,
                   const int32_t *__restrict__ uniq_off,
                   const float *__restrict__ grad_out, float *__restrict__ grad_rows,
                   double *__restrict__ partials, u32 *__restrict__ long_list, u32 *__restrict__ counters,
-                  u32 *__restrict__ absmax, int T, int D,
+                  u32 *__restrict__ absmax, int T, int D_any,
                   int64_t L, int64_t G, int64_t num_chunks, int *__restrict__ status)
 {
+    // EXACT: the feature size fills the lanes exactly, so it is a compile-time constant and the
+    // per-vector range checks fall away
+    const int D = EXACT ? LPR * VEC * CH : D_any;
     extern __shared__ unsigned char smem_raw[];
     u32 *s_uoff = reinterpret_cast<u32 *>(smem_raw);                                     // [T+1]
     u32 *s_vals = s_uoff + (T + 1) + (size_t)(threadIdx.x / LPR) * CHUNK;                // this group's [CHUNK]
@@ -196,7 +201,7 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
 #pragma unroll
                 for (int ch = 0; ch < CH; ++ch) {
                     const int cv = ch * LPR + lane;
-                    if (cv < dv) {
+                    if (EXACT || cv < dv) {
                         float *dst = grad_rows + (int64_t)u * D + cv * VEC;
                         if constexpr (VEC == 1) { float r = (float)acc[ch][0]; *dst = r; m = fmaxf(m, fabsf(r)); }
                         else if constexpr (VEC == 2) {
@@ -216,7 +221,7 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
 #pragma unroll
                 for (int ch = 0; ch < CH; ++ch) {
                     const int cv = ch * LPR + lane;
-                    if (cv < dv) {
+                    if (EXACT || cv < dv) {
 #pragma unroll
                         for (int q = 0; q < VEC; ++q) pdst[cv * VEC + q] = acc[ch][q];
                     }
@@ -232,36 +237,42 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
             }
         };
 
-        for (int eb = 0; eb < n; eb += NB) {
-            vec_t r[NB][CH];
+        // a full chunk (all but the arena's last) needs no per-entry range checks
+        auto walk = [&](auto full_tag) {
+            constexpr bool FULL = decltype(full_tag)::value;
+            const int n_walk = FULL ? CHUNK : n;
+            for (int eb = 0; eb < n_walk; eb += NB) {
+                vec_t r[NB][CH];
 #pragma unroll
-            for (int e = 0; e < NB; ++e) {
-                if (eb + e < n) {
-                    const vec_t *src = g_lane + (int64_t)s_vals[eb + e] * dv;
-#pragma unroll
-                    for (int ch = 0; ch < CH; ++ch)
-                        if (ch * LPR + lane < dv) r[e][ch] = __ldg(src + ch * LPR);
-                }
-            }
-            const u32 hb = heads >> eb;
-#pragma unroll
-            for (int e = 0; e < NB; ++e) {
-                if (eb + e < n) {
-                    if ((hb >> e) & 1u) {
-                        flush(run_start, eb + e);
-                        u += 1;
-                        run_start = eb + e;
+                for (int e = 0; e < NB; ++e) {
+                    if (FULL || eb + e < n) {
+                        const vec_t *src = g_lane + (int64_t)s_vals[eb + e] * dv;
 #pragma unroll
                         for (int ch = 0; ch < CH; ++ch)
-#pragma unroll
-                            for (int q = 0; q < VEC; ++q) acc[ch][q] = 0.0;
+                            if (EXACT || ch * LPR + lane < dv) r[e][ch] = __ldg(src + ch * LPR);
                     }
+                }
+                const u32 hb = heads >> eb;
 #pragma unroll
-                    for (int ch = 0; ch < CH; ++ch)
-                        if (ch * LPR + lane < dv) vec_add<VEC>(acc[ch], r[e][ch]);
+                for (int e = 0; e < NB; ++e) {
+                    if (FULL || eb + e < n) {
+                        if ((hb >> e) & 1u) {
+                            flush(run_start, eb + e);
+                            u += 1;
+                            run_start = eb + e;
+#pragma unroll
+                            for (int ch = 0; ch < CH; ++ch)
+#pragma unroll
+                                for (int q = 0; q < VEC; ++q) acc[ch][q] = 0.0;
+                        }
+#pragma unroll
+                        for (int ch = 0; ch < CH; ++ch)
+                            if (EXACT || ch * LPR + lane < dv) vec_add<VEC>(acc[ch], r[e][ch]);
+                    }
                 }
             }
-        }
+        };
+        if (n == CHUNK) walk(std::true_type{}); else walk(std::false_type{});
         flush(run_start, n);
     }
     absmax_push<LPR>(tr, absmax);      // group-uniform: all lanes of a group walk the same chunks
