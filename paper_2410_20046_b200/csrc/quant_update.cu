@@ -71,14 +71,16 @@ absmax_kernel(const float *__restrict__ grad_rows, const int32_t *__restrict__ u
 // rows in flight per lane group: fewer when a lane already holds several vectors of every row
 template <int CH> struct RowsInFlight { static constexpr int v = CH >= 4 ? 1 : (CH == 2 ? 2 : 4); };
 
-template <int MODE, int LPR, int CH>
+// EXACT: the feature size is 4*LPR*CH, a compile-time constant, and the per-vector range checks fall away
+template <int MODE, int LPR, int CH, bool EXACT>
 __global__ void __launch_bounds__(QU_THREADS)
 row_stream_kernel(float *__restrict__ tables, const int64_t *__restrict__ row_off,
                   const int32_t *__restrict__ unique_rows, const int32_t *__restrict__ uniq_off,
                   const float *__restrict__ grad_rows, const u32 *__restrict__ absmax,
-                  int8_t *__restrict__ codes, float *__restrict__ grad_scales, float lr, int T, int D)
+                  int8_t *__restrict__ codes, float *__restrict__ grad_scales, float lr, int T, int D_any)
 {
     constexpr int NB = RowsInFlight<CH>::v;
+    const int D = EXACT ? 4 * LPR * CH : D_any;
     extern __shared__ unsigned char smem_raw[];
     int32_t *s_uoff = reinterpret_cast<int32_t *>(smem_raw);      // [T+1]
     float *s_scale = reinterpret_cast<float *>(s_uoff + (T + 1)); // [T] gradient scale of every table
@@ -128,7 +130,7 @@ row_stream_kernel(float *__restrict__ tables, const int64_t *__restrict__ row_of
 #pragma unroll
                 for (int ch = 0; ch < CH; ++ch) {
                     const int c4 = ch * LPR + lane;
-                    if (c4 < d4) {
+                    if (EXACT || c4 < d4) {
                         if (MODE == MODE_UPDATE) cin[b][ch] = *reinterpret_cast<const char4 *>(codes + (u + b) * D + 4 * c4);
                         else g[b][ch] = __ldg(reinterpret_cast<const float4 *>(grad_rows + (u + b) * D) + c4);
                         if (MODE != MODE_QUANT) w[b][ch] = wrow[b][c4];
@@ -142,7 +144,7 @@ row_stream_kernel(float *__restrict__ tables, const int64_t *__restrict__ row_of
 #pragma unroll
                 for (int ch = 0; ch < CH; ++ch) {
                     const int c4 = ch * LPR + lane;
-                    if (c4 < d4) {
+                    if (EXACT || c4 < d4) {
                         float4 q;                      // integer codes held as floats
                         if (MODE == MODE_UPDATE) {
                             q = make_float4((float)cin[b][ch].x, (float)cin[b][ch].y, (float)cin[b][ch].z, (float)cin[b][ch].w);
@@ -176,9 +178,12 @@ int launch_rows(dqrm_ctx *ctx, float *tables, const int32_t *unique_rows, const 
 {
     const size_t smem = (size_t)(ctx->T + 1) * sizeof(int32_t) + (size_t)ctx->T * sizeof(float);
     int grid = ctx->num_sms * 8;      // U lives on the device: a fixed grid splits the rows evenly
-    row_stream_kernel<MODE, LPR, CH><<<grid, QU_THREADS, smem, st>>>(tables, ctx->d_row_off, unique_rows, uniq_off,
-                                                                     grad_rows, absmax, codes, grad_scales, lr,
-                                                                     ctx->T, ctx->D);
+    if (ctx->D == 4 * LPR * CH)
+        row_stream_kernel<MODE, LPR, CH, true><<<grid, QU_THREADS, smem, st>>>(
+            tables, ctx->d_row_off, unique_rows, uniq_off, grad_rows, absmax, codes, grad_scales, lr, ctx->T, ctx->D);
+    else
+        row_stream_kernel<MODE, LPR, CH, false><<<grid, QU_THREADS, smem, st>>>(
+            tables, ctx->d_row_off, unique_rows, uniq_off, grad_rows, absmax, codes, grad_scales, lr, ctx->T, ctx->D);
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
     dq_mark(ctx, st, MODE == MODE_QUANT ? DQ_K_QUANT : (MODE == MODE_UPDATE ? DQ_K_UPDATE : DQ_K_QUANT_UPDATE));
     return DQRM_OK;
