@@ -232,3 +232,30 @@ def packed_fwd(packed, row_off, D, B, indices, offsets, scales, bits):
                                  _p(np.ascontiguousarray(scales, dtype=np.float32), np.float32), int(bits),
                                  _p(out, np.float32))
     return out
+
+
+def emb_fwd_codes(tables, row_off, D, B, indices, offsets, scales, bits):
+    """Packed codes of every one-index bag's row -> uint8 [B, T, D*bits/8]."""
+    T = len(row_off) - 1
+    assert bits in (2, 4, 8) and (D * bits) % 8 == 0
+    row_off = np.ascontiguousarray(row_off, dtype=np.int64)
+    payload = np.empty((B, T, D * bits // 8), dtype=np.uint8)
+    f = lib().dqrm_oracle_emb_fwd_codes
+    f.restype = ctypes.c_int
+    rc = f(_p(tables, np.float32), _p(row_off, np.int64), T, int(D), int(B), _p(indices, np.int32),
+           _p(offsets, np.int32), _p(np.ascontiguousarray(scales, dtype=np.float32), np.float32), int(bits),
+           _p(payload, np.uint8))
+    if rc != 0:
+        raise ValueError("emb_fwd_codes needs exactly one index per bag")
+    return payload
+
+
+def decode_payload(payload, scales, bits, D, T_total, t0, out=None):
+    """out[i, t0 + j, :] = code * scales[j] for payload [B, T_blk, D*bits/8]."""
+    B, T_blk = payload.shape[0], payload.shape[1]
+    if out is None:
+        out = np.zeros((B, T_total, D), dtype=np.float32)
+    lib().dqrm_oracle_decode_payload(_p(np.ascontiguousarray(payload), np.uint8),
+                                     _p(np.ascontiguousarray(scales, dtype=np.float32), np.float32), int(bits), int(B),
+                                     int(T_blk), int(T_total), int(t0), int(D), _p(out, np.float32))
+    return out

@@ -355,3 +355,43 @@ void dqrm_oracle_packed_fwd(const uint8_t *packed, const int64_t *row_off, int T
         }
     free(acc);
 }
+
+/* ---- table-sharded forward payload (paper Section 4.3, the remark on hybrid parallelism: the
+ * all-to-all that carries embedding vectors shrinks with the code width) -------------------------
+ * For one-index bags the pooled vector is the dequantised row, so the owner of a table can send the
+ * row's b-bit codes instead of FP32 values.  payload[i][t] holds the packed codes (layout of
+ * dqrm_oracle_pack_tables) of bag (t, i)'s row.  Returns 0, or -1 when a bag does not hold exactly
+ * one index. */
+int dqrm_oracle_emb_fwd_codes(const float *tables, const int64_t *row_off, int T, int D, int B,
+                              const int32_t *indices, const int32_t *offsets, const float *scales, int bits,
+                              uint8_t *payload /* [B][T][D*bits/8] */)
+{
+    const int row_bytes = D * bits / 8;
+    const uint32_t mask = (1u << bits) - 1u;
+    for (int t = 0; t < T; ++t)
+        for (int i = 0; i < B; ++i) {
+            int64_t g = (int64_t)t * B + i;
+            if (offsets[g + 1] - offsets[g] != 1) return -1;
+            const float *row = tables + (row_off[t] + (int64_t)indices[offsets[g]]) * D;
+            uint8_t *dst = payload + ((int64_t)i * T + t) * row_bytes;
+            memset(dst, 0, (size_t)row_bytes);
+            for (int d = 0; d < D; ++d) {
+                int32_t q = dqrm_oracle_quantize(row[d], scales[t], bits);
+                dst[(d * bits) / 8] |= (uint8_t)(((uint32_t)q & mask) << ((d * bits) % 8));
+            }
+        }
+    return 0;
+}
+
+/* receiver side: out[i][t0 + j][:] = code * scales[j] for the T_blk tables of one sender */
+void dqrm_oracle_decode_payload(const uint8_t *payload /* [B][T_blk][D*bits/8] */, const float *scales /* [T_blk] */,
+                                int bits, int B, int T_blk, int T_total, int t0, int D, float *out /* [B][T_total][D] */)
+{
+    const int row_bytes = D * bits / 8;
+    for (int i = 0; i < B; ++i)
+        for (int j = 0; j < T_blk; ++j) {
+            const uint8_t *row = payload + ((int64_t)i * T_blk + j) * row_bytes;
+            float *o = out + ((int64_t)i * T_total + t0 + j) * D;
+            for (int d = 0; d < D; ++d) o[d] = dqrm_oracle_dequantize(unpack_code(row, d, bits), scales[j]);
+        }
+}
