@@ -256,6 +256,23 @@ int dqrm_pack_tables(dqrm_ctx *ctx, const float *tables, const float *scales, in
 int dqrm_packed_fwd(dqrm_ctx *ctx, const uint8_t *packed, const int32_t *indices, const int32_t *offsets,
                     const float *scales, int bits, float *out, int B, int64_t L, void *stream);
 
+/* ---- table-sharded forward payload (Section 4.3, the remark on hybrid parallelism) -----------
+ * With the tables sharded over ranks, the all-to-all that carries embedding vectors shrinks with
+ * the code width: for one-index bags the pooled vector is the dequantised row, so a table's owner
+ * sends the row's bit-packed codes (layout of dqrm_pack_tables, bits in {2, 4, 8} for all tables)
+ * and the samples' owner multiplies by the table's scale.
+ * dqrm_emb_fwd_codes: payload[i][t][D*bits/8] = packed Q(row of bag (t, i)) for the context's T
+ *   tables and B bags per table; every bag must hold exactly one index (L == T*B, else
+ *   DQRM_ERR_INVALID_ARG; a bag that does not is reported as DQRM_ERR_INDEX_RANGE and left unwritten).
+ * dqrm_decode_payload: out[i][t0 + j][:] = code * scales[j] for a payload block [B][T_blk][D*bits/8]
+ *   of T_blk consecutive tables starting at table t0 of an output [B][T_total][D] (D is the
+ *   context's; its tables are not used).  Decoding every sender's block gives, bit for bit, what
+ *   dqrm_emb_fwd computes on the unsharded problem. */
+int dqrm_emb_fwd_codes(dqrm_ctx *ctx, const float *tables, const int32_t *indices, const int32_t *offsets,
+                       const float *scales, int bits, uint8_t *payload, int B, int64_t L, void *stream);
+int dqrm_decode_payload(dqrm_ctx *ctx, const uint8_t *payload, const float *scales, int bits, float *out, int B,
+                        int T_blk, int T_total, int t0, void *stream);
+
 /* ---- choice of the backward's sort (no counterpart in the paper) --------------------
  * dqrm_emb_bwd and dqrm_train_step order the batch's lookups by row before they sum
  * duplicates.  path 0 (default): one thread-block cluster per table sorts that table's

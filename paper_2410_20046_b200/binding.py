@@ -52,6 +52,8 @@ SIGNATURES = {
     "dqrm_packed_bytes": (_sz, [_vp, _i]),
     "dqrm_pack_tables": (_i, [_vp, _vp, _vp, _i, _vp, _vp]),
     "dqrm_packed_fwd": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _vp, _i, _i64, _vp]),
+    "dqrm_emb_fwd_codes": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _vp, _i, _i64, _vp]),
+    "dqrm_decode_payload": (_i, [_vp, _vp, _vp, _i, _vp, _i, _i, _i, _i, _vp]),
     "dqrm_set_sort_path": (_i, [_vp, _i]),
     "dqrm_set_overlap": (_i, [_vp, _i]),
     "dqrm_launch_count": (_i64, [_vp]),
@@ -231,6 +233,21 @@ class Context:
         self._check("dqrm_packed_fwd", self.lib.dqrm_packed_fwd(
             self._h, _ptr(packed, torch.uint8), _ptr(indices, torch.int32), _ptr(offsets, torch.int32),
             _ptr(scales, torch.float32), int(bits), _ptr(out, torch.float32), int(B), int(L), _stream(stream)))
+
+    # ---- table-sharded forward payload ----
+    def emb_fwd_codes(self, tables, indices, offsets, scales, bits, payload, *, B, L, stream=None):
+        import torch
+
+        self._check("dqrm_emb_fwd_codes", self.lib.dqrm_emb_fwd_codes(
+            self._h, _ptr(tables, torch.float32), _ptr(indices, torch.int32), _ptr(offsets, torch.int32),
+            _ptr(scales, torch.float32), int(bits), _ptr(payload, torch.uint8), int(B), int(L), _stream(stream)))
+
+    def decode_payload(self, payload, scales, bits, out, *, B, T_blk, T_total, t0, stream=None):
+        import torch
+
+        self._check("dqrm_decode_payload", self.lib.dqrm_decode_payload(
+            self._h, _ptr(payload, torch.uint8), _ptr(scales, torch.float32), int(bits), _ptr(out, torch.float32),
+            int(B), int(T_blk), int(T_total), int(t0), _stream(stream)))
 
     def set_overlap(self, on: bool):
         self._check("dqrm_set_overlap", self.lib.dqrm_set_overlap(self._h, int(bool(on))))

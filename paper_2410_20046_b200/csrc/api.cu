@@ -195,7 +195,7 @@ const char *dqrm_kernel_name(int kernel_id)
         "begin", "refresh_kernel", "fwd_kernel", "memset", "prepare_kernel", "sort_scan_kernel",
         "sort_scatter_kernel", "seg_count_kernel", "seg_emit_kernel", "seg_reduce_kernel", "seg_fixup_kernel",
         "absmax_kernel", "row_stream_kernel<quant>", "row_stream_kernel<update>", "row_stream_kernel<fused>",
-        "copy", "seg_fixup_big_kernel", "cluster_sort_kernel", "dp_pack_kernel", "dp_sum_update_kernel", "pack_kernel", "packed_fwd_kernel"};
+        "copy", "seg_fixup_big_kernel", "cluster_sort_kernel", "dp_pack_kernel", "dp_sum_update_kernel", "pack_kernel", "packed_fwd_kernel", "fwd_codes_kernel", "decode_payload_kernel"};
     return (kernel_id >= 0 && kernel_id < DQ_K_COUNT) ? names[kernel_id] : "?";
 }
 
@@ -364,6 +364,24 @@ int dqrm_train_step_sorted(dqrm_ctx *ctx, float *tables, const int32_t *indices,
     if (rc != DQRM_OK) return rc;
     return dq_launch_quant_update(ctx, tables, unique_rows, uniq_off, grad_rows,
                                   dq_bwd_absmax_bits(ctx, L, workspace), codes, grad_scales, lr, st);
+}
+
+int dqrm_emb_fwd_codes(dqrm_ctx *ctx, const float *tables, const int32_t *indices, const int32_t *offsets,
+                       const float *scales, int bits, uint8_t *payload, int B, int64_t L, void *stream)
+{
+    if (!batch_ok(ctx, B, L) || !tables || !offsets || !scales || !payload || (bits != 2 && bits != 4 && bits != 8))
+        return DQRM_ERR_INVALID_ARG;
+    if (L != (int64_t)ctx->T * B || (L > 0 && !indices)) return DQRM_ERR_INVALID_ARG;     // one index per bag
+    return dq_launch_fwd_codes(ctx, tables, indices, offsets, scales, bits, payload, B, L, as_stream(stream));
+}
+
+int dqrm_decode_payload(dqrm_ctx *ctx, const uint8_t *payload, const float *scales, int bits, float *out, int B,
+                        int T_blk, int T_total, int t0, void *stream)
+{
+    if (!ctx || !payload || !scales || !out || B < 0 || T_blk < 0 || t0 < 0 || t0 + T_blk > T_total ||
+        (bits != 2 && bits != 4 && bits != 8))
+        return DQRM_ERR_INVALID_ARG;
+    return dq_launch_decode_payload(ctx, payload, scales, bits, out, B, T_blk, T_total, t0, as_stream(stream));
 }
 
 size_t dqrm_packed_bytes(const dqrm_ctx *ctx, int bits)

@@ -34,7 +34,7 @@ struct dqrm_ctx {
 enum {
     DQ_K_BEGIN = 0, DQ_K_REFRESH, DQ_K_FWD, DQ_K_MEMSET, DQ_K_PREPARE, DQ_K_SORT_SCAN, DQ_K_SORT_SCATTER,
     DQ_K_SEG_COUNT, DQ_K_SEG_EMIT, DQ_K_SEG_REDUCE, DQ_K_SEG_FIXUP, DQ_K_ABSMAX, DQ_K_QUANT, DQ_K_UPDATE,
-    DQ_K_QUANT_UPDATE, DQ_K_COPY, DQ_K_SEG_FIXUP_BIG, DQ_K_CLUSTER_SORT, DQ_K_DP_PACK, DQ_K_DP_SUM_UPDATE, DQ_K_PACK, DQ_K_PACKED_FWD, DQ_K_COUNT
+    DQ_K_QUANT_UPDATE, DQ_K_COPY, DQ_K_SEG_FIXUP_BIG, DQ_K_CLUSTER_SORT, DQ_K_DP_PACK, DQ_K_DP_SUM_UPDATE, DQ_K_PACK, DQ_K_PACKED_FWD, DQ_K_FWD_CODES, DQ_K_DECODE_PAYLOAD, DQ_K_COUNT
 };
 constexpr int DQ_PROF_MAX = 4096;
 
@@ -207,6 +207,10 @@ int dq_launch_grad_quant_unified(dqrm_ctx *ctx, const float *grad_rows, const in
 int dq_launch_pack(dqrm_ctx *ctx, const float *tables, const float *scales, int bits, uint8_t *packed, cudaStream_t st);
 int dq_launch_packed_fwd(dqrm_ctx *ctx, const uint8_t *packed, const int32_t *indices, const int32_t *offsets,
                          const float *scales, int bits, float *out, int B, int64_t L, cudaStream_t st);
+int dq_launch_fwd_codes(dqrm_ctx *ctx, const float *tables, const int32_t *indices, const int32_t *offsets,
+                        const float *scales, int bits, uint8_t *payload, int B, int64_t L, cudaStream_t st);
+int dq_launch_decode_payload(dqrm_ctx *ctx, const uint8_t *payload, const float *scales, int bits, float *out, int B,
+                             int T_blk, int T_total, int t0, cudaStream_t st);
 size_t dq_dp_ws_bytes(const dqrm_ctx *ctx, int64_t max_entries);
 int dq_launch_dp_merge_update(dqrm_ctx *ctx, float *tables, int W, int64_t rank_stride, const int32_t *rows_cat,
                               const int32_t *uoff_cat, const int8_t *codes_cat, const float *grad_scales, float lr,
