@@ -47,6 +47,13 @@ def get_workload(name):
 
     if name in W.BY_NAME:
         return W.BY_NAME[name]()
+    if name.startswith("sweep_"):   # sweep_d64_b8_zipf: one table of 10 M rows, batch 65536 (feature size, bits, index law)
+        try:
+            d, b, dist = name.split("_")[1:]
+            assert d[0] == "d" and b[0] == "b" and dist in ("uniform", "zipf")
+            return W.sweep(D=int(d[1:]), bits=int(b[1:]), zipf=(dist == "zipf"))
+        except (ValueError, AssertionError):
+            raise SystemExit(f"bad sweep name {name}; expected sweep_d<16|32|64|128>_b<2|4|8>_<uniform|zipf>")
     if name == "kaggle_smoke":      # small stand-in used by the tests of this script
         return W.scaled_down(W.kaggle(), total_rows=200_000, B=1024, name="kaggle_smoke")
     raise SystemExit(f"unknown workload {name}; choose from {sorted(W.BY_NAME)}")
@@ -217,6 +224,10 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     dq.load_library()
+    capture_stream = None
+    if args.train_priority != 0:                     # the whole run, graph capture included, on a stream of that priority
+        torch.cuda.set_stream(torch.cuda.Stream(priority=args.train_priority))
+        capture_stream = torch.cuda.Stream(priority=args.train_priority)
 
     wl = get_workload(args.workload)
     G = wl.T * wl.B
@@ -268,7 +279,7 @@ def run_ours(args):
     pipelined = not args.no_pipeline and not (args.dp_exchange and world > 1)
     if pipelined:
         assert N_BATCHES % 2 == 0
-        side = torch.cuda.Stream(priority=-1)
+        side = torch.cuda.Stream(priority=args.sort_priority)
         ctx._workspace(1)                                   # allocate the second workspace before any capture
         urs = [ur, torch.empty_like(ur)]
         uos = [uo, torch.empty_like(uo)]
@@ -302,8 +313,14 @@ def run_ours(args):
         def launch_step(bi):     # noqa: F811  (the exchange has host-side size reads, so no graph capture)
             b = batches[bi]
             dp_step.step(tables, b["idx"], b["off"], b["go"], scales, bits, wl.lr, b["L"])
-    graphs = None
+    graphs = None            # one CUDA graph per pre-staged batch: that batch's step
+    group_graphs = None      # one CUDA graph per `spg` consecutive batches: their steps back to back
     launches_per_step = 0
+    # steps per graph: whole groups must tile the batch ring and the refresh period; a timed region that is not a
+    # whole number of groups ends with single-step graphs
+    spg = args.steps_per_graph
+    if spg < 1 or N_BATCHES % spg or wl.period % spg:
+        spg = 1
     if not args.no_graph and dp_step is None:
         try:
             if pipelined:
@@ -311,42 +328,54 @@ def run_ours(args):
             for bi in range(2):
                 launch_step(bi)                      # first use outside capture (function attributes, caches)
             torch.cuda.synchronize()
-            graphs = []
-            for bi in range(N_BATCHES):
+
+            def capture(first, count):
                 g = torch.cuda.CUDAGraph()
-                n_before = ctx.launch_count()
-                with torch.cuda.graph(g):
-                    launch_step(bi)
-                launches_per_step = ctx.launch_count() - n_before      # kernels recorded into the graph
-                graphs.append(g)
+                with torch.cuda.graph(g, stream=capture_stream):
+                    for bi in range(first, first + count):
+                        launch_step(bi)
+                return g
+
+            n_before = ctx.launch_count()
+            graphs = [capture(bi, 1) for bi in range(N_BATCHES)]
+            launches_per_step = (ctx.launch_count() - n_before) // N_BATCHES    # kernels recorded per step
+            if spg > 1:
+                group_graphs = [capture(b0, spg) for b0 in range(0, N_BATCHES, spg)]
             torch.cuda.synchronize()
         except Exception as e:                       # capture refused: plain launches
             print(f"bench: CUDA graph capture failed ({e}); launching directly", file=sys.stderr)
-            graphs = None
+            graphs = group_graphs = None
             torch.cuda.synchronize()
 
     last = {"s": None}
 
-    def step(s, direct=False):
+    def step(s, end=None, direct=False):
+        """Runs step s, or steps s .. s+spg-1 from one graph when they all lie before `end`; returns how many."""
         if s % wl.period == 0:
             ctx.scale_refresh(tables, bits, scales)
         if direct and pipelined:                     # the per-kernel timing pass: one stream, one call per step
             launch_unpipelined(s % N_BATCHES)
             last["s"] = None
-            return
+            return 1
         if pipelined and last["s"] != s - 1:
             prime(s % N_BATCHES)                     # (re)start of the pipeline: this batch is not sorted yet
+        if group_graphs is not None and not direct and s % spg == 0 and end is not None and s + spg <= end:
+            group_graphs[(s % N_BATCHES) // spg].replay()      # no refresh falls inside: spg divides the period
+            last["s"] = s + spg - 1
+            return spg
         last["s"] = s
         if graphs is not None and not direct:
             graphs[s % N_BATCHES].replay()
         else:
             launch_step(s % N_BATCHES)
+        return 1
 
-    def step_host(s):
+    def step_host(s, end=None):
         if s % wl.period == 0:
             ctx.scale_refresh(tables, bits, scales)
         b = batches[s % N_BATCHES]
         ctx.train_step_host(tables, b["idx_h"], b["off_h"], b["go_h"], scales, bits, out_h, wl.lr, B=wl.B, L=b["L"])
+        return 1
 
     def sync_all():
         torch.cuda.synchronize()
@@ -355,8 +384,9 @@ def run_ours(args):
             torch.cuda.synchronize()
 
     def timed(fn, steps, warmup, sample_clocks=False):
-        for s in range(warmup):
-            fn(s)
+        s = 0
+        while s < warmup:
+            s += fn(s, warmup)
         sync_all()
         sampler = ClockSampler(local_rank) if (sample_clocks and rank == 0) else None
         if sampler:
@@ -364,8 +394,8 @@ def run_ours(args):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         n0 = ctx.launch_count()
         e0.record()
-        for s in range(steps):
-            fn(warmup + s)
+        while s < warmup + steps:                      # exactly `steps` steps: s never passes the end
+            s += fn(s, warmup + steps)
         e1.record()
         sync_all()
         ms = e0.elapsed_time(e1)
@@ -434,7 +464,8 @@ def run_ours(args):
             "config": {"workload": wl.name, "tables": wl.T, "dim": wl.D, "batch_per_gpu": wl.B,
                        "lookups_per_step_per_gpu": Lavg, "unique_rows_per_step": Uavg, "unique_fraction": Uavg / Lavg,
                        "bits": wl.bits, "grad_bits": 8, "refresh_period": wl.period, "table_bytes": wl.table_bytes(),
-                       "launch": ("CUDA graph replay per step" if graphs is not None else "direct launches") +
+                       "launch": ((f"CUDA graph replay, {spg} consecutive steps per graph" if group_graphs is not None else
+                                   "CUDA graph replay per step") if graphs is not None else "direct launches") +
                                  ("; the index sort of batch k+1 runs on a second stream while batch k trains "
                                   "(two workspaces, every step does one sort and one training half)" if pipelined
                                   else ""),
@@ -573,6 +604,13 @@ def main():
                          "instead of running independent replicas")
     ap.add_argument("--no-graph", action="store_true", help="launch every step directly instead of replaying CUDA graphs")
     ap.add_argument("--no-overlap", action="store_true", help="keep the index sort on the caller's stream")
+    ap.add_argument("--steps-per-graph", type=int, default=4,
+                    help="consecutive steps replayed from one CUDA graph (must divide 16 and the refresh period, else 1; "
+                         "a remainder of the timed region runs from single-step graphs)")
+    ap.add_argument("--sort-priority", type=int, default=0,
+                    help="priority of the second stream that sorts the next batch (-1 high, 0 default)")
+    ap.add_argument("--train-priority", type=int, default=-1,
+                    help="priority of the stream the training half runs on (0: torch's current stream)")
     ap.add_argument("--sort-path", type=int, default=0, help="0: per-table cluster sort, 1: global radix sort")
     args = ap.parse_args()
     if args.impl == "reference":
