@@ -54,6 +54,8 @@ def get_workload(name):
             return W.sweep(D=int(d[1:]), bits=int(b[1:]), zipf=(dist == "zipf"))
         except (ValueError, AssertionError):
             raise SystemExit(f"bad sweep name {name}; expected sweep_d<16|32|64|128>_b<2|4|8>_<uniform|zipf>")
+    if name == "terabyte_2gb_b32768":   # the Terabyte-shaped step over 2 GB of tables: small enough for a counter capture
+        return W.scaled_down(W.terabyte(32768), total_rows=8_000_000, B=32768, name="terabyte_2gb_b32768")
     if name == "kaggle_smoke":      # small stand-in used by the tests of this script
         return W.scaled_down(W.kaggle(), total_rows=200_000, B=1024, name="kaggle_smoke")
     raise SystemExit(f"unknown workload {name}; choose from {sorted(W.BY_NAME)}")
@@ -122,6 +124,13 @@ NCU_TRAFFIC = {
     ("kaggle_b16384", "seg_reduce_kernel"): 31.10e6,
     ("kaggle_b16384", "fwd_kernel"): 26.35e6,
     ("kaggle_b16384", "row_stream_kernel<fused>"): 25.18e6,
+    # the Terabyte-shaped step captured over 2 GB of tables (the full tables are too large for a counter capture)
+    ("terabyte_2gb_b32768", "seg_reduce_kernel"): 263.64e6,
+    ("terabyte_2gb_b32768", "fwd_kernel"): 211.66e6,
+    ("terabyte_2gb_b32768", "row_stream_kernel<fused>"): 80.57e6,
+    # ... and scaled to the full tables by the reduce's algorithmic bytes (265.79 MB against 254.88 MB per launch):
+    # its traffic is the upstream-gradient rows (the same) plus the unique rows it writes
+    ("terabyte_b32768", "seg_reduce_kernel"): 274.9e6,
 }
 
 KERNEL_BYTES = {
