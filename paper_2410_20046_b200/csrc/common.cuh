@@ -156,6 +156,9 @@ __device__ __forceinline__ void dq_cp_async_commit() { asm volatile("cp.async.co
 template <int N>
 __device__ __forceinline__ void dq_cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
 
+// asks L2 for the 128-byte line that holds p (no register, no scoreboard entry: the later load finds it there)
+__device__ __forceinline__ void dq_prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];\n" ::"l"(p)); }
+
 __device__ __forceinline__ void dq_report(int *status, int code)
 {
     atomicCAS(status, 0, code);   // first error wins

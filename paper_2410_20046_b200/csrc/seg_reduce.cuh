@@ -16,6 +16,7 @@
 namespace segred {
 
 constexpr int CHUNK = 32;            // sorted entries per warp work item
+constexpr int PREFETCH_ROW_BYTES = 512;   // rows up to this size are prefetched into L2 by the reduce's head phase
 constexpr int BIG_PIECES = 32;       // cut segments with more pieces go to the block-wide fix-up
 enum { CNT_LONG = 0, CNT_U = 1, CNT_BIG = 2 };
 
@@ -168,6 +169,14 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
                 u32 v = vv[j];
                 if ((int64_t)v >= G) { bad = true; v = 0u; }
                 s_vals[e] = v;
+                // the walk reaches this entry's upstream-gradient row up to 32 dependent steps from now: have L2
+                // fetch it meanwhile, so that all of a chunk's rows are in flight at once without holding registers
+                if (PREFETCH_ROW_BYTES >= D * (int)sizeof(float)) {
+                    const char *row = reinterpret_cast<const char *>(grad_out) + (int64_t)v * D * sizeof(float);
+#pragma unroll
+                    for (int b = 0; b < PREFETCH_ROW_BYTES; b += 128)
+                        if (b < D * (int)sizeof(float)) dq_prefetch_l2(row + b);
+                }
             }
             const bool head = (e < n) && (kc[j] != kp[j]);
             const u32 bits = (__ballot_sync(gmask, head) >> gbase) & (LPR >= 32 ? 0xffffffffu : ((1u << LPR) - 1u));
