@@ -121,16 +121,16 @@ def algorithmic_bytes(wl, L, G, U):
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (set an entry to None when its kernel has changed since the capture)
 NCU_TRAFFIC = {
-    ("kaggle_b16384", "seg_reduce_kernel"): None,
+    ("kaggle_b16384", "seg_reduce_kernel"): 31.11e6,
     ("kaggle_b16384", "fwd_kernel"): 26.35e6,
     ("kaggle_b16384", "row_stream_kernel<fused>"): 25.18e6,
     # the Terabyte-shaped step captured over 2 GB of tables (the full tables are too large for a counter capture)
-    ("terabyte_2gb_b32768", "seg_reduce_kernel"): None,
-    ("terabyte_2gb_b32768", "fwd_kernel"): 211.66e6,
-    ("terabyte_2gb_b32768", "row_stream_kernel<fused>"): 80.57e6,
+    ("terabyte_2gb_b32768", "seg_reduce_kernel"): 274.15e6,
+    ("terabyte_2gb_b32768", "fwd_kernel"): 211.26e6,
+    ("terabyte_2gb_b32768", "row_stream_kernel<fused>"): 80.37e6,
     # ... and scaled to the full tables by the reduce's algorithmic bytes (265.79 MB against 254.88 MB per launch):
     # its traffic is the upstream-gradient rows (the same) plus the unique rows it writes
-    ("terabyte_b32768", "seg_reduce_kernel"): None,
+    ("terabyte_b32768", "seg_reduce_kernel"): 285.9e6,
 }
 
 KERNEL_BYTES = {
@@ -301,10 +301,17 @@ def run_ours(args):
             b, nb, slot = batches[bi], batches[(bi + 1) % N_BATCHES], bi & 1
             cur = torch.cuda.current_stream()
             side.wait_stream(cur)
-            ctx.sort_batch(nb["idx"], nb["off"], urs[slot ^ 1], uos[slot ^ 1], B=wl.B, L=nb["L"], ws=slot ^ 1,
-                           stream=side)
-            ctx.train_step_sorted(tables, b["idx"], b["off"], b["go"], scales, bits, out, urs[slot], uos[slot], gr,
-                                  codes, gs, wl.lr, B=wl.B, L=b["L"], ws=slot, stream=cur)
+            if args.sort_after_forward:               # the sort runs beside the gradient summation and the update
+                ctx.train_step_sorted(tables, b["idx"], b["off"], b["go"], scales, bits, out, urs[slot], uos[slot], gr,
+                                      codes, gs, wl.lr, B=wl.B, L=b["L"], ws=slot, stream=cur)
+                ctx.stream_wait_forward(side)
+                ctx.sort_batch(nb["idx"], nb["off"], urs[slot ^ 1], uos[slot ^ 1], B=wl.B, L=nb["L"], ws=slot ^ 1,
+                               stream=side)
+            else:                                     # the sort runs beside the whole training half
+                ctx.sort_batch(nb["idx"], nb["off"], urs[slot ^ 1], uos[slot ^ 1], B=wl.B, L=nb["L"], ws=slot ^ 1,
+                               stream=side)
+                ctx.train_step_sorted(tables, b["idx"], b["off"], b["go"], scales, bits, out, urs[slot], uos[slot], gr,
+                                      codes, gs, wl.lr, B=wl.B, L=b["L"], ws=slot, stream=cur)
             cur.wait_stream(side)
 
         def launch_unpipelined(bi):
@@ -620,6 +627,8 @@ def main():
                     help="priority of the second stream that sorts the next batch (-1 high, 0 default)")
     ap.add_argument("--train-priority", type=int, default=-1,
                     help="priority of the stream the training half runs on (0: torch's current stream)")
+    ap.add_argument("--sort-after-forward", type=int, default=0,
+                    help="1: the next batch's sort waits for this batch's forward and runs beside the rest of the step")
     ap.add_argument("--sort-path", type=int, default=0, help="0: per-table cluster sort, 1: global radix sort")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -173,6 +173,17 @@ int dqrm_train_step_sorted(dqrm_ctx *ctx, float *tables, const int32_t *indices,
                            int8_t *codes, float *grad_scales, float lr, int B, int64_t L,
                            void *workspace, size_t workspace_bytes, void *stream);
 
+/* Makes `stream` wait until the forward of the last dqrm_train_step_sorted enqueued on this
+ * context has finished (no counterpart in the paper).  For the pipelined loop above: the sort of
+ * batch k+1 shares the SMs with whatever runs beside it, and the forward is the one kernel of the
+ * step that is bound by instruction issue, so a loop may hold the sort back until batch k's
+ * forward is done and let it run beside the gradient summation and the update instead:
+ *   dqrm_train_step_sorted(batch k, stream A); dqrm_stream_wait_forward(ctx, stream B);
+ *   dqrm_sort_batch(batch k+1, stream B).
+ * Before the first dqrm_train_step_sorted the wait returns at once.  Inside a stream capture both
+ * calls must belong to the same capture. */
+int dqrm_stream_wait_forward(dqrm_ctx *ctx, void *stream);
+
 /* Bytes of workspace dqrm_train_step_host needs (device staging for the host buffers,
  * the step's intermediate outputs and the scratch of dqrm_train_step). */
 size_t dqrm_host_step_workspace_bytes(const dqrm_ctx *ctx, int64_t max_lookups, int64_t max_bags);

@@ -41,6 +41,7 @@ SIGNATURES = {
                                     _vp, _sz, _vp]),
     "dqrm_train_step": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _f, _i, _i64,
                              _vp, _sz, _vp]),
+    "dqrm_stream_wait_forward": (_i, [_vp, _vp]),
     "dqrm_host_step_workspace_bytes": (_sz, [_vp, _i64, _i64]),
     "dqrm_train_step_host": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _f, _i, _i64, _vp, _sz, _vp]),
     "dqrm_grad_quant_int8_static": (_i, [_i, _i, _vp, _vp, _vp, _vp, _vp]),
@@ -346,6 +347,9 @@ class Context:
             _ptr(out, torch.float32), _ptr(unique_rows, torch.int32), _ptr(uniq_off, torch.int32),
             _ptr(grad_rows, torch.float32), _ptr(codes, torch.int8), _ptr(grad_scales, torch.float32),
             float(lr), int(B), int(L), self._workspace(ws), self.workspace_bytes, _stream(stream)))
+
+    def stream_wait_forward(self, stream):
+        self._check("dqrm_stream_wait_forward", self.lib.dqrm_stream_wait_forward(self._h, _stream(stream)))
 
     def train_step_host(self, tables, h_indices, h_offsets, h_grad_out, scales, bits, h_out, lr, *, B, L,
                         stream=None):

@@ -81,6 +81,7 @@ int dqrm_create(dqrm_ctx **out, int T, int D, const int64_t *h_row_off)
     }
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fwd, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaMemcpy(ctx->d_row_off, h_row_off, sizeof(int64_t) * (T + 1), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(ctx->d_done, 0, sizeof(u32));
@@ -104,6 +105,7 @@ int dqrm_destroy(dqrm_ctx *ctx)
     if (ctx->side) cudaStreamDestroy(ctx->side);
     if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
     if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
+    if (ctx->ev_fwd) cudaEventDestroy(ctx->ev_fwd);
     if (ctx->prof_events) {
         for (int i = 0; i < DQ_PROF_MAX; ++i) cudaEventDestroy(ctx->prof_events[i]);
         delete[] ctx->prof_events;
@@ -360,10 +362,18 @@ int dqrm_train_step_sorted(dqrm_ctx *ctx, float *tables, const int32_t *indices,
     if (ctx->prof_on) dq_mark(ctx, st, DQ_K_BEGIN);
     int rc = dq_launch_fwd(ctx, tables, indices, offsets, scales, bits, out, nullptr, B, L, st);
     if (rc != DQRM_OK) return rc;
+    DQRM_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_fwd, st));      // for dqrm_stream_wait_forward
     rc = dq_launch_bwd_reduce(ctx, grad_out, uniq_off, grad_rows, B, L, workspace, workspace_bytes, st);
     if (rc != DQRM_OK) return rc;
     return dq_launch_quant_update(ctx, tables, unique_rows, uniq_off, grad_rows,
                                   dq_bwd_absmax_bits(ctx, L, workspace), codes, grad_scales, lr, st);
+}
+
+int dqrm_stream_wait_forward(dqrm_ctx *ctx, void *stream)
+{
+    if (!ctx) return DQRM_ERR_INVALID_ARG;
+    DQRM_CUDA_TRY(ctx, cudaStreamWaitEvent(as_stream(stream), ctx->ev_fwd, 0));
+    return DQRM_OK;
 }
 
 int dqrm_emb_fwd_codes(dqrm_ctx *ctx, const float *tables, const int32_t *indices, const int32_t *offsets,

@@ -22,6 +22,7 @@ struct dqrm_ctx {
     int sort_path = 0;              // 0: per-table cluster sort, 1: global radix sort
     cudaStream_t side = nullptr;    // second stream: a training step sorts the indices beside its forward
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    cudaEvent_t ev_fwd = nullptr;   // recorded behind the forward of the last training step enqueued
     int overlap = 1;                // 0: keep everything on the caller's stream
     int payload_position = 0;       // sort payload: 0 = row of grad_out, 1 = position of the lookup (set by the merge)
     // launch accounting and optional per-launch timing (see dqrm_profile_*)

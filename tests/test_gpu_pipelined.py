@@ -115,3 +115,57 @@ def test_two_calls_equal_one_call():
     for a, b in zip(*res):
         assert bit_equal(a, b)
     c.ctx.close()
+
+
+def test_sort_held_until_the_forward_is_done_equals_one_call():
+    """dqrm_stream_wait_forward: the next batch's sort starts only behind this batch's forward and runs
+    beside the rest of the step; the trajectory must equal the single-call loop's bit for bit."""
+    import torch
+
+    wl = W.scaled_down(W.terabyte(), total_rows=400_000, B=1500, name="terabyte_small")
+    c = Case(wl)
+    tables = W.tables_np(wl)
+    steps = 6
+    batches = [c.batch(s) for s in range(steps)]
+    res = []
+    for held in (False, True):
+        d_tables = c.dev(tables)
+        scales = c.empty(wl.T, torch.float32)
+        c.ctx.scale_refresh(d_tables, c.bits, scales)
+        out = c.empty((wl.B, wl.T, wl.D), torch.float32)
+        Lmax = max(len(b[0]) for b in batches)
+        urs = [torch.full((Lmax,), -1, dtype=torch.int32, device="cuda") for _ in range(2)]
+        uos = [c.empty(wl.T + 1, torch.int32) for _ in range(2)]
+        gr = torch.zeros((Lmax, wl.D), dtype=torch.float32, device="cuda")
+        codes = torch.zeros((Lmax, wl.D), dtype=torch.int8, device="cuda")
+        gs = c.empty(wl.T, torch.float32)
+        dev = [(c.dev(i), c.dev(o), c.dev(g), len(i)) for i, o, g in batches]
+        torch.cuda.synchronize()
+        outs = []
+        if not held:
+            for i, o, g, L in dev:
+                c.ctx.train_step(d_tables, i, o, g, scales, c.bits, out, urs[0], uos[0], gr, codes, gs, wl.lr, B=wl.B, L=L)
+                outs.append(out.cpu().numpy().copy())
+        else:
+            main, side = torch.cuda.Stream(), torch.cuda.Stream()
+            c.ctx.sort_batch(dev[0][0], dev[0][1], urs[0], uos[0], B=wl.B, L=dev[0][3], ws=0, stream=main)
+            for k, (i, o, g, L) in enumerate(dev):
+                slot = k & 1
+                side.wait_stream(main)                      # workspace slot^1: its previous batch has trained
+                c.ctx.train_step_sorted(d_tables, i, o, g, scales, c.bits, out, urs[slot], uos[slot], gr, codes, gs,
+                                        wl.lr, B=wl.B, L=L, ws=slot, stream=main)
+                if k + 1 < steps:
+                    ni, no, _, nL = dev[k + 1]
+                    c.ctx.stream_wait_forward(side)
+                    c.ctx.sort_batch(ni, no, urs[slot ^ 1], uos[slot ^ 1], B=wl.B, L=nL, ws=slot ^ 1, stream=side)
+                main.wait_stream(side)
+                main.synchronize()
+                outs.append(out.cpu().numpy().copy())
+        torch.cuda.synchronize()
+        c.ctx.raise_on_device_error()
+        res.append((d_tables.cpu().numpy(), outs, gs.cpu().numpy()))
+    assert bit_equal(res[0][0], res[1][0])
+    assert bit_equal(res[0][2], res[1][2])
+    for a, b in zip(res[0][1], res[1][1]):
+        assert bit_equal(a, b)
+    c.ctx.close()
