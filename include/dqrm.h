@@ -175,9 +175,10 @@ int dqrm_train_step_sorted(dqrm_ctx *ctx, float *tables, const int32_t *indices,
 
 /* Makes `stream` wait until the forward of the last dqrm_train_step_sorted enqueued on this
  * context has finished (no counterpart in the paper).  For the pipelined loop above: the sort of
- * batch k+1 shares the SMs with whatever runs beside it, and the forward is the one kernel of the
- * step that is bound by instruction issue, so a loop may hold the sort back until batch k's
- * forward is done and let it run beside the gradient summation and the update instead:
+ * batch k+1 shares the SMs with whatever runs beside it, so a loop may hold the sort back until
+ * batch k's forward is done and let it run beside the gradient summation and the update instead
+ * (whether that pays depends on the shapes: it helped 64-byte rows and hurt 256-byte rows when
+ * measured on a B200):
  *   dqrm_train_step_sorted(batch k, stream A); dqrm_stream_wait_forward(ctx, stream B);
  *   dqrm_sort_batch(batch k+1, stream B).
  * Before the first dqrm_train_step_sorted the wait returns at once.  Inside a stream capture both
