@@ -191,9 +191,15 @@ size_t dqrm_host_step_workspace_bytes(const dqrm_ctx *ctx, int64_t max_lookups, 
 
 /* dqrm_train_step for callers whose batch lives in HOST memory: copies h_indices [L],
  * h_offsets [T*B+1] and h_grad_out [B][T][D] to the device, runs the step, and copies
- * the pooled output back to h_out [B][T][D]; all on `stream`, asynchronously when the
- * host buffers are pinned.  tables, scales and bits stay on the device.  The sparse
- * gradient (unique rows, codes, scales) stays in the workspace. */
+ * the pooled output back to h_out [B][T][D]; asynchronously when the host buffers are
+ * pinned.  The call is ordered on `stream`: it starts behind the work already on `stream`,
+ * and work put on `stream` afterwards starts once the step and both copies are complete.
+ * Inside the call the upstream gradient comes in and the pooled output goes out on two
+ * streams owned by the context, beside the index sort and the forward (the two transfers
+ * run in opposite directions); with dqrm_set_overlap(ctx, 0) everything stays on `stream`.
+ * tables, scales and bits stay on the device.  The sparse gradient (unique rows, codes,
+ * scales) stays in the workspace.  h_grad_out and h_out must stay valid and untouched
+ * until the call's work on `stream` is complete. */
 int dqrm_train_step_host(dqrm_ctx *ctx, float *tables, const int32_t *h_indices,
                          const int32_t *h_offsets, const float *h_grad_out,
                          const float *scales, const int32_t *bits, float *h_out,

@@ -82,6 +82,12 @@ int dqrm_create(dqrm_ctx **out, int T, int D, const int64_t *h_row_off)
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fwd, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->copy_in, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->copy_out, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_h_start, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_h_go, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_h_fwd, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_h_out, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaMemcpy(ctx->d_row_off, h_row_off, sizeof(int64_t) * (T + 1), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(ctx->d_done, 0, sizeof(u32));
@@ -106,6 +112,12 @@ int dqrm_destroy(dqrm_ctx *ctx)
     if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
     if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
     if (ctx->ev_fwd) cudaEventDestroy(ctx->ev_fwd);
+    if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
+    if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
+    if (ctx->ev_h_start) cudaEventDestroy(ctx->ev_h_start);
+    if (ctx->ev_h_go) cudaEventDestroy(ctx->ev_h_go);
+    if (ctx->ev_h_fwd) cudaEventDestroy(ctx->ev_h_fwd);
+    if (ctx->ev_h_out) cudaEventDestroy(ctx->ev_h_out);
     if (ctx->prof_events) {
         for (int i = 0; i < DQ_PROF_MAX; ++i) cudaEventDestroy(ctx->prof_events[i]);
         delete[] ctx->prof_events;
@@ -437,18 +449,53 @@ int dqrm_train_step_host(dqrm_ctx *ctx, float *tables, const int32_t *h_indices,
     int32_t *d_off = reinterpret_cast<int32_t *>(ws + y.offsets);
     float *d_go = reinterpret_cast<float *>(ws + y.grad_out);
     float *d_out = reinterpret_cast<float *>(ws + y.out);
-    if (L > 0) DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(d_idx, h_indices, sizeof(int32_t) * L, cudaMemcpyHostToDevice, st));
+    int32_t *d_ur = reinterpret_cast<int32_t *>(ws + y.unique_rows);
+    int32_t *d_uo = reinterpret_cast<int32_t *>(ws + y.uniq_off);
+    float *d_gr = reinterpret_cast<float *>(ws + y.grad_rows);
+    int8_t *d_codes = reinterpret_cast<int8_t *>(ws + y.codes);
+    float *d_gs = reinterpret_cast<float *>(ws + y.grad_scales);
+    const size_t go_bytes = sizeof(float) * G * ctx->D;
+    if (!ctx->overlap || ctx->prof_on || L == 0) {
+        // everything in order on the caller's stream
+        if (L > 0) DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(d_idx, h_indices, sizeof(int32_t) * L, cudaMemcpyHostToDevice, st));
+        DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(d_off, h_offsets, sizeof(int32_t) * (G + 1), cudaMemcpyHostToDevice, st));
+        DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(d_go, h_grad_out, go_bytes, cudaMemcpyHostToDevice, st));
+        int rc = dqrm_train_step(ctx, tables, d_idx, d_off, d_go, scales, bits, d_out, d_ur, d_uo, d_gr, d_codes, d_gs, lr, B,
+                                 L, ws + y.step_ws, workspace_bytes - y.step_ws, stream);
+        if (rc != DQRM_OK) return rc;
+        DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(h_out, d_out, go_bytes, cudaMemcpyDeviceToHost, st));
+        return DQRM_OK;
+    }
+    // The two large transfers go in opposite directions and neither is needed where the other is: the upstream
+    // gradient (host to device) is first read by the gradient summation, the pooled output (device to host) is
+    // complete once the forward is.  Each gets a stream of the context, so that they overlap each other, the index
+    // sort and the forward; the caller's stream waits for both before the call's work on it is complete.
+    DQRM_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_h_start, st));          // the staging buffers' previous users are done
+    DQRM_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->copy_in, ctx->ev_h_start, 0));
+    DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(d_go, h_grad_out, go_bytes, cudaMemcpyHostToDevice, ctx->copy_in));
+    DQRM_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_h_go, ctx->copy_in));
+    DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(d_idx, h_indices, sizeof(int32_t) * L, cudaMemcpyHostToDevice, st));
     DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(d_off, h_offsets, sizeof(int32_t) * (G + 1), cudaMemcpyHostToDevice, st));
-    DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(d_go, h_grad_out, sizeof(float) * G * ctx->D, cudaMemcpyHostToDevice, st));
-    int rc = dqrm_train_step(ctx, tables, d_idx, d_off, d_go, scales, bits, d_out,
-                             reinterpret_cast<int32_t *>(ws + y.unique_rows),
-                             reinterpret_cast<int32_t *>(ws + y.uniq_off),
-                             reinterpret_cast<float *>(ws + y.grad_rows),
-                             reinterpret_cast<int8_t *>(ws + y.codes),
-                             reinterpret_cast<float *>(ws + y.grad_scales), lr, B, L,
-                             ws + y.step_ws, workspace_bytes - y.step_ws, stream);
+    DQRM_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_fork, st));
+    DQRM_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
+    char *step_ws = ws + y.step_ws;
+    const size_t step_ws_bytes = workspace_bytes - y.step_ws;
+    const u32 *absmax = nullptr;
+    int rc = dq_launch_bwd_sort(ctx, d_idx, d_off, d_ur, d_uo, B, L, step_ws, step_ws_bytes, ctx->side, &absmax);
+    if (rc == DQRM_OK) rc = dq_launch_fwd(ctx, tables, d_idx, d_off, scales, bits, d_out, nullptr, B, L, st);
+    // join every stream even after an error, so that the caller's stream stays ordered behind them
+    cudaEventRecord(ctx->ev_h_fwd, st);
+    cudaStreamWaitEvent(ctx->copy_out, ctx->ev_h_fwd, 0);
+    if (rc == DQRM_OK) cudaMemcpyAsync(h_out, d_out, go_bytes, cudaMemcpyDeviceToHost, ctx->copy_out);
+    cudaEventRecord(ctx->ev_h_out, ctx->copy_out);
+    cudaEventRecord(ctx->ev_join, ctx->side);
+    cudaStreamWaitEvent(st, ctx->ev_join, 0);
+    cudaStreamWaitEvent(st, ctx->ev_h_go, 0);
+    if (rc == DQRM_OK) rc = dq_launch_bwd_reduce(ctx, d_go, d_uo, d_gr, B, L, step_ws, step_ws_bytes, st);
+    if (rc == DQRM_OK) rc = dq_launch_quant_update(ctx, tables, d_ur, d_uo, d_gr, absmax, d_codes, d_gs, lr, st);
+    cudaStreamWaitEvent(st, ctx->ev_h_out, 0);
     if (rc != DQRM_OK) return rc;
-    DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(h_out, d_out, sizeof(float) * G * ctx->D, cudaMemcpyDeviceToHost, st));
+    DQRM_CUDA_TRY(ctx, cudaGetLastError());
     return DQRM_OK;
 }
 

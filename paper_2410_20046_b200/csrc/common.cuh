@@ -23,6 +23,9 @@ struct dqrm_ctx {
     cudaStream_t side = nullptr;    // second stream: a training step sorts the indices beside its forward
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     cudaEvent_t ev_fwd = nullptr;   // recorded behind the forward of the last training step enqueued
+    // host-buffer step: the upstream gradient comes in and the pooled output goes out on streams of their own
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    cudaEvent_t ev_h_start = nullptr, ev_h_go = nullptr, ev_h_fwd = nullptr, ev_h_out = nullptr;
     int overlap = 1;                // 0: keep everything on the caller's stream
     int payload_position = 0;       // sort payload: 0 = row of grad_out, 1 = position of the lookup (set by the merge)
     // launch accounting and optional per-launch timing (see dqrm_profile_*)
