@@ -15,14 +15,19 @@
  *   - Appendix B.1: the local step uses the dequantised gradient; Section 3.1: the FP32
  *     master copy is what is updated                            -> dqrm_row_update
  *
- * Quantiser (the paper prints no formula; Section 4.1 fixes "one scale per table",
- * Appendix A "uniform mapping" and "static min-max clipping range"):
+ * Quantiser (the paper prints no formula; Section 4.1 gives every table a single scale,
+ * Appendix A describes a uniform quantiser whose clipping range is the table's fixed
+ * minimum and maximum):
  *     n(b) = 2^(b-1) - 1
  *     scale(absmax, b) = max(absmax, 1e-8f) / (float)n(b)                 one FP32 divide
  *     Q(x; s, b) = clamp(round_half_even(x / s), -2^(b-1), 2^(b-1) - 1)   one FP32 divide
  *     DQ(q; s)   = (float)q * s                                           one FP32 multiply
- * Every FP32 operation is a single IEEE round-to-nearest operation (no reciprocal
- * shortcuts, no fused multiply-add where two roundings are specified).
+ * These are the results every call reproduces bit for bit: each FP32 operation above is a
+ * single IEEE round-to-nearest operation, and no fused multiply-add stands where two
+ * roundings are specified.  Where one scale serves many elements the kernels reach the
+ * same codes through a reciprocal multiply that is provably equal away from rounding
+ * ties and redo the rare element near a tie with the IEEE division (see
+ * dqrm_selfcheck_quantizer).
  *
  * Conventions
  *   - All array arguments are DEVICE pointers unless the name starts with h_ (host).

@@ -10,8 +10,8 @@
  *
  * The paper states the method in prose and prints no formula for its
  * quantiser.  What it fixes: one FP32 scale per table (Section 4.1), a uniform
- * mapping with a static min-max clipping range (Appendix A, "Prior QAT
- * Techniques on DLRM"), a scale found by traversing the whole table and
+ * quantiser clipped to the table's fixed minimum and maximum (Appendix A, the
+ * part on earlier QAT techniques), a scale found by traversing the whole table and
  * refreshed only periodically (Section 3.2), quantisation applied to the rows
  * a batch actually gathers (Section 3.1, Figure 2(b)), embedding gradients
  * kept as sparse (indices, values) whose values alone are quantised to INT8

@@ -323,8 +323,11 @@ seg_emit_kernel(const u32 *__restrict__ keys, int64_t L, const u32 *__restrict__
                 const u32 u = heads_before;
                 heads_before += 1;
                 seg_start[u] = (u32)i;
-                while ((int64_t)k[e] >= s_off[t + 1]) ++t;        // ends: every key lies below s_off[T]
-                unique_rows[u] = (int32_t)((int64_t)k[e] - s_off[t]);
+                // a sort that refused a table leaves that table's keys undefined: keep them inside the arena and
+                // the walk inside the offset list, whatever they hold
+                const int64_t key = min((int64_t)k[e], s_off[T] - 1);
+                while (t < T - 1 && key >= s_off[t + 1]) ++t;
+                unique_rows[u] = (int32_t)max((int64_t)0, key - s_off[t]);
                 for (int tt = t_prev + 1; tt <= t; ++tt) uniq_off[tt] = (int32_t)u;
                 t_prev = t;
             }
@@ -374,7 +377,7 @@ int launch_reduce(dqrm_ctx *ctx, const Layout &y, char *ws, const u32 *keys, con
     int fgrid = (int)(fblocks < (int64_t)ctx->num_sms * 4 ? (fblocks < 1 ? 1 : fblocks) : (int64_t)ctx->num_sms * 4);
     const size_t fix_smem = (size_t)(256 / LPR) * ctx->D * sizeof(double) + smem;
     if (fix_smem > 48 * 1024) {
-        static bool raised = false;
+        bool &raised = ctx->smem_raised[dq_smem_slot_fixup(LPR, CH)];
         if (!raised) {
             DQRM_CUDA_TRY(ctx, cudaFuncSetAttribute(seg_fixup_kernel<LPR, CH>,
                                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fix_smem));
@@ -447,7 +450,7 @@ int dq_launch_bwd_sort(dqrm_ctx *ctx, const int32_t *indices, const int32_t *off
         ca.payload_position = ctx->payload_position;
         ca.tile_heads = reinterpret_cast<u32 *>(ws + y.tile_heads);
         const size_t smem = csort::smem_bytes(ca.cap);
-        static bool raised = false;
+        bool &raised = ctx->smem_raised[DQ_SMEM_SLOT_CSORT];
         cudaError_t e = cudaSuccess;
         if (!raised) {
             e = cudaFuncSetAttribute(csort::cluster_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -17,10 +17,6 @@
 #include <cooperative_groups.h>
 #include "common.cuh"
 
-// phase time stamps for bench-top studies of this kernel; compiled out in the library
-#ifndef CSORT_TS
-#define CSORT_TS(i)
-#endif
 
 namespace csort {
 
@@ -99,27 +95,34 @@ cluster_sort_kernel(const Args a)
     } else {
         pb0 = a.gp[0] + tb0 + (int64_t)c * npc; pb1 = a.gp[1] + tb0 + (int64_t)c * npc;
     }
-
-    CSORT_TS(0)
     // ---- are this table's bags all one-index bags in order (offsets = identity)? ----
+    // Any other batch has its offsets checked here: they must not decrease inside the table, so that
+    // the search for a lookup's bag below walks an ordered list.
     {
         if (threadIdx.x == 0) s_flag = 1;
         __syncthreads();
         int ok = 1;
         const int per = (a.B + CLUSTER - 1) / CLUSTER;
         const int b0 = c * per, b1 = min(a.B, b0 + per);
-        if (n != a.B) ok = 0;
-        else
+        const int32_t *off_t = a.offsets + (int64_t)t * a.B;
+        if (n != a.B) {
+            ok = 0;
+            bool dec = false;
+            for (int i = b0 + threadIdx.x; i < b1; i += THREADS) dec |= __ldg(off_t + i) > __ldg(off_t + i + 1);
+            if (dec) dq_report(a.status, DQRM_ERR_INDEX_RANGE);
+        } else {
             for (int i = b0 + threadIdx.x; i < b1; i += THREADS)
-                if ((int64_t)__ldg(a.offsets + (int64_t)t * a.B + i) != tb0 + i) ok = 0;
+                if ((int64_t)__ldg(off_t + i) != tb0 + i) ok = 0;
+        }
         if (!ok) s_flag = 0;
+        if (blockIdx.x == 0 && threadIdx.x == 0 &&
+            (__ldg(a.offsets) != 0 || (int64_t)__ldg(a.offsets + (int64_t)a.T * a.B) != a.L))
+            dq_report(a.status, DQRM_ERR_INDEX_RANGE);
         __syncthreads();
     }
     cluster.sync();
     bool onehot = true;
     for (unsigned cc = 0; cc < CLUSTER; ++cc) onehot &= (*cluster.map_shared_rank(&s_flag, cc) != 0);
-
-    CSORT_TS(1)
     // ---- load this block's slice: key = row within the table, payload = row of grad_out ----
     bool bad = false;
     for (int i = threadIdx.x; i < my_n; i += THREADS) {
@@ -150,7 +153,9 @@ cluster_sort_kernel(const Args a)
 
     int s = 0;
     __syncthreads();
-    CSORT_TS(2)
+    // a one-row table takes no pass, so no cluster barrier separates the loads above from the
+    // neighbour's read of this slice's last pair in the write-out below
+    if (passes == 0) cluster.sync();
     for (int pass = 0; pass < passes; ++pass) {
         const int shift = 8 * pass;
         const uint2 *src = s ? pb1 : pb0;                           // this pass reads stage s ...
@@ -158,11 +163,9 @@ cluster_sort_kernel(const Args a)
         uint2 *gdst = s ? a.gp[0] : a.gp[1];
         for (int i = threadIdx.x; i < WARPS * BINS; i += THREADS) (&s_cnt[0][0])[i] = 0u;
         __syncthreads();
-        CSORT_TS(3 + 6 * pass)
         // phase 1: digit counts of this warp's part
         for (int i = w0 + lane; i < w1; i += 32) atomicAdd(&s_cnt[warp][(src[i].x >> shift) & 255u], 1u);
         __syncthreads();
-        CSORT_TS(4 + 6 * pass)
         if (threadIdx.x < BINS) {
             u32 h = 0;
 #pragma unroll 8
@@ -170,7 +173,6 @@ cluster_sort_kernel(const Args a)
             s_hist[threadIdx.x] = h;
         }
         cluster.sync();
-        CSORT_TS(5 + 6 * pass)
         // offsets: digits first, then blocks of the cluster, then warps of this block
         u32 tot = 0, pre = 0, incl = 0;
         if (threadIdx.x < BINS) {                  // one thread per digit (the first BINS / 32 warps)
@@ -200,7 +202,6 @@ cluster_sort_kernel(const Args a)
             }
         }
         __syncthreads();
-        CSORT_TS(6 + 6 * pass)
         // phase 2: rank again and scatter into the owners' buffers of the other stage
         for (int i0 = w0; i0 < w1; i0 += 32) {
             const int i = i0 + lane;
@@ -227,12 +228,9 @@ cluster_sort_kernel(const Args a)
                 }
             }
         }
-        CSORT_TS(7 + 6 * pass)
         cluster.sync();
-        CSORT_TS(8 + 6 * pass)
         s ^= 1;
     }
-    CSORT_TS(30)
     // ---- write the sorted slice: arena row keys ----
     // and count, per 2048-entry tile of the sorted order, the entries that start a new row
     {
@@ -265,7 +263,6 @@ cluster_sort_kernel(const Args a)
             }
         }
     }
-    CSORT_TS(31)
     cluster.sync();      // nobody leaves while its shared memory may still be read or written
 }
 

@@ -28,6 +28,9 @@ struct dqrm_ctx {
     cudaEvent_t ev_h_start = nullptr, ev_h_go = nullptr, ev_h_fwd = nullptr, ev_h_out = nullptr;
     int overlap = 1;                // 0: keep everything on the caller's stream
     int payload_position = 0;       // sort payload: 0 = row of grad_out, 1 = position of the lookup (set by the merge)
+    // kernels whose dynamic shared-memory limit has been raised on this context's device (the attribute is
+    // per device, so the record lives here and not in a process-wide flag)
+    bool smem_raised[32] = {};
     // launch accounting and optional per-launch timing (see dqrm_profile_*)
     int64_t launch_count = 0;
     int prof_on = 0, prof_n = 0;
@@ -64,6 +67,11 @@ static inline void dq_mark(dqrm_ctx *ctx, cudaStream_t st, int kernel_id)
     } while (0)
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// slots of dqrm_ctx::smem_raised
+constexpr int DQ_SMEM_SLOT_CSORT = 24;
+constexpr int dq_log2c(int x) { return x <= 1 ? 0 : 1 + dq_log2c(x / 2); }
+constexpr int dq_smem_slot_fixup(int lpr, int ch) { return dq_log2c(lpr) * 4 + dq_log2c(ch); }
 
 // ---------------------------------------------------------------------------------
 // quantiser arithmetic: each operation is one IEEE round-to-nearest FP32 operation

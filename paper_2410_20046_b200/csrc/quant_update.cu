@@ -8,6 +8,7 @@
 // A group of LPR lanes owns a contiguous range of unique rows and keeps a few of them in flight;
 // rows are distinct, so the read-modify-write of the master rows needs no atomics.  All
 // streams are 128-bit per lane.
+#include <mutex>
 #include "common.cuh"
 
 namespace {
@@ -77,7 +78,8 @@ __global__ void __launch_bounds__(QU_THREADS)
 row_stream_kernel(float *__restrict__ tables, const int64_t *__restrict__ row_off,
                   const int32_t *__restrict__ unique_rows, const int32_t *__restrict__ uniq_off,
                   const float *__restrict__ grad_rows, const u32 *__restrict__ absmax,
-                  int8_t *__restrict__ codes, float *__restrict__ grad_scales, float lr, int T, int D_any)
+                  int8_t *__restrict__ codes, float *__restrict__ grad_scales, float lr, int T, int D_any,
+                  int *__restrict__ status)
 {
     constexpr int NB = RowsInFlight<CH>::v;
     const int D = EXACT ? 4 * LPR * CH : D_any;
@@ -102,14 +104,15 @@ row_stream_kernel(float *__restrict__ tables, const int64_t *__restrict__ row_of
     if (per < NB) per = NB;             // few rows: fewer groups, each with a full set of rows in flight
     const int64_t u_begin = group * per, u_end = min(U, u_begin + per);
     int cur_t = -1;
-    int64_t cur_end = -1, r0 = 0;
+    int64_t cur_end = -1, r0 = 0, nrows = 1;
+    bool bad = false;
     float s = 1.f;
     QuantScale qs = dq_make_scale(1.f, 8);
     for (int64_t u = u_begin; u < u_end;) {
         if (u >= cur_end) {
             cur_t = table_of_row(s_uoff, T, u);
             cur_end = s_uoff[cur_t + 1];
-            if (MODE != MODE_QUANT) r0 = __ldg(row_off + cur_t);
+            if (MODE != MODE_QUANT) { r0 = __ldg(row_off + cur_t); nrows = __ldg(row_off + cur_t + 1) - r0; }
             s = s_scale[cur_t];
             qs = dq_make_scale(s, 8);
         }
@@ -121,8 +124,12 @@ row_stream_kernel(float *__restrict__ tables, const int64_t *__restrict__ row_of
 #pragma unroll
         for (int b = 0; b < NB; ++b) {
             wrow[b] = nullptr;
-            if (b < nb && MODE != MODE_QUANT)
-                wrow[b] = reinterpret_cast<float4 *>(tables + (r0 + __ldg(unique_rows + u + b)) * D);
+            if (b < nb && MODE != MODE_QUANT) {
+                // a row number outside its table is reported and kept inside the arena, never followed
+                int64_t row = __ldg(unique_rows + u + b);
+                if (row < 0 || row >= nrows) { bad = true; row = row < 0 ? 0 : nrows - 1; }
+                wrow[b] = reinterpret_cast<float4 *>(tables + (r0 + row) * D);
+            }
         }
 #pragma unroll
         for (int b = 0; b < NB; ++b) {
@@ -169,6 +176,7 @@ row_stream_kernel(float *__restrict__ tables, const int64_t *__restrict__ row_of
         }
         u += nb;
     }
+    if (MODE != MODE_QUANT && bad) dq_report(status, DQRM_ERR_INDEX_RANGE);
 }
 
 template <int MODE, int LPR, int CH>
@@ -180,10 +188,12 @@ int launch_rows(dqrm_ctx *ctx, float *tables, const int32_t *unique_rows, const 
     int grid = ctx->num_sms * 8;      // U lives on the device: a fixed grid splits the rows evenly
     if (ctx->D == 4 * LPR * CH)
         row_stream_kernel<MODE, LPR, CH, true><<<grid, QU_THREADS, smem, st>>>(
-            tables, ctx->d_row_off, unique_rows, uniq_off, grad_rows, absmax, codes, grad_scales, lr, ctx->T, ctx->D);
+            tables, ctx->d_row_off, unique_rows, uniq_off, grad_rows, absmax, codes, grad_scales, lr, ctx->T, ctx->D,
+            ctx->d_status);
     else
         row_stream_kernel<MODE, LPR, CH, false><<<grid, QU_THREADS, smem, st>>>(
-            tables, ctx->d_row_off, unique_rows, uniq_off, grad_rows, absmax, codes, grad_scales, lr, ctx->T, ctx->D);
+            tables, ctx->d_row_off, unique_rows, uniq_off, grad_rows, absmax, codes, grad_scales, lr, ctx->T, ctx->D,
+            ctx->d_status);
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
     dq_mark(ctx, st, MODE == MODE_QUANT ? DQ_K_QUANT : (MODE == MODE_UPDATE ? DQ_K_UPDATE : DQ_K_QUANT_UPDATE));
     return DQRM_OK;
@@ -289,6 +299,7 @@ struct StaticSlot {
     bool ready = false;
 };
 StaticSlot g_static_slots[STATIC_MAX_DEVICES];
+std::mutex g_static_mutex;        // host threads may make a device's first call at the same time
 
 }  // namespace
 
@@ -303,17 +314,22 @@ extern "C" int dqrm_grad_quant_int8_static(int T, int D, const float *grad_rows,
         (void)cudaGetLastError();
         return DQRM_ERR_CUDA;
     }
-    StaticSlot &slot = g_static_slots[dev];
-    if (!slot.ready) {
-        // first call on this device: resolve the array's device address (with this device current)
-        u32 *p = nullptr;
-        if (cudaGetSymbolAddress(reinterpret_cast<void **>(&p), g_static_absmax) != cudaSuccess || !p ||
-            cudaDeviceGetAttribute(&slot.num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
-            (void)cudaGetLastError();
-            return DQRM_ERR_CUDA;
+    StaticSlot slot;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        StaticSlot &shared = g_static_slots[dev];
+        if (!shared.ready) {
+            // first call on this device: resolve the array's device address (with this device current)
+            u32 *p = nullptr;
+            if (cudaGetSymbolAddress(reinterpret_cast<void **>(&p), g_static_absmax) != cudaSuccess || !p ||
+                cudaDeviceGetAttribute(&shared.num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+                (void)cudaGetLastError();
+                return DQRM_ERR_CUDA;
+            }
+            shared.absmax = p;
+            shared.ready = true;
         }
-        slot.absmax = p;
-        slot.ready = true;
+        slot = shared;
     }
     // a stack context carries the shape to the shared launch helpers; nothing is allocated
     dqrm_ctx tmp;

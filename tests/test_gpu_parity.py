@@ -34,6 +34,9 @@ def _cases():
         "odd_d20": replace(W.scaled_down(kg, total_rows=50_000, B=333), D=20, name="odd_d20"),
         "wide_d384": W.Workload("wide_d384", (700, 90, 5000), D=384, B=257, alpha=1.1, bits=8),
         "one_row_tables": W.Workload("one_row_tables", (1, 1, 7, 1), D=16, B=100, alpha=1.05, bits=4),
+        # a one-row table whose 6000 lookups span all blocks of its sort cluster and three 2048-entry tiles,
+        # with other tables behind it (their unique rows must not shift)
+        "one_row_wide": W.Workload("one_row_wide", (1, 3000, 1, 50), D=16, B=6000, alpha=1.05, bits=4),
     }
 
 
@@ -293,6 +296,31 @@ def test_out_of_range_index_is_reported_not_trapped(oracle):
     # the context is still usable and correct
     out, _ = c.gpu_fwd(c.dev(tables), idx, off, c.dev(o_scales), want_codes=False)
     assert bit_equal(out, oracle.emb_fwd(tables, c.row_off, wl.D, wl.B, idx, off, o_scales, c.bits_np))
+    c.ctx.close()
+
+
+@pytest.mark.parametrize("sort_path", [0, 1])
+def test_decreasing_offsets_are_reported_not_followed(oracle, sort_path):
+    """Offsets that decrease inside a table are an error the device reports; nothing is read or written
+    out of bounds and the context stays usable."""
+    import paper_2410_20046_b200 as dq
+
+    wl = W.Workload("mini_bags", (50, 7, 300), D=16, B=64, alpha=1.1, bits=4, bag_mean=3.0, bag_max=6)
+    c = Case(wl)
+    idx, off, go = c.batch(0)
+    bad = off.copy()
+    g = wl.B + 5                                  # a bag inside table 1
+    bad[g], bad[g + 1] = off[g + 1], off[g]       # (only a decrease when that bag is not empty)
+    assert bad[g] > bad[g + 1]
+    c.ctx.set_sort_path(sort_path)
+    with pytest.raises(dq.DqrmError) as e:
+        c.gpu_bwd(idx, bad, go)
+    assert e.value.status == dq.ERR_INDEX_RANGE
+    assert c.ctx.check_status() == dq.OK
+    ur, uo, gr = c.gpu_bwd(idx, off, go)          # still usable and correct
+    o_ur, o_uo, o_gr = oracle.emb_bwd(go, wl.T, wl.D, wl.B, idx, off)
+    assert bit_equal(ur, o_ur) and bit_equal(uo, o_uo)
+    assert_close_fp32(gr, o_gr)
     c.ctx.close()
 
 

@@ -4,8 +4,9 @@ It exists for callers that cannot allocate device memory where they quantise (a 
 inside a framework that already owns the GPU's memory, or a loop that cannot take the
 device-wide stall of cudaMalloc/cudaFree), so it has neither context nor workspace: its
 scratch is a fixed array inside the library.  This file checks, through the C ABI, that
-it gives the same scales and codes as `dqrm_grad_quant_int8` on two calls in a row (the
-second with much smaller gradients, so maxima left over from the first call would show),
+it gives the same scales and codes as `dqrm_grad_quant_int8`, and as the CPU oracle's
+quantiser, on two calls in a row (the second with much smaller gradients, so maxima left
+over from the first call would show),
 and that a table count beyond the built-in limit is refused without launching anything.
 It is collected last on purpose: a failure here leaves every other test already run.
 """
@@ -27,6 +28,7 @@ def _sparse_grads(wl, step, scale):
 
 
 def test_static_quantiser_matches_workspace_quantiser_twice_in_a_row():
+    import oracle
     import torch
     import paper_2410_20046_b200 as dq
 
@@ -50,6 +52,10 @@ def test_static_quantiser_matches_workspace_quantiser_twice_in_a_row():
         # integer codes and scales are compared bit for bit, as everywhere in this suite
         assert scales.cpu().numpy().tobytes() == ref_scales.cpu().numpy().tobytes(), f"call {call}: scales"
         assert torch.equal(codes, ref_codes), f"call {call}: codes"
+        # ... and with the oracle's quantiser on the same host arrays
+        o_codes, o_scales = oracle.grad_quant_int8(grad_rows, uniq_off, wl.D)
+        assert scales.cpu().numpy().tobytes() == o_scales.tobytes(), f"call {call}: scales vs oracle"
+        assert codes.cpu().numpy().tobytes() == o_codes.tobytes(), f"call {call}: codes vs oracle"
         assert int(codes.abs().max()) == 127
     ctx.close()
 
