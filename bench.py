@@ -8,6 +8,9 @@ Prints ONE JSON line.  `value` is whole-job lookups/s with inputs resident in HB
 `e2e` the same through the host-buffer entry point (copies inside the timed region),
 `roofline` the dominant kernel against the measured HBM copy rate, `cpu_baseline` the
 CPU oracle timed on the host cores.  With --impl reference the oracle itself is timed.
+The default run (N = 1, workload kaggle_b16384) also measures terabyte_b32768 in the same
+process and carries it in the line's `also` block.  With --gpus N > 1 and no launcher in
+the environment the script starts N ranks itself (one process per GPU, torchrun).
 By default consecutive steps are software-pipelined: the index sort of batch k+1 runs on a
 second stream while batch k trains (--no-pipeline: one call per step).  --packed times the
 bit-packed export and the packed inference lookup instead of the training step.
@@ -107,13 +110,24 @@ class ClockSampler:
 
 
 def algorithmic_bytes(wl, L, G, U):
-    """Bytes the method must move per call (each touched row once)."""
+    """Bytes the method must move per call (each touched row once).  `step` counts what the calls of
+    the fused step move; `step_separate_calls` adds the D*U bytes of INT8 codes that a separate update
+    call reads back (8L + 8G + 8DG + U(8 + 22D))."""
     D = wl.D
     fwd = 4 * L + 4 * G + 4 * D * U + 4 * D * G
     bwd = 4 * D * G + 4 * L + 4 * G + 4 * U + 4 * D * U
     qu = 4 * D * U + D * U + 4 * U + 8 * D * U          # read grads, write codes, read rows, RMW rows
     return {"fwd": fwd, "bwd": bwd, "quant_update": qu, "step": fwd + bwd + qu,
+            "step_separate_calls": 8 * L + 8 * G + 8 * D * G + U * (8 + 22 * D),
             "refresh": wl.table_bytes()}
+
+
+def base_config(wl):
+    """The workload, in the same words for both arms."""
+    return {"workload": wl.name, "tables": wl.T, "dim": wl.D, "batch_per_gpu": wl.B, "bits": wl.bits, "grad_bits": 8,
+            "refresh_period": wl.period, "table_bytes": wl.table_bytes(),
+            "inputs": f"seeded synthetic batches, distinct per step and cycled ({N_BATCHES} on the GPU arm, 4 on the "
+                      "CPU arm); one batch's rows, gradients and outputs plus the tables exceed the 126 MB L2"}
 
 
 # kernel -> which algorithmic byte count bounds it (the sort kernels carry no algorithmic
@@ -121,30 +135,31 @@ def algorithmic_bytes(wl, L, G, U):
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (set an entry to None when its kernel has changed since the capture)
 NCU_TRAFFIC = {
-    ("kaggle_b16384", "seg_reduce_kernel"): 31.11e6,
-    ("kaggle_b16384", "fwd_kernel"): 26.35e6,
-    ("kaggle_b16384", "row_stream_kernel<fused>"): 25.18e6,
-    # the Terabyte-shaped step captured over 2 GB of tables (the full tables are too large for a counter capture)
-    ("terabyte_2gb_b32768", "seg_reduce_kernel"): 274.15e6,
-    ("terabyte_2gb_b32768", "fwd_kernel"): 211.26e6,
-    ("terabyte_2gb_b32768", "row_stream_kernel<fused>"): 80.37e6,
-    # ... and scaled to the full tables by the reduce's algorithmic bytes (265.79 MB against 254.88 MB per launch):
-    # its traffic is the upstream-gradient rows (the same) plus the unique rows it writes
-    ("terabyte_b32768", "seg_reduce_kernel"): 285.9e6,
 }
 
 KERNEL_BYTES = {
     "fwd_kernel": lambda ab, wl, L, G, U: ab["fwd"],
     "seg_reduce_kernel": lambda ab, wl, L, G, U: 4 * wl.D * G + 4 * wl.D * U,
     "row_stream_kernel<fused>": lambda ab, wl, L, G, U: ab["quant_update"],
+    "step_tail_kernel": lambda ab, wl, L, G, U: ab["quant_update"],
     "refresh_kernel": lambda ab, wl, L, G, U: ab["refresh"],
 }
 
 
+def host_cores():
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
 def oracle_sample(wl, tables_h, n_steps, period):
-    """Times the CPU oracle, as it stands, on `n_steps` full batches and one refresh."""
+    """Times the CPU oracle, as it stands, on `n_steps` full batches and one refresh: on one host core,
+    and on all cores of the affinity mask with one table per thread (tables are independent, so the
+    results are the same bits; a single table splits nothing)."""
     import numpy as np
     import oracle
+    from concurrent.futures import ThreadPoolExecutor
     from dqrm_inputs import workloads as W
 
     off = wl.row_off()
@@ -153,16 +168,47 @@ def oracle_sample(wl, tables_h, n_steps, period):
     t0 = time.perf_counter()
     scales, _ = oracle.scale_refresh(tables_h, off, wl.D, bits)
     t_refresh = time.perf_counter() - t0
+    batches = [(*W.make_batch(wl, s, samplers), W.grad_out_np(wl, s)) for s in range(n_steps)]
     t_steps, lookups = 0.0, 0
-    for s in range(n_steps):
-        idx, offs = W.make_batch(wl, s, samplers)
-        go = W.grad_out_np(wl, s)
+    for idx, offs, go in batches:
         t0 = time.perf_counter()
         oracle.train_step(tables_h, off, wl.D, wl.B, idx, offs, go, scales, bits, wl.lr)
         t_steps += time.perf_counter() - t0
         lookups += len(idx)
     per_step = t_steps / n_steps + t_refresh / period
-    return (lookups / n_steps) / per_step, t_steps / n_steps, t_refresh
+    one = ((lookups / n_steps) / per_step, t_steps / n_steps, t_refresh)
+
+    # all cores: the same calls on one-table problems, a thread each (the C calls release the interpreter lock)
+    cores = host_cores()
+    threads = max(1, min(cores, wl.T))
+    one_off = lambda t: np.array([0, off[t + 1] - off[t]], dtype=np.int64)
+
+    def table_refresh(t):
+        return oracle.scale_refresh(tables_h[off[t]:off[t + 1]], one_off(t), wl.D, bits[t:t + 1])
+
+    def table_step(job):
+        t, idx_t, offs_t, go_t = job
+        oracle.train_step(tables_h[off[t]:off[t + 1]], one_off(t), wl.D, wl.B, idx_t, offs_t, go_t, scales[t:t + 1],
+                          bits[t:t + 1], wl.lr)
+
+    with ThreadPoolExecutor(max_workers=threads) as pool:
+        t0 = time.perf_counter()
+        list(pool.map(table_refresh, range(wl.T)))
+        t_refresh_mc = time.perf_counter() - t0
+        t_steps_mc = 0.0
+        for idx, offs, go in batches:
+            jobs = []
+            for t in range(wl.T):                      # slicing the batch by table is the harness's work, not timed
+                lo, hi = offs[t * wl.B], offs[(t + 1) * wl.B]
+                jobs.append((t, np.ascontiguousarray(idx[lo:hi]),
+                             np.ascontiguousarray(offs[t * wl.B:(t + 1) * wl.B + 1] - lo),
+                             np.ascontiguousarray(go[:, t:t + 1, :])))
+            t0 = time.perf_counter()
+            list(pool.map(table_step, jobs))
+            t_steps_mc += time.perf_counter() - t0
+    per_step_mc = t_steps_mc / n_steps + t_refresh_mc / period
+    many = ((lookups / n_steps) / per_step_mc, t_steps_mc / n_steps, t_refresh_mc, threads, cores)
+    return one, many
 
 
 def host_tables(wl):
@@ -208,21 +254,17 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": wl.name, "tables": wl.T, "dim": wl.D, "batch": wl.B, "bits": wl.bits,
-                   "refresh_period": wl.period},
+        "config": base_config(wl),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
 
 def run_ours(args):
-    import numpy as np
     import torch
     import torch.distributed as dist
 
     import paper_2410_20046_b200 as dq
-    from dqrm_inputs import workloads as W
-    from paper_2410_20046_b200 import harness
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -237,11 +279,41 @@ def run_ours(args):
     if args.train_priority != 0:                     # the whole run, graph capture included, on a stream of that priority
         torch.cuda.set_stream(torch.cuda.Stream(priority=args.train_priority))
         capture_stream = torch.cuda.Stream(priority=args.train_priority)
+    where = (rank, world, local_rank, capture_stream)
 
-    wl = get_workload(args.workload)
+    line = measure(args, get_workload(args.workload), where, primary=True)
+    # the other target configuration, measured in the same process (single GPU, default workload only)
+    if world == 1 and args.workload == "kaggle_b16384" and not args.no_also:
+        import copy
+        a2 = copy.copy(args)
+        a2.steps = min(args.steps, 500)
+        import gc
+        gc.collect()
+        torch.cuda.empty_cache()                     # the first workload's tables and batches
+        other = measure(a2, get_workload("terabyte_b32768"), where, primary=False)
+        line["also"] = [{k: other[k] for k in ("value", "unit", "steps", "warmup", "ms_per_step", "config", "e2e",
+                                               "gpu_launches", "roofline", "step_roofline", "kernel_rooflines",
+                                               "kernels", "refresh")}]
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def measure(args, wl, where, primary):
+    """Times `args.steps` steps of workload `wl` on this rank's GPU and returns the JSON line as a dict."""
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    import paper_2410_20046_b200 as dq
+    from dqrm_inputs import workloads as W
+    from paper_2410_20046_b200 import harness
+
+    rank, world, local_rank, capture_stream = where
     G = wl.T * wl.B
     tables = W.tables_torch(wl, "cuda")
-    tables_h = tables.cpu().numpy() if (rank == 0 and world == 1 and not args.no_cpu_baseline) else None
+    tables_h = tables.cpu().numpy() if (primary and rank == 0 and world == 1 and not args.no_cpu_baseline) else None
 
     # every rank is a full replica that takes its own B samples (weak scaling, no exchange)
     samplers = W.make_samplers(wl)
@@ -364,11 +436,13 @@ def run_ours(args):
             torch.cuda.synchronize()
 
     last = {"s": None}
+    refreshes = {"n": 0}     # scale refreshes launched since the timed region began
 
     def step(s, end=None, direct=False):
         """Runs step s, or steps s .. s+spg-1 from one graph when they all lie before `end`; returns how many."""
         if s % wl.period == 0:
             ctx.scale_refresh(tables, bits, scales)
+            refreshes["n"] += 1
         if direct and pipelined:                     # the per-kernel timing pass: one stream, one call per step
             launch_unpipelined(s % N_BATCHES)
             last["s"] = None
@@ -409,6 +483,7 @@ def run_ours(args):
             sampler.start()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         n0 = ctx.launch_count()
+        refreshes["n"] = 0
         e0.record()
         while s < warmup + steps:                      # exactly `steps` steps: s never passes the end
             s += fn(s, warmup + steps)
@@ -423,7 +498,8 @@ def run_ours(args):
         return ms, clocks, launches
 
     warm = max(3, args.warmup)
-    ms, clocks, launches = timed(step, args.steps, warm, sample_clocks=True)
+    ms, clocks, launches = timed(step, args.steps, warm, sample_clocks=primary)
+    timed_refreshes = refreshes["n"]
     ctx.raise_on_device_error()
     lookups_per_step = Lavg * world
     value = harness.job_throughput(Lavg, world, args.steps, ms)
@@ -441,6 +517,7 @@ def run_ours(args):
         step(s)
     torch.cuda.synchronize()
     ctx.profile_begin()
+    ctx.scale_refresh(tables, bits, scales)          # one refresh is always among the profiled launches
     for s in range(prof_steps):
         step(warm + s, direct=True)
     prof = ctx.profile_end()
@@ -461,53 +538,77 @@ def run_ours(args):
             gbs = by / (prof[k][0] * 1e-3 / prof[k][1]) / 1e9
             per_kernel_roofline[k] = {"algorithmic_bytes": int(by), "GB/s": round(gbs, 1),
                                       "frac_of_" + peak_kind: round(gbs / peak, 4)}
-    step_bytes = ab["step"] + ab["refresh"] / wl.period
-    step_gbs = step_bytes * world / (ms * 1e-3 / args.steps) / 1e9
+    # bytes of the timed region: the steps, plus the whole-table reads of the refreshes that ran inside it
+    step_bytes = ab["step"] + ab["refresh"] * timed_refreshes / args.steps
+    step_bytes_sep = ab["step_separate_calls"] + ab["refresh"] * timed_refreshes / args.steps
+    s_per_step = ms * 1e-3 / args.steps
+    step_gbs = step_bytes / s_per_step / 1e9                      # per GPU: every rank moves these bytes in that time
+    step_gbs_sep = step_bytes_sep / s_per_step / 1e9
+    # the refresh by itself, and the step time with one refresh charged every `period` steps whatever --steps was
+    refresh_us = 1e3 * prof["refresh_kernel"][0] / prof["refresh_kernel"][1] if "refresh_kernel" in prof else None
+    steps_only_us = (ms * 1e3 - (refresh_us or 0.0) * timed_refreshes) / args.steps
+    amortised_us = steps_only_us + (refresh_us or 0.0) / wl.period
+    amortised_bytes = ab["step"] + ab["refresh"] / wl.period
 
     cpu_baseline = None
     if tables_h is not None:
         n = 2 if wl.table_bytes() > 1e9 else 3
-        v, t_step, t_ref = oracle_sample(wl, tables_h, n, wl.period)
+        (v, t_step, t_ref), (v_mc, t_step_mc, t_ref_mc, threads, cores) = oracle_sample(wl, tables_h, n, wl.period)
+        sample = (f"{n} full steps of batch {wl.B} ({{:.0f}} ms each) plus one whole-table refresh ({{:.0f}} ms) "
+                  f"charged at 1/{wl.period} per step")
         cpu_baseline = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
-                        "sample": (f"{n} full steps of batch {wl.B} ({t_step * 1e3:.0f} ms each) plus one whole-table "
-                                   f"refresh ({t_ref * 1e3:.0f} ms) charged at 1/{wl.period} per step")}
+                        "sample": sample.format(t_step * 1e3, t_ref * 1e3),
+                        "all_cores": {"value": v_mc, "unit": UNIT, "cores": threads, "host_cores": cores,
+                                      "kind": "oracle, one table per thread",
+                                      "sample": sample.format(t_step_mc * 1e3, t_ref_mc * 1e3)}}
 
-    if rank == 0:
-        print(json.dumps({
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": warm, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": wl.name, "tables": wl.T, "dim": wl.D, "batch_per_gpu": wl.B,
-                       "lookups_per_step_per_gpu": Lavg, "unique_rows_per_step": Uavg, "unique_fraction": Uavg / Lavg,
-                       "bits": wl.bits, "grad_bits": 8, "refresh_period": wl.period, "table_bytes": wl.table_bytes(),
-                       "launch": ((f"CUDA graph replay, {spg} consecutive steps per graph" if group_graphs is not None else
-                                   "CUDA graph replay per step") if graphs is not None else "direct launches") +
-                                 ("; the index sort of batch k+1 runs on a second stream while batch k trains "
-                                  "(two workspaces, every step does one sort and one training half)" if pipelined
-                                  else ""),
-                       "parallelism": (f"{world} ranks, sparse INT8 gradient exchange every step" if dp_step is not None
-                                       else f"{world} replica(s), batch sharded by sample, no exchange"),
-                       "l2": f"{N_BATCHES} distinct pre-staged batches cycled; their rows, gradients and outputs "
-                             f"exceed the 126 MB L2 and the table is {wl.table_bytes() / 1e9:.2f} GB"},
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps},
-            "gpu_launches": int(launches),
-            "clocks": clocks,
-            "roofline": {"bound": "hbm", "kernel": dominant, "achieved": round(achieved, 1), "peak": peak,
-                         "peak_kind": peak_kind, "unit": "GB/s", "frac": round(achieved / peak, 4),
-                         "frac_of_8TBps_nominal": round(achieved / NOMINAL_HBM_GBS, 4),
-                         "traffic": NCU_TRAFFIC.get((wl.name, dominant)),
-                         "algorithmic_bytes_per_launch": int(dom_bytes)},
-            "step_roofline": {"algorithmic_bytes_per_step": int(step_bytes), "GB/s": round(step_gbs, 1),
-                              "frac_of_" + peak_kind: round(step_gbs / peak / world, 4),
-                              "frac_of_8TBps_nominal": round(step_gbs / NOMINAL_HBM_GBS / world, 4)},
-            "kernel_rooflines": per_kernel_roofline,
-            "kernels": kernels,
-            "cpu_baseline": cpu_baseline,
-        }))
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": warm, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": base_config(wl),
+        "run": {"lookups_per_step_per_gpu": Lavg, "unique_rows_per_step": Uavg, "unique_fraction": Uavg / Lavg,
+                "launch": ((f"CUDA graph replay, {spg} consecutive steps per graph" if group_graphs is not None else
+                            "CUDA graph replay per step") if graphs is not None else "direct launches") +
+                          ("; the index sort of batch k+1 runs on a second stream while batch k trains "
+                           "(two workspaces, every step does one sort and one training half)" if pipelined
+                           else ""),
+                "parallelism": (f"{world} ranks, sparse INT8 gradient exchange every step" if dp_step is not None
+                                else f"{world} replica(s), batch sharded by sample, no exchange"),
+                "l2": f"{N_BATCHES} distinct pre-staged batches cycled; their rows, gradients and outputs "
+                      f"exceed the 126 MB L2 and the table is {wl.table_bytes() / 1e9:.2f} GB",
+                "refreshes_in_timed_region": timed_refreshes},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "kernel": dominant, "achieved": round(achieved, 1), "peak": peak,
+                     "peak_kind": peak_kind, "unit": "GB/s", "frac": round(achieved / peak, 4),
+                     "frac_of_8TBps_nominal": round(achieved / NOMINAL_HBM_GBS, 4),
+                     "traffic": NCU_TRAFFIC.get((wl.name, dominant)),
+                     "algorithmic_bytes_per_launch": int(dom_bytes)},
+        # the timed region as it ran: its steps and the refreshes that fell inside it, bytes over time
+        "step_roofline": {"algorithmic_bytes_per_step": int(step_bytes), "GB/s": round(step_gbs, 1),
+                          "frac_of_" + peak_kind: round(step_gbs / peak, 4),
+                          "frac_of_8TBps_nominal": round(step_gbs / NOMINAL_HBM_GBS, 4),
+                          "separate_calls_bytes_per_step": int(step_bytes_sep),
+                          "separate_calls_frac_of_" + peak_kind: round(step_gbs_sep / peak, 4),
+                          "separate_calls_frac_of_8TBps_nominal": round(step_gbs_sep / NOMINAL_HBM_GBS, 4)},
+        # the same with one refresh charged every `period` steps (its own measured time and its bytes), whatever
+        # --steps was
+        "refresh": {"us": None if refresh_us is None else round(refresh_us, 2), "bytes": int(ab["refresh"]),
+                    "period": wl.period, "us_per_step_amortised": round(amortised_us, 3),
+                    "lookups_per_s_amortised": Lavg * world / (amortised_us * 1e-6),
+                    "bytes_per_step_amortised": int(amortised_bytes),
+                    "frac_of_" + peak_kind: round(amortised_bytes / (amortised_us * 1e-6) / 1e9 / peak, 4),
+                    "frac_of_8TBps_nominal": round(amortised_bytes / (amortised_us * 1e-6) / 1e9 / NOMINAL_HBM_GBS, 4)},
+        "kernel_rooflines": per_kernel_roofline,
+        "kernels": kernels,
+        "cpu_baseline": cpu_baseline,
+    }
     ctx.close()
-    if world > 1:
-        dist.destroy_process_group()
+    torch.cuda.synchronize()
+    return line
 
 
 def run_packed(args):
@@ -602,6 +703,59 @@ def run_packed(args):
     ctx.close()
 
 
+def launch_ranks(args):
+    """--gpus N without a launcher in the environment: start N ranks of this script, one per GPU, the way
+    the contract's launcher does, and pass their output through.  NCCL's initialisation log goes to files
+    of a temporary folder; its communicator lines are echoed to stderr afterwards."""
+    import glob
+    import socket
+    import tempfile
+
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    env = dict(os.environ)
+    logdir = tempfile.mkdtemp(prefix="dqrm_nccl_")
+    env.setdefault("NCCL_DEBUG", "INFO")
+    env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    env.setdefault("NCCL_DEBUG_FILE", os.path.join(logdir, "nccl.%h.%p.log"))
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *sys.argv[1:]]
+    rc = subprocess.call(cmd, env=env, cwd=ROOT)
+    shown = 0
+    for f in sorted(glob.glob(os.path.join(logdir, "*.log"))):
+        with open(f, errors="replace") as fh:
+            for ln in fh:
+                if shown < 60 and any(k in ln for k in ("Init COMPLETE", "NVLS", "comm 0x", "Connected all")):
+                    print("nccl:", ln.rstrip(), file=sys.stderr)
+                    shown += 1
+    return rc
+
+
+def run_stub(args):
+    """Launcher and rendezvous check without a GPU (used by the CPU tests): every rank sleeps through its
+    steps on the gloo backend, the job's time is the slowest rank's, rank 0 prints the line."""
+    import torch.distributed as dist
+    from paper_2410_20046_b200 import harness
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        time.sleep(0.002 * (1 + rank))
+    ms = harness.max_over_ranks((time.perf_counter() - t0) * 1e3)
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "value": harness.job_throughput(1000, world, args.steps, ms), "unit": UNIT,
+                          "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+                          "higher_is_better": True, "scaling": "weak", "stub": True}))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -615,6 +769,8 @@ def main():
     ap.add_argument("--workload", default="kaggle_b16384")
     ap.add_argument("--e2e-steps", type=int, default=50)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-also", action="store_true",
+                    help="with the default workload: do not measure terabyte_b32768 as well")
     ap.add_argument("--dp-exchange", action="store_true",
                     help="with --gpus N > 1: exchange the sparse INT8 gradient every step (paper's data parallelism) "
                          "instead of running independent replicas")
@@ -630,8 +786,13 @@ def main():
     ap.add_argument("--sort-after-forward", type=int, default=0,
                     help="1: the next batch's sort waits for this batch's forward and runs beside the rest of the step")
     ap.add_argument("--sort-path", type=int, default=0, help="0: per-table cluster sort, 1: global radix sort")
+    ap.add_argument("--stub-step", action="store_true", help=argparse.SUPPRESS)
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours" and not args.packed:
+        sys.exit(launch_ranks(args))
+    if args.stub_step:
+        run_stub(args)
+    elif args.impl == "reference":
         run_reference(args)
     elif args.packed:
         run_packed(args)

@@ -319,16 +319,17 @@ class Context:
             _ptr(grad_rows, torch.float32), _ptr(codes, torch.int8), _ptr(grad_scales, torch.float32),
             float(lr), int(B), int(L), self._ws_ptr, self.workspace_bytes, _stream(stream)))
 
-    # ---- the step in two calls; `ws` picks one of two workspaces (the second is made on first use) ----
+    # ---- the step in two calls; `ws` picks a workspace (number 0 exists, the others are made on first use) ----
     def _workspace(self, ws: int) -> int:
         import torch
 
         if ws == 0:
             return self._ws_ptr
-        if getattr(self, "workspace2", None) is None:
-            self.workspace2 = torch.empty(self.workspace_bytes + 256, dtype=torch.uint8, device="cuda")
-            self._ws2_ptr = (self.workspace2.data_ptr() + 255) // 256 * 256
-        return self._ws2_ptr
+        more = self.__dict__.setdefault("_more_workspaces", {})
+        if ws not in more:
+            buf = torch.empty(self.workspace_bytes + 256, dtype=torch.uint8, device="cuda")
+            more[ws] = (buf, (buf.data_ptr() + 255) // 256 * 256)
+        return more[ws][1]
 
     def sort_batch(self, indices, offsets, unique_rows, uniq_off, *, B, L, ws=0, stream=None):
         import torch

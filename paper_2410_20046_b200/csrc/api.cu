@@ -285,32 +285,28 @@ int dqrm_train_step(dqrm_ctx *ctx, float *tables, const int32_t *indices, const 
     if (!ws_ok(workspace, workspace_bytes, dq_bwd_ws_bytes(ctx, L, (int64_t)ctx->T * B))) return DQRM_ERR_WORKSPACE;
     cudaStream_t st = as_stream(stream);
     if (ctx->prof_on) dq_mark(ctx, st, DQ_K_BEGIN);
-    // The sort half of the backward needs only the indices, so it runs on the context's second
-    // stream while the forward runs on the caller's (per-launch profiling keeps one stream,
-    // because its events time consecutive launches).
+    // The backward up to the summed gradient needs the indices and the upstream gradient but neither the
+    // tables nor the forward's output, so it runs on the context's second stream while the forward runs on
+    // the caller's (per-launch profiling keeps one stream, because its events time consecutive launches).
+    // The quantise-and-update kernel writes the rows the forward reads, so it waits for both.
     const bool overlap = ctx->overlap && !ctx->prof_on && L > 0;
     cudaStream_t ss = overlap ? ctx->side : st;
-    const u32 *absmax = nullptr;
     if (overlap) {
         DQRM_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_fork, st));
         DQRM_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
     }
-    int rc;
-    if (overlap) {
-        rc = dq_launch_bwd_sort(ctx, indices, offsets, unique_rows, uniq_off, B, L, workspace, workspace_bytes, ss, &absmax);
-        if (rc == DQRM_OK) rc = dq_launch_fwd(ctx, tables, indices, offsets, scales, bits, out, nullptr, B, L, st);
-        // join even after an error so that the caller's stream stays ordered behind the side stream
+    int rc = dq_launch_bwd_sort(ctx, indices, offsets, unique_rows, uniq_off, B, L, workspace, workspace_bytes, ss, nullptr);
+    if (rc == DQRM_OK)
+        rc = dq_launch_bwd_reduce(ctx, grad_out, uniq_off, grad_rows, B, L, workspace, workspace_bytes, ss);
+    int rc2 = dq_launch_fwd(ctx, tables, indices, offsets, scales, bits, out, nullptr, B, L, st);
+    if (overlap) {   // join even after an error so that the caller's stream stays ordered behind the side stream
         cudaEventRecord(ctx->ev_join, ctx->side);
         cudaStreamWaitEvent(st, ctx->ev_join, 0);
-    } else {
-        rc = dq_launch_fwd(ctx, tables, indices, offsets, scales, bits, out, nullptr, B, L, st);
-        if (rc == DQRM_OK)
-            rc = dq_launch_bwd_sort(ctx, indices, offsets, unique_rows, uniq_off, B, L, workspace, workspace_bytes, st, &absmax);
     }
     if (rc != DQRM_OK) return rc;
-    rc = dq_launch_bwd_reduce(ctx, grad_out, uniq_off, grad_rows, B, L, workspace, workspace_bytes, st);
-    if (rc != DQRM_OK) return rc;
-    return dq_launch_quant_update(ctx, tables, unique_rows, uniq_off, grad_rows, absmax, codes, grad_scales, lr, st);
+    if (rc2 != DQRM_OK) return rc2;
+    return dq_launch_quant_update(ctx, tables, unique_rows, uniq_off, grad_rows, dq_bwd_absmax_bits(ctx, L, workspace),
+                                  codes, grad_scales, lr, st);
 }
 
 int dqrm_grad_absmax(dqrm_ctx *ctx, const float *grad_rows, const int32_t *uniq_off, float *absmax, void *stream)
@@ -372,13 +368,24 @@ int dqrm_train_step_sorted(dqrm_ctx *ctx, float *tables, const int32_t *indices,
     if (!ws_ok(workspace, workspace_bytes, dq_bwd_ws_bytes(ctx, L, (int64_t)ctx->T * B))) return DQRM_ERR_WORKSPACE;
     cudaStream_t st = as_stream(stream);
     if (ctx->prof_on) dq_mark(ctx, st, DQ_K_BEGIN);
-    int rc = dq_launch_fwd(ctx, tables, indices, offsets, scales, bits, out, nullptr, B, L, st);
+    // the gradient summation (second stream of the context) runs beside the forward (caller's stream)
+    const bool overlap = ctx->overlap && !ctx->prof_on && L > 0;
+    cudaStream_t ss = overlap ? ctx->side : st;
+    if (overlap) {
+        DQRM_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_fork, st));
+        DQRM_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
+    }
+    int rc = dq_launch_bwd_reduce(ctx, grad_out, uniq_off, grad_rows, B, L, workspace, workspace_bytes, ss);
+    int rc2 = dq_launch_fwd(ctx, tables, indices, offsets, scales, bits, out, nullptr, B, L, st);
+    cudaEventRecord(ctx->ev_fwd, st);                           // for dqrm_stream_wait_forward
+    if (overlap) {
+        cudaEventRecord(ctx->ev_join, ctx->side);
+        cudaStreamWaitEvent(st, ctx->ev_join, 0);
+    }
     if (rc != DQRM_OK) return rc;
-    DQRM_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_fwd, st));      // for dqrm_stream_wait_forward
-    rc = dq_launch_bwd_reduce(ctx, grad_out, uniq_off, grad_rows, B, L, workspace, workspace_bytes, st);
-    if (rc != DQRM_OK) return rc;
-    return dq_launch_quant_update(ctx, tables, unique_rows, uniq_off, grad_rows,
-                                  dq_bwd_absmax_bits(ctx, L, workspace), codes, grad_scales, lr, st);
+    if (rc2 != DQRM_OK) return rc2;
+    return dq_launch_quant_update(ctx, tables, unique_rows, uniq_off, grad_rows, dq_bwd_absmax_bits(ctx, L, workspace),
+                                  codes, grad_scales, lr, st);
 }
 
 int dqrm_stream_wait_forward(dqrm_ctx *ctx, void *stream)
@@ -480,19 +487,20 @@ int dqrm_train_step_host(dqrm_ctx *ctx, float *tables, const int32_t *h_indices,
     DQRM_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
     char *step_ws = ws + y.step_ws;
     const size_t step_ws_bytes = workspace_bytes - y.step_ws;
-    const u32 *absmax = nullptr;
-    int rc = dq_launch_bwd_sort(ctx, d_idx, d_off, d_ur, d_uo, B, L, step_ws, step_ws_bytes, ctx->side, &absmax);
+    int rc = dq_launch_bwd_sort(ctx, d_idx, d_off, d_ur, d_uo, B, L, step_ws, step_ws_bytes, ctx->side, nullptr);
     if (rc == DQRM_OK) rc = dq_launch_fwd(ctx, tables, d_idx, d_off, scales, bits, d_out, nullptr, B, L, st);
     // join every stream even after an error, so that the caller's stream stays ordered behind them
     cudaEventRecord(ctx->ev_h_fwd, st);
     cudaStreamWaitEvent(ctx->copy_out, ctx->ev_h_fwd, 0);
     if (rc == DQRM_OK) cudaMemcpyAsync(h_out, d_out, go_bytes, cudaMemcpyDeviceToHost, ctx->copy_out);
     cudaEventRecord(ctx->ev_h_out, ctx->copy_out);
+    // the gradient summation follows the sort on the second stream as soon as the upstream gradient has arrived
+    cudaStreamWaitEvent(ctx->side, ctx->ev_h_go, 0);
+    if (rc == DQRM_OK) rc = dq_launch_bwd_reduce(ctx, d_go, d_uo, d_gr, B, L, step_ws, step_ws_bytes, ctx->side);
     cudaEventRecord(ctx->ev_join, ctx->side);
     cudaStreamWaitEvent(st, ctx->ev_join, 0);
-    cudaStreamWaitEvent(st, ctx->ev_h_go, 0);
-    if (rc == DQRM_OK) rc = dq_launch_bwd_reduce(ctx, d_go, d_uo, d_gr, B, L, step_ws, step_ws_bytes, st);
-    if (rc == DQRM_OK) rc = dq_launch_quant_update(ctx, tables, d_ur, d_uo, d_gr, absmax, d_codes, d_gs, lr, st);
+    if (rc == DQRM_OK)
+        rc = dq_launch_quant_update(ctx, tables, d_ur, d_uo, d_gr, dq_bwd_absmax_bits(ctx, L, step_ws), d_codes, d_gs, lr, st);
     cudaStreamWaitEvent(st, ctx->ev_h_out, 0);
     if (rc != DQRM_OK) return rc;
     DQRM_CUDA_TRY(ctx, cudaGetLastError());

@@ -362,7 +362,7 @@ int launch_reduce(dqrm_ctx *ctx, const Layout &y, char *ws, const u32 *keys, con
     const u32 *seg_start = reinterpret_cast<const u32 *>(ws + y.seg_start);
     double *partials = reinterpret_cast<double *>(ws + y.partials);
     u32 *long_list = reinterpret_cast<u32 *>(ws + y.long_list);
-    const size_t red_smem = (size_t)(ctx->T + 1) * sizeof(u32) + (size_t)gpb * SEG_CHUNK * sizeof(u32);
+    const size_t red_smem = (size_t)(ctx->T + 1) * sizeof(u32) + (size_t)gpb * 2 * SEG_CHUNK * sizeof(u32);
     if (ctx->D == RL * RV * RC)
         seg_reduce_kernel<RL, RV, RC, true><<<grid, 256, red_smem, st>>>(
             keys, vals, seg_start, reinterpret_cast<const u32 *>(ws + y.chunk_first), uniq_off, grad_out, grad_rows,

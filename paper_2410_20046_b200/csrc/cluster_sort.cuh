@@ -46,16 +46,11 @@ __device__ __forceinline__ u32 *remote(cg::cluster_group &cluster, u32 *p, unsig
     return cluster.map_shared_rank(p, rank);
 }
 
-// lanes of the warp that hold the same 8-bit digit as this lane (ballot per bit: the match
-// instruction costs tens of cycles of a shared unit when all 32 digits differ)
+// lanes of the warp that hold the same 8-bit digit as this lane (one call by all lanes; a lane without an
+// entry matches nobody)
 __device__ __forceinline__ u32 same_digit_lanes(u32 d, bool valid)
 {
-    u32 peers = __ballot_sync(0xffffffffu, valid);
-#pragma unroll
-    for (int b = 0; b < 8; ++b) {
-        const u32 m = __ballot_sync(0xffffffffu, (d >> b) & 1u);
-        peers &= ((d >> b) & 1u) ? m : ~m;
-    }
+    const u32 peers = __match_any_sync(0xffffffffu, valid ? d : 256u + (threadIdx.x & 31));
     return valid ? peers : 0u;
 }
 

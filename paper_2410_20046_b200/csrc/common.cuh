@@ -20,7 +20,7 @@ struct dqrm_ctx {
     int num_sms = 0;
     int key_bits = 1;               // bits of an arena row number
     int sort_path = 0;              // 0: per-table cluster sort, 1: global radix sort
-    cudaStream_t side = nullptr;    // second stream: a training step sorts the indices beside its forward
+    cudaStream_t side = nullptr;    // second stream: a training step sorts the indices and sums the gradient beside its forward
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     cudaEvent_t ev_fwd = nullptr;   // recorded behind the forward of the last training step enqueued
     // host-buffer step: the upstream gradient comes in and the pooled output goes out on streams of their own
@@ -170,6 +170,27 @@ __device__ __forceinline__ void dq_cp_async_wait() { asm volatile("cp.async.wait
 
 // asks L2 for the 128-byte line that holds p (no register, no scoreboard entry: the later load finds it there)
 __device__ __forceinline__ void dq_prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];\n" ::"l"(p)); }
+
+// L2 eviction priorities.  Data that a later kernel of the same step reads again (the summed gradient rows, the
+// touched master rows) is marked to be evicted last; what is touched once is streamed (__ldcs / __stcs).
+__device__ __forceinline__ uint64_t dq_policy_evict_last()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;\n" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ float4 dq_ld_nc_keep(const float4 *p, uint64_t pol)
+{
+    float4 v;
+    asm volatile("ld.global.nc.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;\n"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p), "l"(pol));
+    return v;
+}
+__device__ __forceinline__ void dq_st_keep(float4 *p, const float4 &v, uint64_t pol)
+{
+    asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;\n"
+                 :: "l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "l"(pol) : "memory");
+}
 
 __device__ __forceinline__ void dq_report(int *status, int code)
 {

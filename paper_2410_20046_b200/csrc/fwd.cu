@@ -118,6 +118,7 @@ fwd_onehot_kernel(const FwdArgs a)
     const float4 *tbl_lane = reinterpret_cast<const float4 *>(tc.tbl) + lane;
     const int TD4 = a.T * d4;                 // 128-bit vectors between the output rows of bags i and i+1
     bool bad = false;
+    const uint64_t keep = dq_policy_evict_last();
 
     for (int i0 = (blockIdx.x * WPB + warp) * 32; i0 < a.B; i0 += gridDim.x * (WPB * 32)) {
         // ---- lane-per-bag bookkeeping
@@ -152,7 +153,7 @@ fwd_onehot_kernel(const FwdArgs a)
                 for (int b = 0; b < NB; ++b) {
                     const int bag = k0 + b * RPW + grp;
                     if (bag < 32 && ((one >> bag) & 1u) && (EXACT || c4 < d4))
-                        v[b] = __ldg(tbl_lane + (int64_t)ib[b] * d4 + c * LPR);
+                        v[b] = dq_ld_nc_keep(tbl_lane + (int64_t)ib[b] * d4 + c * LPR, keep);   // the update reads the row again
                 }
 #pragma unroll
                 for (int b = 0; b < NB; ++b) {
@@ -160,7 +161,7 @@ fwd_onehot_kernel(const FwdArgs a)
                     if (bag < 32 && ((one >> bag) & 1u) && (EXACT || c4 < d4)) {
                         float4 cd, f;
                         dq_fq4(v[b], tc.qs, cd, f);
-                        out_lane[(int64_t)bag * TD4 + c * LPR] = f;
+                        __stcs(out_lane + (int64_t)bag * TD4 + c * LPR, f);   // written once, read by nobody here
                     }
                 }
             }

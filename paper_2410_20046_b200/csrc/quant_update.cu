@@ -10,22 +10,11 @@
 // streams are 128-bit per lane.
 #include <mutex>
 #include "common.cuh"
+#include "row_stream.cuh"
 
 namespace {
 
-constexpr int QU_THREADS = 256;
-enum { MODE_QUANT = 0, MODE_UPDATE = 1, MODE_FUSED = 2 };
-
-// largest t with uoff[t] <= u, skipping empty tables
-__device__ __forceinline__ int table_of_row(const int32_t *uoff, int T, int64_t u)
-{
-    int lo = 0, hi = T;
-    while (hi - lo > 1) {
-        int mid = (lo + hi) >> 1;
-        if (uoff[mid] <= u) lo = mid; else hi = mid;
-    }
-    return lo;
-}
+using namespace rowstream;
 
 __global__ void __launch_bounds__(QU_THREADS)
 absmax_kernel(const float *__restrict__ grad_rows, const int32_t *__restrict__ uniq_off, int T, int D,
@@ -69,10 +58,6 @@ absmax_kernel(const float *__restrict__ grad_rows, const int32_t *__restrict__ u
         if (s_max[t]) atomicMax(&absmax[t], s_max[t]);
 }
 
-// rows in flight per lane group: fewer when a lane already holds several vectors of every row
-template <int CH> struct RowsInFlight { static constexpr int v = CH >= 4 ? 1 : (CH == 2 ? 2 : 4); };
-
-// EXACT: the feature size is 4*LPR*CH, a compile-time constant, and the per-vector range checks fall away
 template <int MODE, int LPR, int CH, bool EXACT>
 __global__ void __launch_bounds__(QU_THREADS)
 row_stream_kernel(float *__restrict__ tables, const int64_t *__restrict__ row_off,
@@ -81,102 +66,9 @@ row_stream_kernel(float *__restrict__ tables, const int64_t *__restrict__ row_of
                   int8_t *__restrict__ codes, float *__restrict__ grad_scales, float lr, int T, int D_any,
                   int *__restrict__ status)
 {
-    constexpr int NB = RowsInFlight<CH>::v;
-    const int D = EXACT ? 4 * LPR * CH : D_any;
     extern __shared__ unsigned char smem_raw[];
-    int32_t *s_uoff = reinterpret_cast<int32_t *>(smem_raw);      // [T+1]
-    float *s_scale = reinterpret_cast<float *>(s_uoff + (T + 1)); // [T] gradient scale of every table
-    for (int t = threadIdx.x; t <= T; t += QU_THREADS) s_uoff[t] = uniq_off[t];
-    for (int t = threadIdx.x; t < T; t += QU_THREADS) {
-        const float sc = (MODE == MODE_UPDATE) ? grad_scales[t] : dq_scale_from_absmax(__uint_as_float(absmax[t]), 8);
-        s_scale[t] = sc;
-        if (MODE != MODE_UPDATE && blockIdx.x == 0) grad_scales[t] = sc;
-    }
-    __syncthreads();
-    const int d4 = D >> 2;
-    const int64_t U = s_uoff[T];
-    const int lane = threadIdx.x % LPR;
-    const int64_t group = ((int64_t)blockIdx.x * QU_THREADS + threadIdx.x) / LPR;
-    const int64_t n_groups = (int64_t)gridDim.x * QU_THREADS / LPR;
-    // a lane group owns a contiguous range of unique rows: its rows mostly share a table, and its reads
-    // of the gradient rows and writes of the codes are sequential
-    int64_t per = (U + n_groups - 1) / n_groups;
-    if (per < NB) per = NB;             // few rows: fewer groups, each with a full set of rows in flight
-    const int64_t u_begin = group * per, u_end = min(U, u_begin + per);
-    int cur_t = -1;
-    int64_t cur_end = -1, r0 = 0, nrows = 1;
-    bool bad = false;
-    float s = 1.f;
-    QuantScale qs = dq_make_scale(1.f, 8);
-    for (int64_t u = u_begin; u < u_end;) {
-        if (u >= cur_end) {
-            cur_t = table_of_row(s_uoff, T, u);
-            cur_end = s_uoff[cur_t + 1];
-            if (MODE != MODE_QUANT) { r0 = __ldg(row_off + cur_t); nrows = __ldg(row_off + cur_t + 1) - r0; }
-            s = s_scale[cur_t];
-            qs = dq_make_scale(s, 8);
-        }
-        // up to NB rows of the current table at once
-        const int nb = (int)min((int64_t)NB, min(u_end, cur_end) - u);
-        float4 *wrow[NB];
-        float4 g[NB][CH], w[NB][CH];
-        char4 cin[NB][CH];
-#pragma unroll
-        for (int b = 0; b < NB; ++b) {
-            wrow[b] = nullptr;
-            if (b < nb && MODE != MODE_QUANT) {
-                // a row number outside its table is reported and kept inside the arena, never followed
-                int64_t row = __ldg(unique_rows + u + b);
-                if (row < 0 || row >= nrows) { bad = true; row = row < 0 ? 0 : nrows - 1; }
-                wrow[b] = reinterpret_cast<float4 *>(tables + (r0 + row) * D);
-            }
-        }
-#pragma unroll
-        for (int b = 0; b < NB; ++b) {
-            if (b < nb) {
-#pragma unroll
-                for (int ch = 0; ch < CH; ++ch) {
-                    const int c4 = ch * LPR + lane;
-                    if (EXACT || c4 < d4) {
-                        if (MODE == MODE_UPDATE) cin[b][ch] = *reinterpret_cast<const char4 *>(codes + (u + b) * D + 4 * c4);
-                        else g[b][ch] = __ldg(reinterpret_cast<const float4 *>(grad_rows + (u + b) * D) + c4);
-                        if (MODE != MODE_QUANT) w[b][ch] = wrow[b][c4];
-                    }
-                }
-            }
-        }
-#pragma unroll
-        for (int b = 0; b < NB; ++b) {
-            if (b < nb) {
-#pragma unroll
-                for (int ch = 0; ch < CH; ++ch) {
-                    const int c4 = ch * LPR + lane;
-                    if (EXACT || c4 < d4) {
-                        float4 q;                      // integer codes held as floats
-                        if (MODE == MODE_UPDATE) {
-                            q = make_float4((float)cin[b][ch].x, (float)cin[b][ch].y, (float)cin[b][ch].z, (float)cin[b][ch].w);
-                        } else {
-                            float4 dq_unused;
-                            dq_fq4(g[b][ch], qs, q, dq_unused);
-                            *reinterpret_cast<char4 *>(codes + (u + b) * D + 4 * c4) =
-                                make_char4((signed char)(int)q.x, (signed char)(int)q.y, (signed char)(int)q.z,
-                                           (signed char)(int)q.w);
-                        }
-                        if (MODE != MODE_QUANT) {
-                            float4 x = w[b][ch];
-                            x.x = __fsub_rn(x.x, __fmul_rn(lr, __fmul_rn(q.x, s)));
-                            x.y = __fsub_rn(x.y, __fmul_rn(lr, __fmul_rn(q.y, s)));
-                            x.z = __fsub_rn(x.z, __fmul_rn(lr, __fmul_rn(q.z, s)));
-                            x.w = __fsub_rn(x.w, __fmul_rn(lr, __fmul_rn(q.w, s)));
-                            wrow[b][c4] = x;
-                        }
-                    }
-                }
-            }
-        }
-        u += nb;
-    }
-    if (MODE != MODE_QUANT && bad) dq_report(status, DQRM_ERR_INDEX_RANGE);
+    row_stream_body<MODE, LPR, CH, EXACT>(smem_raw, tables, row_off, unique_rows, uniq_off, grad_rows, absmax, codes,
+                                          grad_scales, lr, T, D_any, status);
 }
 
 template <int MODE, int LPR, int CH>

@@ -3,12 +3,14 @@
 //
 // Input: keys[L] (arena rows, ascending), vals[L] (row of grad_out for each lookup, in
 // stable order), chunk_first[c] = index of the segment that holds sorted entry 32*c,
-// seg_start[U+1].  One lane group owns one chunk of 32 sorted entries and walks it in
-// order with a few upstream-gradient rows in flight.  All sums are FP64 and have a shape
-// fixed by the entry positions, so results are reproducible.  A run that is a whole segment is rounded to
-// FP32 and written; a run cut by the chunk boundary leaves an FP64 partial and the
-// segment is finished by one of the fix-up kernels (a warp for up to 32 pieces, a block
-// beyond that).  The per-table abs-max of the rounded sums is collected on the way.
+// seg_start[U+1].  Work is dealt in chunks of 32 sorted entries, one lane group per chunk,
+// but a segment is summed by the group in whose chunk it BEGINS, tail in the next chunk
+// included; the group sees where that tail ends from the next chunk's keys, which it loads
+// with its own.  All sums are FP64 and have a shape fixed by the entry positions, so results
+// are reproducible.  Only a segment whose tail is not over within the next chunk (a hot row)
+// is summed in pieces: every chunk it covers leaves an FP64 partial and the segment is
+// finished by one of the fix-up kernels (a warp for up to 32 pieces, a block beyond that).
+// The per-table abs-max of the rounded sums is collected on the way.
 #pragma once
 #include <type_traits>
 #include "common.cuh"
@@ -102,14 +104,16 @@ __device__ __forceinline__ void vec_add(double (&acc)[VEC], const typename Vec<V
     else { acc[0] += (double)v.x; acc[1] += (double)v.y; acc[2] += (double)v.z; acc[3] += (double)v.w; }
 }
 
-// One lane group (LPR lanes) owns one chunk of 32 sorted entries and walks it in order,
-// NB upstream-gradient rows in flight at a time.  Lane `lane` holds, for ch < CH, the VEC
-// consecutive features starting at (ch*LPR + lane)*VEC.  Per chunk, one lane per entry compares
-// neighbouring keys once; the resulting bit mask of segment heads and the payloads (parked in
-// shared memory) are all the walk needs, so an entry costs one shared load, one address, one
-// 128-bit load, a bit test and the FP64 adds.
+// One lane group (LPR lanes) owns one chunk of 32 sorted entries and walks in order the segments that
+// BEGIN in it, NB upstream-gradient rows in flight at a time: a segment's tail in the next chunk is
+// read by the same group, and a leading run that began in the chunk before is skipped, so the common
+// segment that straddles a chunk boundary needs no partial sum.  Lane `lane` holds, for ch < CH, the
+// VEC consecutive features starting at (ch*LPR + lane)*VEC.  Per chunk, one lane per entry compares
+// neighbouring keys once (this chunk's and the next one's); the resulting bit masks of segment heads
+// and the payloads (parked in shared memory) are all the walk needs, so an entry costs one shared
+// load, one address, one 128-bit load, a bit test and the FP64 adds.
 // (256-byte rows want four resident blocks per SM: that caps the kernel at 64 registers)
-template <int LPR, int VEC, int CH, bool EXACT>
+template <int LPR, int VEC, int CH, bool EXACT, bool OWN = (LPR >= 8)>
 __global__ void __launch_bounds__(256, (LPR == 16 && VEC == 4 && CH == 1) ? 4 : 1)
 seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
                   const u32 *__restrict__ seg_start, const u32 *__restrict__ chunk_first,
@@ -124,7 +128,7 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
     const int D = EXACT ? LPR * VEC * CH : D_any;
     extern __shared__ unsigned char smem_raw[];
     u32 *s_uoff = reinterpret_cast<u32 *>(smem_raw);                                     // [T+1]
-    u32 *s_vals = s_uoff + (T + 1) + (size_t)(threadIdx.x / LPR) * CHUNK;                // this group's [CHUNK]
+    u32 *s_vals = s_uoff + (T + 1) + (size_t)(threadIdx.x / LPR) * (2 * CHUNK);          // this group's [2*CHUNK]
     for (int t = threadIdx.x; t <= T; t += blockDim.x) s_uoff[t] = (u32)uniq_off[t];
     __syncthreads();
 
@@ -140,14 +144,16 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
     const int64_t n_groups = (int64_t)gridDim.x * blockDim.x / LPR;
     AbsmaxTracker tr;
     bool bad = false;
+    const uint64_t keep = dq_policy_evict_last();
 
     for (int64_t c = group; c < num_chunks; c += n_groups) {
         const int64_t i0 = c * CHUNK;
         const int n = (int)(min(i0 + (int64_t)CHUNK, L) - i0);
-        // heads: entry e starts a segment when its key differs from the key before it.  All loads are
-        // issued before the first vote so that they are in flight together.
-        u32 heads = 0;
-        u32 kc[EPL], kp[EPL], vv[EPL];
+        const int n_next = (int)max((int64_t)0, min((int64_t)CHUNK, L - i0 - CHUNK));
+        // Heads: entry e starts a segment when its key differs from the key before it; the same for the
+        // chunk behind, whose first head tells where this chunk's last segment ends.  All loads are issued
+        // before the first vote so that they are in flight together.
+        u32 kc[EPL], kp[EPL], vv[EPL], kn[OWN ? EPL : 1], knp[OWN ? EPL : 1], vn[OWN ? EPL : 1];
 #pragma unroll
         for (int j = 0; j < EPL; ++j) {
             const int e = j * LPR + lane;
@@ -158,10 +164,23 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
                 kc[j] = keys[i];
                 kp[j] = i > 0 ? keys[i - 1] : ~kc[j];
             }
+            if (OWN) {
+                kn[j] = knp[j] = vn[j] = 0u;
+                if (e < n_next) {
+                    vn[j] = vals[i + CHUNK];
+                    kn[j] = keys[i + CHUNK];
+                    knp[j] = keys[i + CHUNK - 1];
+                }
+            }
         }
-        const u32 k_after = (i0 + n == L) ? 0u : keys[i0 + n];
+        // OWN: did the run that enters this chunk begin in the chunk before?  (the keys ascend: it did unless the
+        // key 33 entries back is still the same).  Otherwise: the key behind the chunk tells whether its last run ends
+        u32 k_x = 0u;
+        if (OWN) { if (i0 > CHUNK) k_x = keys[i0 - CHUNK - 1]; }
+        else if (i0 + n < L) k_x = keys[i0 + n];
         const u32 u_first = chunk_first[c];
         __syncwarp(gmask);                        // the previous chunk's payloads are no longer read
+        u32 heads = 0, heads_n = 0;
 #pragma unroll
         for (int j = 0; j < EPL; ++j) {
             const int e = j * LPR + lane;
@@ -178,10 +197,21 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
                         if (b < D * (int)sizeof(float)) dq_prefetch_l2(row + b);
                 }
             }
+            const u32 lm = LPR >= 32 ? 0xffffffffu : ((1u << LPR) - 1u);
+            if (OWN) {
+                if (e < n_next) {
+                    u32 v = vn[j];
+                    if ((int64_t)v >= G) { bad = true; v = 0u; }
+                    s_vals[CHUNK + e] = v;
+                }
+                const bool head_n = (e < n_next) && (kn[j] != knp[j]);
+                heads_n |= ((__ballot_sync(gmask, head_n) >> gbase) & lm) << (j * LPR);
+            }
             const bool head = (e < n) && (kc[j] != kp[j]);
-            const u32 bits = (__ballot_sync(gmask, head) >> gbase) & (LPR >= 32 ? 0xffffffffu : ((1u << LPR) - 1u));
-            heads |= bits << (j * LPR);
+            heads |= ((__ballot_sync(gmask, head) >> gbase) & lm) << (j * LPR);
         }
+        if (n_next < CHUNK) heads_n |= 1u << n_next;   // the end of the array closes a run like a head
+        const u32 k_0 = __shfl_sync(gmask, kc[0], gbase);
         // the chunk's last key sits in lane (n-1) % LPR, register (n-1) / LPR
         u32 k_last = 0u;
 #pragma unroll
@@ -189,22 +219,44 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
             if ((n - 1) / LPR == j) k_last = kc[j];
         k_last = __shfl_sync(gmask, k_last, gbase + (n - 1) % LPR);
         __syncwarp(gmask);
-        // does the chunk's first run begin here, does its last run end here?
-        const bool first_begins = heads & 1u;
-        const bool last_ends = (i0 + n == L) || (k_after != k_last);
-        heads &= ~1u;                             // the walk starts a run at entry 0 either way
-        u32 u = u_first;
-        int run_start = 0;
+
+        // ---- which entries this group sums: [ea, eb) relative to i0, eb up to 2*CHUNK.
+        // A segment is summed where it BEGINS, together with its tail in the next chunk; a leading run that
+        // began in the chunk before and ends here was summed there.  Only a segment whose tail is not over
+        // within the next chunk is summed in pieces (FP64 partials, folded by the fix-up kernel).
+        // (Without OWN - rows so narrow that the extra keys and payloads would cost more registers than the
+        // fix-up saves - a group sums exactly its chunk and every run cut by a chunk boundary is a piece.)
+        const bool any_head = heads != 0u;
+        const int f = any_head ? __ffs(heads) - 1 : n;                 // first head (n: none)
+        bool lead_piece, trail_long;
+        int ea, eb;
+        if (OWN) {
+            const bool closes_here = any_head || n < CHUNK;
+            const bool began_prev = (i0 <= CHUNK) || (k_x != k_0);
+            lead_piece = f > 0 && !(closes_here && began_prev);
+            ea = lead_piece ? 0 : f;
+            trail_long = any_head && heads_n == 0u;
+            eb = n + ((any_head && heads_n != 0u) ? __ffs(heads_n) - 1 : 0);    // (an extension only when n == CHUNK)
+        } else {
+            lead_piece = f > 0;
+            ea = 0;
+            trail_long = !((i0 + n == L) || (k_x != k_last));
+            eb = n;
+        }
+        if (eb <= ea) continue;                   // group-uniform
+        heads &= ~1u;                             // the walk starts a run at its first entry either way
+        u32 u = u_first + ((ea > 0) ? 1u : 0u);   // segment of entry ea (ea > 0: it is the chunk's first head)
+        int run_start = ea;
         double acc[CH][VEC];
 #pragma unroll
         for (int ch = 0; ch < CH; ++ch)
 #pragma unroll
             for (int q = 0; q < VEC; ++q) acc[ch][q] = 0.0;
 
-        // closes run [a, b) (chunk-relative) of segment u; runs strictly inside the chunk are whole segments
-        auto flush = [&](int a, int b) {
-            const bool begins = (a != 0) || first_begins;
-            const bool ends = (b != n) || last_ends;
+        // closes run [rs, re) (chunk-relative) of segment u
+        auto flush = [&](int rs, int re) {
+            const bool begins = !(lead_piece && rs == 0);
+            const bool ends = !(trail_long && re == eb);
             if (begins && ends) {
                 float m = 0.f;
 #pragma unroll
@@ -219,7 +271,7 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
                             m = fmaxf(m, fmaxf(fabsf(r.x), fabsf(r.y)));
                         } else {
                             float4 r = make_float4((float)acc[ch][0], (float)acc[ch][1], (float)acc[ch][2], (float)acc[ch][3]);
-                            *reinterpret_cast<float4 *>(dst) = r;
+                            dq_st_keep(reinterpret_cast<float4 *>(dst), r, keep);   // quantise+update reads it next
                             m = fmaxf(fmaxf(m, fmaxf(fabsf(r.x), fabsf(r.y))), fmaxf(fabsf(r.z), fabsf(r.w)));
                         }
                     }
@@ -238,51 +290,56 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
                 if (begins && lane == 0) {
                     const u32 sa = seg_start[u], sb = seg_start[u + 1];
                     const u32 npieces = (sb - 1) / CHUNK - sa / CHUNK + 1;
-                    if (npieces > BIG_PIECES)
-                        long_list[num_chunks - 1 - atomicAdd(&counters[CNT_BIG], 1u)] = u;
-                    else
-                        long_list[atomicAdd(&counters[CNT_LONG], 1u)] = u;
+                    // (the list has a slot per chunk and every chunk begins at most one such segment; the bound only
+                    // matters for a workspace that is summed twice without a sort in between, which must not write
+                    // outside the list)
+                    if (npieces > BIG_PIECES) {
+                        const u32 k = atomicAdd(&counters[CNT_BIG], 1u);
+                        if ((int64_t)k < num_chunks) long_list[num_chunks - 1 - k] = u;
+                    } else {
+                        const u32 k = atomicAdd(&counters[CNT_LONG], 1u);
+                        if ((int64_t)k < num_chunks) long_list[k] = u;
+                    }
                 }
             }
         };
 
-        // a full chunk (all but the arena's last) needs no per-entry range checks
-        auto walk = [&](auto full_tag) {
+        // whole batches of NB entries need no per-entry range checks
+        auto walk = [&](int e0, auto full_tag) {
             constexpr bool FULL = decltype(full_tag)::value;
-            const int n_walk = FULL ? CHUNK : n;
-            for (int eb = 0; eb < n_walk; eb += NB) {
-                vec_t r[NB][CH];
+            vec_t r[NB][CH];
 #pragma unroll
-                for (int e = 0; e < NB; ++e) {
-                    if (FULL || eb + e < n) {
-                        const vec_t *src = g_lane + (int64_t)s_vals[eb + e] * dv;
+            for (int k = 0; k < NB; ++k) {
+                if (FULL || e0 + k < eb) {
+                    const vec_t *src = g_lane + (int64_t)s_vals[e0 + k] * dv;
 #pragma unroll
-                        for (int ch = 0; ch < CH; ++ch)
-                            if (EXACT || ch * LPR + lane < dv) r[e][ch] = __ldg(src + ch * LPR);
-                    }
+                    for (int ch = 0; ch < CH; ++ch)
+                        if (EXACT || ch * LPR + lane < dv) r[k][ch] = __ldcs(src + ch * LPR);   // every row is read once
                 }
-                const u32 hb = heads >> eb;
+            }
 #pragma unroll
-                for (int e = 0; e < NB; ++e) {
-                    if (FULL || eb + e < n) {
-                        if ((hb >> e) & 1u) {
-                            flush(run_start, eb + e);
-                            u += 1;
-                            run_start = eb + e;
-#pragma unroll
-                            for (int ch = 0; ch < CH; ++ch)
-#pragma unroll
-                                for (int q = 0; q < VEC; ++q) acc[ch][q] = 0.0;
-                        }
+            for (int k = 0; k < NB; ++k) {
+                const int e = e0 + k;
+                if (FULL || e < eb) {
+                    if (e > ea && e < CHUNK && ((heads >> e) & 1u)) {
+                        flush(run_start, e);
+                        u += 1;
+                        run_start = e;
 #pragma unroll
                         for (int ch = 0; ch < CH; ++ch)
-                            if (EXACT || ch * LPR + lane < dv) vec_add<VEC>(acc[ch], r[e][ch]);
+#pragma unroll
+                            for (int q = 0; q < VEC; ++q) acc[ch][q] = 0.0;
                     }
+#pragma unroll
+                    for (int ch = 0; ch < CH; ++ch)
+                        if (EXACT || ch * LPR + lane < dv) vec_add<VEC>(acc[ch], r[k][ch]);
                 }
             }
         };
-        if (n == CHUNK) walk(std::true_type{}); else walk(std::false_type{});
-        flush(run_start, n);
+        int e0 = ea;
+        for (; e0 + NB <= eb; e0 += NB) walk(e0, std::true_type{});
+        if (e0 < eb) walk(e0, std::false_type{});
+        flush(run_start, eb);
     }
     absmax_push<LPR>(tr, absmax);      // group-uniform: all lanes of a group walk the same chunks
     if (bad) dq_report(status, DQRM_ERR_INDEX_RANGE);
@@ -339,7 +396,7 @@ __device__ __forceinline__ void
 fixup_small(const u32 *__restrict__ keys, const u32 *__restrict__ seg_start,
             const double *__restrict__ partials, const u32 *__restrict__ long_list,
             const u32 *__restrict__ counters, float *__restrict__ grad_rows, u32 *__restrict__ absmax,
-            const int64_t *s_off, int T, int D)
+            const int64_t *s_off, int T, int D, int64_t num_chunks)
 {
     constexpr int SG = 32 / LPR;
     const int d4 = D >> 2;
@@ -347,7 +404,7 @@ fixup_small(const u32 *__restrict__ keys, const u32 *__restrict__ seg_start,
     const int sub = wl / LPR, lane = wl % LPR;
     const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
-    const u32 count = counters[CNT_LONG];
+    const u32 count = (u32)min((int64_t)counters[CNT_LONG], num_chunks);
     for (int64_t s = warp; s < count; s += n_warps) {
         const u32 u = long_list[s];
         const u32 a = seg_start[u], e = seg_start[u + 1];
@@ -381,7 +438,7 @@ fixup_big(const u32 *__restrict__ keys, const u32 *__restrict__ seg_start,
     constexpr int NSG = 256 / LPR;
     const int d4 = D >> 2;
     const int sub = threadIdx.x / LPR, lane = threadIdx.x % LPR;
-    const u32 count = counters[CNT_BIG];
+    const u32 count = (u32)min((int64_t)counters[CNT_BIG], num_chunks);
     for (u32 s = blockIdx.x; s < count; s += gridDim.x) {
         const u32 u = long_list[num_chunks - 1 - s];
         const u32 a = seg_start[u], e = seg_start[u + 1];
@@ -445,7 +502,7 @@ seg_fixup_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ seg_start
     __syncthreads();
     fixup_big<LPR, CH>(keys, seg_start, partials, long_list, counters, grad_rows, absmax, row_off, T, D, num_chunks,
                        s_part);
-    fixup_small<LPR, CH>(keys, seg_start, partials, long_list, counters, grad_rows, absmax, s_off, T, D);
+    fixup_small<LPR, CH>(keys, seg_start, partials, long_list, counters, grad_rows, absmax, s_off, T, D, num_chunks);
 }
 
 }  // namespace segred
