@@ -70,7 +70,7 @@ Layout make_layout(const dqrm_ctx *ctx, int64_t L)
     y.pairs_b = take(sizeof(uint2) * Lc);
     y.seg_start = take(sizeof(u32) * (Lc + 1));
     y.chunk_first = take(sizeof(u32) * y.num_chunks);
-    y.long_list = take(sizeof(u32) * y.num_chunks);
+    y.long_list = take(sizeof(uint4) * y.num_chunks);
     y.partials = take(sizeof(double) * y.num_chunks * 2 * ctx->D);
     y.total = o;
     return y;
@@ -263,6 +263,10 @@ seg_emit_kernel(const u32 *__restrict__ keys, int64_t L, const u32 *__restrict__
     int64_t *s_off = reinterpret_cast<int64_t *>(smem_raw);   // [T+1]
     __shared__ u32 wsum[ST_WARPS];
     __shared__ u32 s_prefix;
+    // this thread's keys first: they depend on nothing, so they fly beside the loads of the prefix below
+    const int64_t i0 = (int64_t)blockIdx.x * ST_TILE + (int64_t)threadIdx.x * ST_ITEMS;
+    u32 k[ST_ITEMS], prev0; int n;
+    load_tile_keys(keys, L, i0, k, prev0, n);
     for (int t = threadIdx.x; t <= T; t += ST_THREADS) s_off[t] = row_off[t];
     // heads in all earlier tiles
     u32 p = 0;
@@ -280,9 +284,6 @@ seg_emit_kernel(const u32 *__restrict__ keys, int64_t L, const u32 *__restrict__
     const u32 tile_prefix = s_prefix;
     __syncthreads();
 
-    const int64_t i0 = (int64_t)blockIdx.x * ST_TILE + (int64_t)threadIdx.x * ST_ITEMS;
-    u32 k[ST_ITEMS], prev0; int n;
-    load_tile_keys(keys, L, i0, k, prev0, n);
     u32 c = 0;
     {
         u32 prev = prev0;
@@ -352,7 +353,6 @@ int launch_reduce(dqrm_ctx *ctx, const Layout &y, char *ws, const u32 *keys, con
                   const float *grad_out, float *grad_rows, int64_t L, int64_t G, cudaStream_t st)
 {
     using namespace segred;
-    const size_t smem = (size_t)(ctx->T + 1) * sizeof(int64_t);
     const int64_t cap = (int64_t)ctx->num_sms * 8;
     const int64_t gpb = 256 / RL;                            // one lane group per chunk
     int64_t blocks = (y.num_chunks + gpb - 1) / gpb;
@@ -361,7 +361,7 @@ int launch_reduce(dqrm_ctx *ctx, const Layout &y, char *ws, const u32 *keys, con
     u32 *absmax = reinterpret_cast<u32 *>(ws + y.absmax);
     const u32 *seg_start = reinterpret_cast<const u32 *>(ws + y.seg_start);
     double *partials = reinterpret_cast<double *>(ws + y.partials);
-    u32 *long_list = reinterpret_cast<u32 *>(ws + y.long_list);
+    uint4 *long_list = reinterpret_cast<uint4 *>(ws + y.long_list);
     const size_t red_smem = (size_t)(ctx->T + 1) * sizeof(u32) + (size_t)gpb * 2 * SEG_CHUNK * sizeof(u32);
     if (ctx->D == RL * RV * RC)
         seg_reduce_kernel<RL, RV, RC, true><<<grid, 256, red_smem, st>>>(
@@ -375,7 +375,7 @@ int launch_reduce(dqrm_ctx *ctx, const Layout &y, char *ws, const u32 *keys, con
     dq_mark(ctx, st, DQ_K_SEG_REDUCE);
     int64_t fblocks = (y.num_chunks + 7) / 8;                // at most one cut segment per chunk, a warp each
     int fgrid = (int)(fblocks < (int64_t)ctx->num_sms * 4 ? (fblocks < 1 ? 1 : fblocks) : (int64_t)ctx->num_sms * 4);
-    const size_t fix_smem = (size_t)(256 / LPR) * ctx->D * sizeof(double) + smem;
+    const size_t fix_smem = (size_t)(256 / LPR) * ctx->D * sizeof(double);
     if (fix_smem > 48 * 1024) {
         bool &raised = ctx->smem_raised[dq_smem_slot_fixup(LPR, CH)];
         if (!raised) {
@@ -384,11 +384,40 @@ int launch_reduce(dqrm_ctx *ctx, const Layout &y, char *ws, const u32 *keys, con
             raised = true;
         }
     }
-    seg_fixup_kernel<LPR, CH><<<fgrid, 256, fix_smem, st>>>(keys, seg_start, partials, long_list, counters, grad_rows,
-                                                            absmax, ctx->d_row_off, ctx->T, ctx->D, y.num_chunks);
+    seg_fixup_kernel<LPR, CH><<<fgrid, 256, fix_smem, st>>>(partials, long_list, counters, grad_rows, absmax, ctx->D,
+                                                            y.num_chunks);
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
     dq_mark(ctx, st, DQ_K_SEG_FIXUP);
     return DQRM_OK;
+}
+
+template <int CL>
+cudaError_t launch_cluster_sort(dqrm_ctx *ctx, csort::Args ca, int64_t per_table, cudaStream_t st)
+{
+    ca.cap = csort::choose_cap(per_table, CL);
+    bool &raised = ctx->smem_raised[DQ_SMEM_SLOT_CSORT + (CL == csort::CLUSTER ? 0 : 1)];
+    cudaError_t e = cudaSuccess;
+    if (!raised) {
+        e = cudaFuncSetAttribute(csort::cluster_sort_kernel<CL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)csort::smem_bytes(12288));
+        if (e == cudaSuccess && CL > 8)       // more than eight blocks in a cluster is an opt-in
+            e = cudaFuncSetAttribute(csort::cluster_sort_kernel<CL>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        raised = (e == cudaSuccess);
+    }
+    if (e == cudaSuccess) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(ctx->T * CL));
+        cfg.blockDim = dim3(csort::THREADS);
+        cfg.dynamicSmemBytes = csort::smem_bytes(ca.cap);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = CL; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, csort::cluster_sort_kernel<CL>, ca);
+    }
+    if (e != cudaSuccess) (void)cudaGetLastError();
+    return e;
 }
 
 }  // namespace
@@ -422,7 +451,8 @@ int dq_launch_bwd_sort(dqrm_ctx *ctx, const int32_t *indices, const int32_t *off
     char *ws = reinterpret_cast<char *>(ws_);
     const int64_t G = (int64_t)ctx->T * B;
     if (absmax_bits_out) *absmax_bits_out = reinterpret_cast<const u32 *>(ws + y.absmax);
-    const bool fits_cluster = (L + ctx->T - 1) / ctx->T <= (int64_t)csort::CLUSTER * 12288;
+    const bool fits_cluster = (L + ctx->T - 1) / ctx->T <= (int64_t)csort::CLUSTER * 12288;   // (a table beyond its
+    // blocks' shared memory still sorts, through global staging, but slowly)
     const bool try_cluster = ctx->sort_path != 1 && fits_cluster;
     DQRM_CUDA_TRY(ctx, cudaMemsetAsync(ws, 0, try_cluster ? y.zero_small : y.zero_bytes, st));
     dq_mark(ctx, st, DQ_K_MEMSET);
@@ -438,43 +468,27 @@ int dq_launch_bwd_sort(dqrm_ctx *ctx, const int32_t *indices, const int32_t *off
     bool sorted = false;
     // (tables far beyond the shared-memory slices sort faster with the global radix sort)
     if (try_cluster) {
-        // one eight-block cluster per table; falls through to the global radix sort if the launch is refused
+        // one cluster of eight blocks per table (sixteen when so few tables would leave most SMs idle); falls
+        // through to the narrower cluster, then to the global radix sort, if a launch is refused
         csort::Args ca;
         ca.indices = indices; ca.offsets = offsets; ca.row_off = ctx->d_row_off;
         ca.T = ctx->T; ca.B = B; ca.L = L;
         ca.keys_out = keys[0]; ca.vals_out = vals[0];
         // global staging of (row, payload) pairs, used only by tables too large for shared memory
         ca.gp[0] = reinterpret_cast<uint2 *>(ws + y.pairs_a); ca.gp[1] = reinterpret_cast<uint2 *>(ws + y.pairs_b);
-        ca.cap = csort::choose_cap((L + ctx->T - 1) / ctx->T);
         ca.status = ctx->d_status;
         ca.payload_position = ctx->payload_position;
         ca.tile_heads = reinterpret_cast<u32 *>(ws + y.tile_heads);
-        const size_t smem = csort::smem_bytes(ca.cap);
-        bool &raised = ctx->smem_raised[DQ_SMEM_SLOT_CSORT];
-        cudaError_t e = cudaSuccess;
-        if (!raised) {
-            e = cudaFuncSetAttribute(csort::cluster_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)csort::smem_bytes(12288));
-            raised = (e == cudaSuccess);
-        }
-        if (e == cudaSuccess) {
-            cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3((unsigned)(ctx->T * csort::CLUSTER));
-            cfg.blockDim = dim3(csort::THREADS);
-            cfg.dynamicSmemBytes = smem;
-            cfg.stream = st;
-            cudaLaunchAttribute attr[1];
-            attr[0].id = cudaLaunchAttributeClusterDimension;
-            attr[0].val.clusterDim.x = csort::CLUSTER; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-            cfg.attrs = attr; cfg.numAttrs = 1;
-            e = cudaLaunchKernelEx(&cfg, csort::cluster_sort_kernel, ca);
-        }
+        const int64_t per_table = (L + ctx->T - 1) / ctx->T;
+        const bool wide = ctx->T * csort::CLUSTER_WIDE * 2 <= ctx->num_sms && per_table >= csort::CLUSTER_WIDE * 1024;
+        cudaError_t e = cudaErrorUnknown;
+        if (wide) e = launch_cluster_sort<csort::CLUSTER_WIDE>(ctx, ca, per_table, st);
+        if (e != cudaSuccess) e = launch_cluster_sort<csort::CLUSTER>(ctx, ca, per_table, st);
         if (e == cudaSuccess) {
             dq_mark(ctx, st, DQ_K_CLUSTER_SORT);
             skeys = keys[0];
             sorted = true;
         } else {
-            (void)cudaGetLastError();
             ctx->last_cuda_error = (int)e;
         }
     }

@@ -24,7 +24,8 @@ namespace cg = cooperative_groups;
 
 constexpr int THREADS = 512;
 constexpr int WARPS = THREADS / 32;
-constexpr int CLUSTER = 8;
+constexpr int CLUSTER = 8;            // blocks per table
+constexpr int CLUSTER_WIDE = 16;      // ... when the batch has so few tables that eight blocks each would leave most SMs idle
 constexpr int BINS = 256;
 
 struct Args {
@@ -54,6 +55,7 @@ __device__ __forceinline__ u32 same_digit_lanes(u32 d, bool valid)
     return valid ? peers : 0u;
 }
 
+template <int CL>
 __global__ void __launch_bounds__(THREADS)
 cluster_sort_kernel(const Args a)
 {
@@ -61,11 +63,10 @@ cluster_sort_kernel(const Args a)
     __shared__ u32 s_cnt[WARPS][BINS];
     __shared__ u32 s_hist[BINS];
     __shared__ u32 s_scan[BINS / 32];
-    __shared__ int s_flag;
 
     cg::cluster_group cluster = cg::this_cluster();
     const unsigned c = cluster.block_rank();
-    const int t = blockIdx.x / CLUSTER;
+    const int t = blockIdx.x / CL;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const u32 lt = (1u << lane) - 1u;
 
@@ -78,9 +79,12 @@ cluster_sort_kernel(const Args a)
     if (n == 0) return;
     const int64_t r0 = __ldg(a.row_off + t);
     const int64_t nrows = __ldg(a.row_off + t + 1) - r0;
-    const int npc = (int)(((n + CLUSTER - 1) / CLUSTER + 31) / 32 * 32);      // pairs per block
+    const int npc = (int)(((n + CL - 1) / CL + 31) / 32 * 32);      // pairs per block
     const bool in_smem = npc <= a.cap;
     const int my_n = (int)max((int64_t)0, min((int64_t)npc, n - (int64_t)c * npc));
+    // the scatter divides every destination by npc: a float reciprocal gives the quotient (a block number,
+    // since pos < n <= CL * npc) to within one, and one correction step settles it
+    const float npc_inv = 1.0f / (float)npc;
 
     // buffers of this block for stage s (shared memory slices, or this block's part of the global staging)
     // a pair travels as one 8-byte store: distributed-shared-memory traffic is bound by the number of stores
@@ -90,48 +94,40 @@ cluster_sort_kernel(const Args a)
     } else {
         pb0 = a.gp[0] + tb0 + (int64_t)c * npc; pb1 = a.gp[1] + tb0 + (int64_t)c * npc;
     }
-    // ---- are this table's bags all one-index bags in order (offsets = identity)? ----
-    // Any other batch has its offsets checked here: they must not decrease inside the table, so that
-    // the search for a lookup's bag below walks an ordered list.
-    {
-        if (threadIdx.x == 0) s_flag = 1;
-        __syncthreads();
-        int ok = 1;
-        const int per = (a.B + CLUSTER - 1) / CLUSTER;
-        const int b0 = c * per, b1 = min(a.B, b0 + per);
-        const int32_t *off_t = a.offsets + (int64_t)t * a.B;
-        if (n != a.B) {
-            ok = 0;
-            bool dec = false;
-            for (int i = b0 + threadIdx.x; i < b1; i += THREADS) dec |= __ldg(off_t + i) > __ldg(off_t + i + 1);
-            if (dec) dq_report(a.status, DQRM_ERR_INDEX_RANGE);
-        } else {
-            for (int i = b0 + threadIdx.x; i < b1; i += THREADS)
-                if ((int64_t)__ldg(off_t + i) != tb0 + i) ok = 0;
-        }
-        if (!ok) s_flag = 0;
-        if (blockIdx.x == 0 && threadIdx.x == 0 &&
-            (__ldg(a.offsets) != 0 || (int64_t)__ldg(a.offsets + (int64_t)a.T * a.B) != a.L))
-            dq_report(a.status, DQRM_ERR_INDEX_RANGE);
-        __syncthreads();
-    }
-    cluster.sync();
-    bool onehot = true;
-    for (unsigned cc = 0; cc < CLUSTER; ++cc) onehot &= (*cluster.map_shared_rank(&s_flag, cc) != 0);
     // ---- load this block's slice: key = row within the table, payload = row of grad_out ----
+    // In a table of one-index bags in order (n == B and offsets = identity, the Criteo-shaped case) the bag of
+    // the lookup at position p is bag p.  That is checked per lookup from the two offsets around it, which are
+    // loaded together with the index, so nothing here waits on another block.  Any other lookup finds its
+    // bag by a search of the offsets, which must not decrease inside the table.
+    const int32_t *off_t = a.offsets + (int64_t)t * a.B;
+    if (n != a.B) {
+        bool dec = false;
+        const int per = (a.B + CL - 1) / CL;
+        const int b0 = c * per, b1 = min(a.B, b0 + per);
+        for (int i = b0 + threadIdx.x; i < b1; i += THREADS) dec |= __ldg(off_t + i) > __ldg(off_t + i + 1);
+        if (dec) dq_report(a.status, DQRM_ERR_INDEX_RANGE);
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0 &&
+        (__ldg(a.offsets) != 0 || (int64_t)__ldg(a.offsets + (int64_t)a.T * a.B) != a.L))
+        dq_report(a.status, DQRM_ERR_INDEX_RANGE);
     bool bad = false;
     for (int i = threadIdx.x; i < my_n; i += THREADS) {
         const int64_t p = (int64_t)c * npc + i;    // position within the table's lookups
         int32_t idx = __ldg(a.indices + tb0 + p);
+        bool single = false;
+        if (n == a.B) {
+            const int64_t o0 = __ldg(off_t + p), o1 = __ldg(off_t + p + 1);
+            single = o0 == tb0 + p && o1 == tb0 + p + 1;
+            if (o0 > o1) dq_report(a.status, DQRM_ERR_INDEX_RANGE);
+        }
         bad |= (idx < 0) | (idx >= nrows);
         idx = (int32_t)min((int64_t)max(idx, 0), nrows - 1);
         int64_t bag = p;
-        if (!onehot) {                             // largest bag b with offsets[t*B + b] <= tb0 + p
+        if (!single) {                             // largest bag b with offsets[t*B + b] <= tb0 + p
             int lo = 0, hi = a.B;
-            const int32_t *off = a.offsets + (int64_t)t * a.B;
             while (hi - lo > 1) {
                 int mid = (lo + hi) >> 1;
-                if ((int64_t)__ldg(off + mid) <= tb0 + p) lo = mid; else hi = mid;
+                if ((int64_t)__ldg(off_t + mid) <= tb0 + p) lo = mid; else hi = mid;
             }
             bag = lo;
         }
@@ -171,11 +167,11 @@ cluster_sort_kernel(const Args a)
         // offsets: digits first, then blocks of the cluster, then warps of this block
         u32 tot = 0, pre = 0, incl = 0;
         if (threadIdx.x < BINS) {                  // one thread per digit (the first BINS / 32 warps)
-            u32 h[CLUSTER];
+            u32 h[CL];
 #pragma unroll
-            for (unsigned cc = 0; cc < CLUSTER; ++cc) h[cc] = *remote(cluster, &s_hist[threadIdx.x], cc);
+            for (unsigned cc = 0; cc < CL; ++cc) h[cc] = *remote(cluster, &s_hist[threadIdx.x], cc);
 #pragma unroll
-            for (unsigned cc = 0; cc < CLUSTER; ++cc) { if (cc < c) pre += h[cc]; tot += h[cc]; }
+            for (unsigned cc = 0; cc < CL; ++cc) { if (cc < c) pre += h[cc]; tot += h[cc]; }
             incl = tot;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -214,7 +210,9 @@ cluster_sort_kernel(const Args a)
                 const u32 pos = base + __popc(peers & lt);      // position within the table, < n
                 if ((int64_t)pos < n) {
                     if (in_smem) {
-                        const unsigned owner = pos / npc;
+                        unsigned owner = (unsigned)((float)pos * npc_inv);       // within one of pos / npc
+                        if (owner * (u32)npc > pos) --owner;
+                        else if ((owner + 1u) * (u32)npc <= pos) ++owner;
                         const u32 j = pos - owner * npc;
                         cluster.map_shared_rank(dst, owner)[j] = pr;
                     } else {
@@ -263,10 +261,10 @@ cluster_sort_kernel(const Args a)
 
 inline size_t smem_bytes(int cap) { return (size_t)2 * cap * sizeof(uint2); }
 
-// pairs per block to provision in shared memory for an expected n per table
-inline int choose_cap(int64_t expect_n)
+// pairs per block to provision in shared memory for an expected n per table sorted by `cluster` blocks
+inline int choose_cap(int64_t expect_n, int cluster)
 {
-    int64_t npc = ((expect_n + CLUSTER - 1) / CLUSTER + 31) / 32 * 32;
+    int64_t npc = ((expect_n + cluster - 1) / cluster + 31) / 32 * 32;
     int64_t cap = (npc + npc / 4 + 31) / 32 * 32;         // 25 % head room for uneven tables
     if (cap < 256) cap = 256;
     if (cap > 12288) cap = 12288;                         // 192 KB of the 227 KB a block may use

@@ -119,7 +119,7 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
                   const u32 *__restrict__ seg_start, const u32 *__restrict__ chunk_first,
                   const int32_t *__restrict__ uniq_off,
                   const float *__restrict__ grad_out, float *__restrict__ grad_rows,
-                  double *__restrict__ partials, u32 *__restrict__ long_list, u32 *__restrict__ counters,
+                  double *__restrict__ partials, uint4 *__restrict__ long_list, u32 *__restrict__ counters,
                   u32 *__restrict__ absmax, int T, int D_any,
                   int64_t L, int64_t G, int64_t num_chunks, int *__restrict__ status)
 {
@@ -288,17 +288,24 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
                     }
                 }
                 if (begins && lane == 0) {
+                    // the segment begins here: leave all the fix-up needs to know about it in one record
                     const u32 sa = seg_start[u], sb = seg_start[u + 1];
                     const u32 npieces = (sb - 1) / CHUNK - sa / CHUNK + 1;
+                    int lo = 0, hi = T;              // its table: largest t with s_uoff[t] <= u
+                    while (hi - lo > 1) {
+                        const int mid = (lo + hi) >> 1;
+                        if (s_uoff[mid] <= u) lo = mid; else hi = mid;
+                    }
+                    const uint4 rec = make_uint4(u, sa / CHUNK, npieces, (u32)lo);
                     // (the list has a slot per chunk and every chunk begins at most one such segment; the bound only
                     // matters for a workspace that is summed twice without a sort in between, which must not write
                     // outside the list)
                     if (npieces > BIG_PIECES) {
                         const u32 k = atomicAdd(&counters[CNT_BIG], 1u);
-                        if ((int64_t)k < num_chunks) long_list[num_chunks - 1 - k] = u;
+                        if ((int64_t)k < num_chunks) long_list[num_chunks - 1 - k] = rec;
                     } else {
                         const u32 k = atomicAdd(&counters[CNT_LONG], 1u);
-                        if ((int64_t)k < num_chunks) long_list[k] = u;
+                        if ((int64_t)k < num_chunks) long_list[k] = rec;
                     }
                 }
             }
@@ -351,12 +358,11 @@ __device__ __forceinline__ const double *piece_ptr(const double *partials, int64
     return partials + ((size_t)(c0 + p) * 2 + (p == 0 ? 1 : 0)) * D;
 }
 
-template <int CH>
+template <int CH, int UN>
 __device__ __forceinline__ void add_pieces(double (&acc)[CH][4], const double *partials, int64_t c0,
                                            int64_t p_begin, int64_t p_end, int64_t stride, int D, int lane,
                                            int lpr, int d4)
 {
-    constexpr int UN = 4;
     for (int64_t p = p_begin; p < p_end; p += stride * UN) {
         double2 x[UN][CH], y[UN][CH];
 #pragma unroll
@@ -390,13 +396,13 @@ __device__ __forceinline__ void add_pieces(double (&acc)[CH][4], const double *p
     }
 }
 
-// one warp per cut segment of at most BIG_PIECES pieces
+// A record of the list: x = segment (unique row), y = chunk in which it begins, z = number of pieces, w = table.
+
+// one warp per listed segment of at most BIG_PIECES pieces
 template <int LPR, int CH>
 __device__ __forceinline__ void
-fixup_small(const u32 *__restrict__ keys, const u32 *__restrict__ seg_start,
-            const double *__restrict__ partials, const u32 *__restrict__ long_list,
-            const u32 *__restrict__ counters, float *__restrict__ grad_rows, u32 *__restrict__ absmax,
-            const int64_t *s_off, int T, int D, int64_t num_chunks)
+fixup_small(const double *__restrict__ partials, const uint4 *__restrict__ long_list, u32 count,
+            float *__restrict__ grad_rows, u32 *__restrict__ absmax, int D)
 {
     constexpr int SG = 32 / LPR;
     const int d4 = D >> 2;
@@ -404,15 +410,12 @@ fixup_small(const u32 *__restrict__ keys, const u32 *__restrict__ seg_start,
     const int sub = wl / LPR, lane = wl % LPR;
     const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
-    const u32 count = (u32)min((int64_t)counters[CNT_LONG], num_chunks);
     for (int64_t s = warp; s < count; s += n_warps) {
-        const u32 u = long_list[s];
-        const u32 a = seg_start[u], e = seg_start[u + 1];
-        const int64_t c0 = a / CHUNK, c1 = (e - 1) / CHUNK;
+        const uint4 rec = __ldcg(long_list + s);
         double acc[CH][4];
 #pragma unroll
         for (int ch = 0; ch < CH; ++ch) acc[ch][0] = acc[ch][1] = acc[ch][2] = acc[ch][3] = 0.0;
-        add_pieces<CH>(acc, partials, c0, sub, c1 - c0 + 1, SG, D, lane, LPR, d4);
+        add_pieces<CH, 4>(acc, partials, rec.y, sub, rec.z, SG, D, lane, LPR, d4);
 #pragma unroll
         for (int o = LPR; o < 32; o <<= 1)
 #pragma unroll
@@ -420,33 +423,29 @@ fixup_small(const u32 *__restrict__ keys, const u32 *__restrict__ seg_start,
 #pragma unroll
                 for (int q = 0; q < 4; ++q) acc[ch][q] += __shfl_xor_sync(0xffffffffu, acc[ch][q], o);
         float m = 0.f;
-        if (sub == 0) m = round_store<CH>(acc, grad_rows + (int64_t)u * D, lane, LPR, d4);
+        if (sub == 0) m = round_store<CH>(acc, grad_rows + (int64_t)rec.x * D, lane, LPR, d4);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-        if (wl == 0 && m > 0.f) atomicMax(&absmax[dq_table_of(s_off, T, (int64_t)keys[a])], __float_as_uint(m));
+        if (wl == 0 && m > 0.f) atomicMax(&absmax[rec.w], __float_as_uint(m));
     }
 }
 
-// one block per cut segment of more than BIG_PIECES pieces (hot rows)
+// one block per listed segment of more than BIG_PIECES pieces (the hottest rows)
 template <int LPR, int CH>
 __device__ __forceinline__ void
-fixup_big(const u32 *__restrict__ keys, const u32 *__restrict__ seg_start,
-          const double *__restrict__ partials, const u32 *__restrict__ long_list,
-          const u32 *__restrict__ counters, float *__restrict__ grad_rows, u32 *__restrict__ absmax,
-          const int64_t *__restrict__ row_off, int T, int D, int64_t num_chunks, double *s_part /*[256/LPR][D]*/)
+fixup_big(const double *__restrict__ partials, const uint4 *__restrict__ long_list, u32 count,
+          float *__restrict__ grad_rows, u32 *__restrict__ absmax, int D, int64_t num_chunks,
+          double *s_part /*[256/LPR][D]*/)
 {
     constexpr int NSG = 256 / LPR;
     const int d4 = D >> 2;
     const int sub = threadIdx.x / LPR, lane = threadIdx.x % LPR;
-    const u32 count = (u32)min((int64_t)counters[CNT_BIG], num_chunks);
     for (u32 s = blockIdx.x; s < count; s += gridDim.x) {
-        const u32 u = long_list[num_chunks - 1 - s];
-        const u32 a = seg_start[u], e = seg_start[u + 1];
-        const int64_t c0 = a / CHUNK, c1 = (e - 1) / CHUNK;
+        const uint4 rec = __ldcg(long_list + (num_chunks - 1 - s));
         double acc[CH][4];
 #pragma unroll
         for (int ch = 0; ch < CH; ++ch) acc[ch][0] = acc[ch][1] = acc[ch][2] = acc[ch][3] = 0.0;
-        add_pieces<CH>(acc, partials, c0, sub, c1 - c0 + 1, NSG, D, lane, LPR, d4);
+        add_pieces<CH, (CH == 1 ? 8 : 4)>(acc, partials, rec.y, sub, rec.z, NSG, D, lane, LPR, d4);
         __syncthreads();
 #pragma unroll
         for (int ch = 0; ch < CH; ++ch) {
@@ -470,39 +469,30 @@ fixup_big(const u32 *__restrict__ keys, const u32 *__restrict__ seg_start,
                         t0 += src[0]; t1 += src[1]; t2 += src[2]; t3 += src[3];
                     }
                     float4 r = make_float4((float)t0, (float)t1, (float)t2, (float)t3);
-                    *reinterpret_cast<float4 *>(grad_rows + (int64_t)u * D + 4 * c4) = r;
+                    *reinterpret_cast<float4 *>(grad_rows + (int64_t)rec.x * D + 4 * c4) = r;
                     m = fmaxf(fmaxf(m, fmaxf(fabsf(r.x), fabsf(r.y))), fmaxf(fabsf(r.z), fabsf(r.w)));
                 }
             }
             m = group_max<LPR>(m);
-            if (lane == 0 && m > 0.f) {
-                // row_off is read from global memory here: this path runs for a handful of hot rows
-                int lo = 0, hi = T;
-                const int64_t key = (int64_t)keys[a];
-                while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (row_off[mid] <= key) lo = mid; else hi = mid; }
-                atomicMax(&absmax[lo], __float_as_uint(m));
-            }
+            if (lane == 0 && m > 0.f) atomicMax(&absmax[rec.w], __float_as_uint(m));
         }
     }
 }
 
-// both fix-ups in one launch: every block first takes its share of the hot rows, then its
-// warps take the short cut segments
+// both fix-ups in one launch: every block first takes its share of the hottest rows, then its
+// warps take the other listed segments
 template <int LPR, int CH>
 __global__ void __launch_bounds__(256)
-seg_fixup_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ seg_start,
-                 const double *__restrict__ partials, const u32 *__restrict__ long_list,
+seg_fixup_kernel(const double *__restrict__ partials, const uint4 *__restrict__ long_list,
                  const u32 *__restrict__ counters, float *__restrict__ grad_rows, u32 *__restrict__ absmax,
-                 const int64_t *__restrict__ row_off, int T, int D, int64_t num_chunks)
+                 int D, int64_t num_chunks)
 {
     extern __shared__ unsigned char smem_raw[];
     double *s_part = reinterpret_cast<double *>(smem_raw);                         // [256/LPR][D]
-    int64_t *s_off = reinterpret_cast<int64_t *>(s_part + (size_t)(256 / LPR) * D);  // [T+1]
-    for (int t = threadIdx.x; t <= T; t += blockDim.x) s_off[t] = row_off[t];
-    __syncthreads();
-    fixup_big<LPR, CH>(keys, seg_start, partials, long_list, counters, grad_rows, absmax, row_off, T, D, num_chunks,
-                       s_part);
-    fixup_small<LPR, CH>(keys, seg_start, partials, long_list, counters, grad_rows, absmax, s_off, T, D, num_chunks);
+    const u32 n_big = (u32)min((int64_t)__ldcg(counters + CNT_BIG), num_chunks);
+    const u32 n_small = (u32)min((int64_t)__ldcg(counters + CNT_LONG), num_chunks);
+    fixup_big<LPR, CH>(partials, long_list, n_big, grad_rows, absmax, D, num_chunks, s_part);
+    fixup_small<LPR, CH>(partials, long_list, n_small, grad_rows, absmax, D);
 }
 
 }  // namespace segred

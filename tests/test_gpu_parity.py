@@ -30,6 +30,8 @@ def _cases():
         "sweep_d32_b4_zipf": W.sweep(D=32, bits=4, zipf=True, rows=200_000, B=5000),
         "sweep_d64_b8_uniform": W.sweep(D=64, bits=8, zipf=False, rows=100_000, B=3000),
         "sweep_d128_b8_zipf": W.sweep(D=128, bits=8, zipf=True, rows=50_000, B=3000),
+        # one table with enough lookups for the sixteen-block sort cluster; 20,000 is no multiple of 16 * 32
+        "sweep_d16_b4_zipf_wide": W.sweep(D=16, bits=4, zipf=True, rows=300_000, B=20_000),
         # feature sizes that are not a power of two / need several vectors per lane
         "odd_d20": replace(W.scaled_down(kg, total_rows=50_000, B=333), D=20, name="odd_d20"),
         "wide_d384": W.Workload("wide_d384", (700, 90, 5000), D=384, B=257, alpha=1.1, bits=8),
