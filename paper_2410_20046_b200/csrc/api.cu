@@ -19,7 +19,8 @@ inline bool batch_ok(const dqrm_ctx *ctx, int B, int64_t L)
 }
 
 struct HostStepLayout {
-    size_t indices, offsets, grad_out, out, unique_rows, uniq_off, grad_rows, codes, grad_scales, step_ws, total;
+    size_t indices[2], offsets[2], grad_out[2], out[2];      // two sets of staging buffers, used by alternate calls
+    size_t unique_rows, uniq_off, grad_rows, codes, grad_scales, step_ws, total;
 };
 
 HostStepLayout host_layout(const dqrm_ctx *ctx, int64_t L, int64_t G)
@@ -28,10 +29,12 @@ HostStepLayout host_layout(const dqrm_ctx *ctx, int64_t L, int64_t G)
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
     const int64_t Lc = L < 1 ? 1 : L;
-    y.indices = take(sizeof(int32_t) * Lc);
-    y.offsets = take(sizeof(int32_t) * (G + 1));
-    y.grad_out = take(sizeof(float) * G * ctx->D);
-    y.out = take(sizeof(float) * G * ctx->D);
+    for (int k = 0; k < 2; ++k) {
+        y.indices[k] = take(sizeof(int32_t) * Lc);
+        y.offsets[k] = take(sizeof(int32_t) * (G + 1));
+        y.grad_out[k] = take(sizeof(float) * G * ctx->D);
+        y.out[k] = take(sizeof(float) * G * ctx->D);
+    }
     y.unique_rows = take(sizeof(int32_t) * Lc);
     y.uniq_off = take(sizeof(int32_t) * (ctx->T + 1));
     y.grad_rows = take(sizeof(float) * Lc * ctx->D);
@@ -88,6 +91,9 @@ int dqrm_create(dqrm_ctx **out, int T, int D, const int64_t *h_row_off)
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_h_go, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_h_fwd, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_h_out, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_h_free[0], cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_h_free[1], cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_h_idx, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaMemcpy(ctx->d_row_off, h_row_off, sizeof(int64_t) * (T + 1), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(ctx->d_done, 0, sizeof(u32));
@@ -118,6 +124,9 @@ int dqrm_destroy(dqrm_ctx *ctx)
     if (ctx->ev_h_go) cudaEventDestroy(ctx->ev_h_go);
     if (ctx->ev_h_fwd) cudaEventDestroy(ctx->ev_h_fwd);
     if (ctx->ev_h_out) cudaEventDestroy(ctx->ev_h_out);
+    if (ctx->ev_h_free[0]) cudaEventDestroy(ctx->ev_h_free[0]);
+    if (ctx->ev_h_free[1]) cudaEventDestroy(ctx->ev_h_free[1]);
+    if (ctx->ev_h_idx) cudaEventDestroy(ctx->ev_h_idx);
     if (ctx->prof_events) {
         for (int i = 0; i < DQ_PROF_MAX; ++i) cudaEventDestroy(ctx->prof_events[i]);
         delete[] ctx->prof_events;
@@ -452,18 +461,19 @@ int dqrm_train_step_host(dqrm_ctx *ctx, float *tables, const int32_t *h_indices,
     if (!ws_ok(workspace, workspace_bytes, y.total)) return DQRM_ERR_WORKSPACE;
     char *ws = reinterpret_cast<char *>(workspace);
     cudaStream_t st = as_stream(stream);
-    int32_t *d_idx = reinterpret_cast<int32_t *>(ws + y.indices);
-    int32_t *d_off = reinterpret_cast<int32_t *>(ws + y.offsets);
-    float *d_go = reinterpret_cast<float *>(ws + y.grad_out);
-    float *d_out = reinterpret_cast<float *>(ws + y.out);
+    const bool plain = !ctx->overlap || ctx->prof_on || L == 0;        // everything in order on the caller's stream
+    const int set = plain ? 0 : (int)(ctx->host_calls++ & 1u);
+    int32_t *d_idx = reinterpret_cast<int32_t *>(ws + y.indices[set]);
+    int32_t *d_off = reinterpret_cast<int32_t *>(ws + y.offsets[set]);
+    float *d_go = reinterpret_cast<float *>(ws + y.grad_out[set]);
+    float *d_out = reinterpret_cast<float *>(ws + y.out[set]);
     int32_t *d_ur = reinterpret_cast<int32_t *>(ws + y.unique_rows);
     int32_t *d_uo = reinterpret_cast<int32_t *>(ws + y.uniq_off);
     float *d_gr = reinterpret_cast<float *>(ws + y.grad_rows);
     int8_t *d_codes = reinterpret_cast<int8_t *>(ws + y.codes);
     float *d_gs = reinterpret_cast<float *>(ws + y.grad_scales);
     const size_t go_bytes = sizeof(float) * G * ctx->D;
-    if (!ctx->overlap || ctx->prof_on || L == 0) {
-        // everything in order on the caller's stream
+    if (plain) {
         if (L > 0) DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(d_idx, h_indices, sizeof(int32_t) * L, cudaMemcpyHostToDevice, st));
         DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(d_off, h_offsets, sizeof(int32_t) * (G + 1), cudaMemcpyHostToDevice, st));
         DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(d_go, h_grad_out, go_bytes, cudaMemcpyHostToDevice, st));
@@ -476,13 +486,20 @@ int dqrm_train_step_host(dqrm_ctx *ctx, float *tables, const int32_t *h_indices,
     // The two large transfers go in opposite directions and neither is needed where the other is: the upstream
     // gradient (host to device) is first read by the gradient summation, the pooled output (device to host) is
     // complete once the forward is.  Each gets a stream of the context, so that they overlap each other, the index
-    // sort and the forward; the caller's stream waits for both before the call's work on it is complete.
-    DQRM_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_h_start, st));          // the staging buffers' previous users are done
-    DQRM_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->copy_in, ctx->ev_h_start, 0));
+    // sort and the forward.  The inputs of this call land in the staging set that the call before the last one used,
+    // as soon as that call is over: they do not wait for the previous call, whose kernels and output copy they
+    // overlap.  The caller's stream waits for everything before the call's work on it is complete.
+    if (ctx->h_set_used[set]) DQRM_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->copy_in, ctx->ev_h_free[set], 0));
+    else {      // first use of this set: only what the caller's stream already holds comes first
+        DQRM_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_h_start, st));
+        DQRM_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->copy_in, ctx->ev_h_start, 0));
+    }
+    DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(d_idx, h_indices, sizeof(int32_t) * L, cudaMemcpyHostToDevice, ctx->copy_in));
+    DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(d_off, h_offsets, sizeof(int32_t) * (G + 1), cudaMemcpyHostToDevice, ctx->copy_in));
+    DQRM_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_h_idx, ctx->copy_in));
     DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(d_go, h_grad_out, go_bytes, cudaMemcpyHostToDevice, ctx->copy_in));
     DQRM_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_h_go, ctx->copy_in));
-    DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(d_idx, h_indices, sizeof(int32_t) * L, cudaMemcpyHostToDevice, st));
-    DQRM_CUDA_TRY(ctx, cudaMemcpyAsync(d_off, h_offsets, sizeof(int32_t) * (G + 1), cudaMemcpyHostToDevice, st));
+    DQRM_CUDA_TRY(ctx, cudaStreamWaitEvent(st, ctx->ev_h_idx, 0));
     DQRM_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_fork, st));
     DQRM_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
     char *step_ws = ws + y.step_ws;
@@ -502,6 +519,8 @@ int dqrm_train_step_host(dqrm_ctx *ctx, float *tables, const int32_t *h_indices,
     if (rc == DQRM_OK)
         rc = dq_launch_quant_update(ctx, tables, d_ur, d_uo, d_gr, dq_bwd_absmax_bits(ctx, L, step_ws), d_codes, d_gs, lr, st);
     cudaStreamWaitEvent(st, ctx->ev_h_out, 0);
+    cudaEventRecord(ctx->ev_h_free[set], st);        // the staging set is free for the call after the next one
+    ctx->h_set_used[set] = true;
     if (rc != DQRM_OK) return rc;
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
     return DQRM_OK;

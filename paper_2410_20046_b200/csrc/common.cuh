@@ -26,6 +26,10 @@ struct dqrm_ctx {
     // host-buffer step: the upstream gradient comes in and the pooled output goes out on streams of their own
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
     cudaEvent_t ev_h_start = nullptr, ev_h_go = nullptr, ev_h_fwd = nullptr, ev_h_out = nullptr;
+    // ... with two sets of staging buffers used alternately: a set is free again when the call that used it is over
+    cudaEvent_t ev_h_free[2] = {nullptr, nullptr}, ev_h_idx = nullptr;
+    bool h_set_used[2] = {false, false};
+    unsigned host_calls = 0;
     int overlap = 1;                // 0: keep everything on the caller's stream
     int payload_position = 0;       // sort payload: 0 = row of grad_out, 1 = position of the lookup (set by the merge)
     // kernels whose dynamic shared-memory limit has been raised on this context's device (the attribute is

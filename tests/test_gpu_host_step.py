@@ -1,6 +1,6 @@
 """GPU parity of dqrm_train_step_host (host buffers in, pooled output back to the host, transfers on
 streams of the context beside the kernels) against the oracle, over consecutive calls that reuse
-the staging buffers, with and without the overlap."""
+the two sets of staging buffers in turn, with and without the overlap."""
 import numpy as np
 import pytest
 
@@ -25,7 +25,7 @@ def test_host_step_equals_oracle(oracle, name, overlap):
     c.ctx.scale_refresh(d_tables, c.bits, scales)
     torch.cuda.synchronize()
     o_scales, _ = oracle.scale_refresh(o_tables, c.row_off, wl.D, c.bits_np)
-    steps = 4
+    steps = 6          # both staging sets are used three times
     batches = [c.batch(s) for s in range(steps)]
     pinned = [tuple(torch.from_numpy(np.ascontiguousarray(a)).pin_memory() for a in b) for b in batches]
     outs = [torch.full((wl.B, wl.T, wl.D), float("nan"), dtype=torch.float32).pin_memory() for _ in range(steps)]
