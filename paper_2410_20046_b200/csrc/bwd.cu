@@ -30,15 +30,15 @@ constexpr int ST_ITEMS = 8;
 constexpr int ST_TILE = ST_THREADS * ST_ITEMS;   // 2048 entries per tile
 constexpr int ST_WARPS = ST_THREADS / 32;
 constexpr int NB_MAX = 512;                      // bins per pass (<= 9 bit digits)
-constexpr int MAX_PASSES = 4;
+constexpr int HIST_CHUNK = 64;                   // tiles per chunk of the radix sort's offset computation
 constexpr int SEG_CHUNK = segred::CHUNK;         // sorted entries per reduce work item
 
 struct Layout {
     int passes, digit_bits, nb;
     int64_t num_tiles, num_chunks;
-    // zeroed at call start: [0, zero_small) always, [0, zero_bytes) by the radix path
-    size_t absmax, counters, tile_heads, zero_small, ghist, tilehist_a, zero_bytes;
-    size_t tilehist_b, keys_a, keys_b, vals_a, vals_b, pairs_a, pairs_b, seg_start, chunk_first, long_list, partials;
+    // zeroed at call start: [0, zero_small)
+    size_t absmax, counters, tile_heads, zero_small, digit_base, chunk_sum, tilehist;
+    size_t keys_a, vals_a, pairs_a, pairs_b, seg_start, chunk_first, long_list, partials;
     size_t total;
 };
 
@@ -58,14 +58,11 @@ Layout make_layout(const dqrm_ctx *ctx, int64_t L)
     y.counters = take(sizeof(u32) * 8);
     y.tile_heads = take(sizeof(u32) * y.num_tiles);
     y.zero_small = o;
-    y.ghist = take(sizeof(u32) * MAX_PASSES * NB_MAX);
-    y.tilehist_a = take(sizeof(u32) * y.nb * y.num_tiles);
-    y.zero_bytes = o;
-    y.tilehist_b = take(sizeof(u32) * y.nb * y.num_tiles);
+    y.digit_base = take(sizeof(u32) * NB_MAX);
+    y.chunk_sum = take(sizeof(u32) * y.nb * ((y.num_tiles + HIST_CHUNK - 1) / HIST_CHUNK));
+    y.tilehist = take(sizeof(u32) * y.nb * y.num_tiles);
     y.keys_a = take(sizeof(u32) * Lc);
-    y.keys_b = take(sizeof(u32) * Lc);
     y.vals_a = take(sizeof(u32) * Lc);
-    y.vals_b = take(sizeof(u32) * Lc);
     y.pairs_a = take(sizeof(uint2) * Lc);
     y.pairs_b = take(sizeof(uint2) * Lc);
     y.seg_start = take(sizeof(u32) * (Lc + 1));
@@ -80,17 +77,13 @@ Layout make_layout(const dqrm_ctx *ctx, int64_t L)
 using segred::CNT_U;
 
 // ---------------------------------------------------------------------------------
+// one thread per bag: (arena-row key, gradient-row payload) of every lookup of the bag, as one 8-byte pair:
+// the passes move pairs, so that a digit's short run in a tile still leaves as whole 32-byte sectors
 __global__ void __launch_bounds__(256)
 prepare_kernel(const int32_t *__restrict__ indices, const int32_t *__restrict__ offsets,
                const int64_t *__restrict__ row_off, int T, int B, int64_t G, int64_t L,
-               u32 *__restrict__ keys, u32 *__restrict__ vals, u32 *__restrict__ ghist,
-               u32 *__restrict__ tilehist0, int64_t num_tiles, int passes, int digit_bits,
-               int payload_position, int *__restrict__ status)
+               uint2 *__restrict__ pairs, int payload_position, int *__restrict__ status)
 {
-    __shared__ u32 sh[MAX_PASSES * NB_MAX];
-    for (int i = threadIdx.x; i < MAX_PASSES * NB_MAX; i += blockDim.x) sh[i] = 0;
-    __syncthreads();
-    const u32 mask = (1u << digit_bits) - 1u;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         if (__ldg(offsets) != 0 || (int64_t)__ldg(offsets + G) != L) dq_report(status, DQRM_ERR_INDEX_RANGE);
     }
@@ -107,55 +100,95 @@ prepare_kernel(const int32_t *__restrict__ indices, const int32_t *__restrict__ 
                 dq_report(status, DQRM_ERR_INDEX_RANGE);
                 idx = idx < 0 ? 0 : (int32_t)(nrows - 1);
             }
-            const u32 key = (u32)(r0 + idx);
-            keys[j] = key;
-            vals[j] = payload_position ? (u32)j : payload;
-            for (int p = 0; p < passes; ++p) atomicAdd(&sh[p * NB_MAX + ((key >> (p * digit_bits)) & mask)], 1u);
-            atomicAdd(&tilehist0[(size_t)(key & mask) * num_tiles + j / ST_TILE], 1u);
+            pairs[j] = make_uint2((u32)(r0 + idx), payload_position ? (u32)j : payload);
         }
     }
-    __syncthreads();
-    for (int i = threadIdx.x; i < MAX_PASSES * NB_MAX; i += blockDim.x)
-        if (sh[i]) atomicAdd(&ghist[i], sh[i]);
 }
 
-// one warp per digit: exclusive scan over tiles, plus the digit's global base
-__global__ void __launch_bounds__(256)
-sort_scan_kernel(u32 *__restrict__ tilehist, const u32 *__restrict__ ghist_p, int nb, int64_t num_tiles,
-                 u32 *__restrict__ next_tilehist, int64_t next_count)
+// Per pass, three small kernels turn the digit counts of every tile of 2048 entries into the scatter's
+// offsets without a single global atomic: tilehist[tile][digit] counts; a thread per digit then walks the
+// 64 tiles of a chunk and leaves the running count in their place and the chunk's total in
+// chunk_sum[chunk][digit]; one block does the same over the chunks and scans the digits' totals.  The
+// scatter adds the three: digit base + chunks before + tiles before within the chunk.
+__global__ void __launch_bounds__(ST_THREADS)
+sort_hist_kernel(const uint2 *__restrict__ pairs, int64_t L, int shift, int nb, u32 *__restrict__ tilehist)
 {
-    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t i = tid; i < next_count; i += nthreads) next_tilehist[i] = 0u;
-    const int b = (int)(tid >> 5);
-    const int lane = threadIdx.x & 31;
-    if (b >= nb) return;
-    u32 sum = 0;
-    for (int bb = lane; bb < b; bb += 32) sum += ghist_p[bb];
+    __shared__ u32 cnt[NB_MAX];
+    for (int i = threadIdx.x; i < nb; i += ST_THREADS) cnt[i] = 0u;
+    __syncthreads();
+    const u32 mask = (u32)nb - 1u;
+    const int64_t base = (int64_t)blockIdx.x * ST_TILE + threadIdx.x;
+    u32 key[ST_ITEMS];
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    u32 carry = sum;
-    u32 *row = tilehist + (size_t)b * num_tiles;
-    for (int64_t t0 = 0; t0 < num_tiles; t0 += 32) {
-        int64_t i = t0 + lane;
-        u32 c = i < num_tiles ? row[i] : 0u;
-        u32 incl = c;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            u32 n = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += n;
-        }
-        if (i < num_tiles) row[i] = carry + incl - c;
-        carry += __shfl_sync(0xffffffffu, incl, 31);
+    for (int k = 0; k < ST_ITEMS; ++k) {
+        const int64_t i = base + (int64_t)k * ST_THREADS;
+        key[k] = i < L ? pairs[i].x : 0u;
     }
+#pragma unroll
+    for (int k = 0; k < ST_ITEMS; ++k)
+        if (base + (int64_t)k * ST_THREADS < L) atomicAdd(&cnt[(key[k] >> shift) & mask], 1u);
+    __syncthreads();
+    for (int i = threadIdx.x; i < nb; i += ST_THREADS) tilehist[(size_t)blockIdx.x * nb + i] = cnt[i];
+}
+
+// block = chunk of HIST_CHUNK tiles, thread = digit
+__global__ void __launch_bounds__(NB_MAX)
+sort_chunk_kernel(u32 *__restrict__ tilehist, int64_t num_tiles, int nb, u32 *__restrict__ chunk_sum)
+{
+    const int d = threadIdx.x;
+    if (d >= nb) return;
+    const int64_t t0 = (int64_t)blockIdx.x * HIST_CHUNK;
+    const int n = (int)min((int64_t)HIST_CHUNK, num_tiles - t0);
+    u32 run = 0;
+    for (int b = 0; b < n; b += 8) {
+        u32 c[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) c[k] = b + k < n ? tilehist[(size_t)(t0 + b + k) * nb + d] : 0u;
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+            if (b + k < n) { tilehist[(size_t)(t0 + b + k) * nb + d] = run; run += c[k]; }
+    }
+    chunk_sum[(size_t)blockIdx.x * nb + d] = run;
+}
+
+// one block, thread = digit: running counts over the chunks, then an exclusive scan of the digits' totals
+__global__ void __launch_bounds__(NB_MAX)
+sort_base_kernel(u32 *__restrict__ chunk_sum, int64_t num_chunks, int nb, u32 *__restrict__ digit_base)
+{
+    __shared__ u32 wsum[NB_MAX / 32];
+    const int d = threadIdx.x, lane = d & 31, warp = d >> 5;
+    u32 run = 0;
+    if (d < nb) {
+        for (int64_t c = 0; c < num_chunks; c += 8) {
+            u32 v[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) v[k] = c + k < num_chunks ? chunk_sum[(size_t)(c + k) * nb + d] : 0u;
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                if (c + k < num_chunks) { chunk_sum[(size_t)(c + k) * nb + d] = run; run += v[k]; }
+        }
+    }
+    u32 incl = run;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const u32 v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    if (lane == 31) wsum[warp] = incl;
+    __syncthreads();
+    u32 woff = 0;
+    for (int w = 0; w < warp; ++w) woff += wsum[w];
+    if (d < nb) digit_base[d] = woff + incl - run;
 }
 
 // stable scatter of one tile by one digit
+// LAST: the final pass leaves keys and payloads in arrays of their own, as the kernels behind the sort read them
+template <bool LAST>
 __global__ void __launch_bounds__(ST_THREADS)
-sort_scatter_kernel(const u32 *__restrict__ keys_in, const u32 *__restrict__ vals_in,
+sort_scatter_kernel(const uint2 *__restrict__ pairs_in, uint2 *__restrict__ pairs_out,
                     u32 *__restrict__ keys_out, u32 *__restrict__ vals_out,
-                    const u32 *__restrict__ tile_offsets, u32 *__restrict__ next_tilehist,
-                    int64_t L, int shift, int nb, int next_shift, int64_t num_tiles, int *__restrict__ status)
+                    const u32 *__restrict__ tilehist, const u32 *__restrict__ chunk_sum,
+                    const u32 *__restrict__ digit_base, int64_t L, int shift, int nb, int *__restrict__ status)
 {
     __shared__ u32 cnt[ST_WARPS][NB_MAX];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -170,8 +203,9 @@ sort_scatter_kernel(const u32 *__restrict__ keys_in, const u32 *__restrict__ val
     for (int k = 0; k < ST_ITEMS; ++k) {
         int64_t i = base + k * 32;
         bool valid = i < L;
-        key[k] = valid ? keys_in[i] : 0u;
-        val[k] = valid ? vals_in[i] : 0u;
+        const uint2 pr = valid ? pairs_in[i] : make_uint2(0u, 0u);
+        key[k] = pr.x;
+        val[k] = pr.y;
     }
     const u32 lt = (1u << lane) - 1u;
 #pragma unroll
@@ -192,7 +226,7 @@ sort_scatter_kernel(const u32 *__restrict__ keys_in, const u32 *__restrict__ val
     __syncthreads();
     // per digit: running offset over warps, starting at this tile's global offset
     for (int b = threadIdx.x; b < nb; b += ST_THREADS) {
-        u32 run = tile_offsets[(size_t)b * num_tiles + tile];
+        u32 run = digit_base[b] + chunk_sum[(size_t)(tile / HIST_CHUNK) * nb + b] + tilehist[(size_t)tile * nb + b];
 #pragma unroll
         for (int w = 0; w < ST_WARPS; ++w) {
             u32 c = cnt[w][b];
@@ -207,10 +241,12 @@ sort_scatter_kernel(const u32 *__restrict__ keys_in, const u32 *__restrict__ val
             u32 digit = (key[k] >> shift) & mask;
             u32 pos = cnt[warp][digit] + rank[k];
             if ((int64_t)pos < L) {
-                keys_out[pos] = key[k];
-                vals_out[pos] = val[k];
-                if (next_tilehist)
-                    atomicAdd(&next_tilehist[(size_t)((key[k] >> next_shift) & mask) * num_tiles + pos / ST_TILE], 1u);
+                if (LAST) {
+                    keys_out[pos] = key[k];
+                    vals_out[pos] = val[k];
+                } else {
+                    pairs_out[pos] = make_uint2(key[k], val[k]);
+                }
             } else {
                 dq_report(status, DQRM_ERR_INDEX_RANGE);   // only reachable with inconsistent offsets
             }
@@ -454,16 +490,17 @@ int dq_launch_bwd_sort(dqrm_ctx *ctx, const int32_t *indices, const int32_t *off
     const bool fits_cluster = (L + ctx->T - 1) / ctx->T <= (int64_t)csort::CLUSTER * 12288;   // (a table beyond its
     // blocks' shared memory still sorts, through global staging, but slowly)
     const bool try_cluster = ctx->sort_path != 1 && fits_cluster;
-    DQRM_CUDA_TRY(ctx, cudaMemsetAsync(ws, 0, try_cluster ? y.zero_small : y.zero_bytes, st));
+    DQRM_CUDA_TRY(ctx, cudaMemsetAsync(ws, 0, y.zero_small, st));
     dq_mark(ctx, st, DQ_K_MEMSET);
     if (L == 0) {
         DQRM_CUDA_TRY(ctx, cudaMemsetAsync(uniq_off, 0, sizeof(int32_t) * (ctx->T + 1), st));
         return DQRM_OK;
     }
-    u32 *keys[2] = {reinterpret_cast<u32 *>(ws + y.keys_a), reinterpret_cast<u32 *>(ws + y.keys_b)};
-    u32 *vals[2] = {reinterpret_cast<u32 *>(ws + y.vals_a), reinterpret_cast<u32 *>(ws + y.vals_b)};
-    u32 *thist[2] = {reinterpret_cast<u32 *>(ws + y.tilehist_a), reinterpret_cast<u32 *>(ws + y.tilehist_b)};
-    u32 *ghist = reinterpret_cast<u32 *>(ws + y.ghist);
+    u32 *keys[1] = {reinterpret_cast<u32 *>(ws + y.keys_a)};
+    u32 *vals[1] = {reinterpret_cast<u32 *>(ws + y.vals_a)};
+    uint2 *pairs[2] = {reinterpret_cast<uint2 *>(ws + y.pairs_a), reinterpret_cast<uint2 *>(ws + y.pairs_b)};
+    u32 *tilehist = reinterpret_cast<u32 *>(ws + y.tilehist), *chunk_sum = reinterpret_cast<u32 *>(ws + y.chunk_sum);
+    u32 *digit_base = reinterpret_cast<u32 *>(ws + y.digit_base);
     const u32 *skeys = nullptr;      // sorted keys; the sorted payloads sit beside them in vals[0]
     bool sorted = false;
     // (tables far beyond the shared-memory slices sort faster with the global radix sort)
@@ -493,33 +530,38 @@ int dq_launch_bwd_sort(dqrm_ctx *ctx, const int32_t *indices, const int32_t *off
         }
     }
     if (!sorted) {
-        if (try_cluster)      // the cluster launch was refused: zero what the radix sort needs as well
-            DQRM_CUDA_TRY(ctx, cudaMemsetAsync(ws + y.zero_small, 0, y.zero_bytes - y.zero_small, st));
     {
         int64_t blocks = (G + 255) / 256;
         int64_t cap = (int64_t)ctx->num_sms * 8;
         int grid = (int)(blocks > cap ? cap : blocks);
-        prepare_kernel<<<grid, 256, 0, st>>>(indices, offsets, ctx->d_row_off, ctx->T, B, G, L, keys[y.passes & 1], vals[y.passes & 1],
-                                             ghist, thist[0], y.num_tiles, y.passes, y.digit_bits, ctx->payload_position, ctx->d_status);
+        prepare_kernel<<<grid, 256, 0, st>>>(indices, offsets, ctx->d_row_off, ctx->T, B, G, L, pairs[0],
+                                             ctx->payload_position, ctx->d_status);
         DQRM_CUDA_TRY(ctx, cudaGetLastError());
         dq_mark(ctx, st, DQ_K_PREPARE);
     }
+    const int64_t hist_chunks = (y.num_tiles + HIST_CHUNK - 1) / HIST_CHUNK;
     for (int p = 0; p < y.passes; ++p) {
-        const bool has_next = p + 1 < y.passes;
-        u32 *cur = thist[p & 1], *nxt = has_next ? thist[(p + 1) & 1] : nullptr;
-        int scan_grid = (y.nb * 32 + 255) / 256;
-        sort_scan_kernel<<<scan_grid, 256, 0, st>>>(cur, ghist + p * NB_MAX, y.nb, y.num_tiles, nxt,
-                                                    has_next ? (int64_t)y.nb * y.num_tiles : 0);
+        const uint2 *pin = pairs[p & 1];
+        const int shift = p * y.digit_bits;
+        sort_hist_kernel<<<(unsigned)y.num_tiles, ST_THREADS, 0, st>>>(pin, L, shift, y.nb, tilehist);
         DQRM_CUDA_TRY(ctx, cudaGetLastError());
         dq_mark(ctx, st, DQ_K_SORT_SCAN);
-        sort_scatter_kernel<<<(unsigned)y.num_tiles, ST_THREADS, 0, st>>>(
-            keys[(p + y.passes) & 1], vals[(p + y.passes) & 1], keys[(p + y.passes + 1) & 1], vals[(p + y.passes + 1) & 1],
-            cur, nxt, L, p * y.digit_bits, y.nb,
-            (p + 1) * y.digit_bits, y.num_tiles, ctx->d_status);
+        sort_chunk_kernel<<<(unsigned)hist_chunks, NB_MAX, 0, st>>>(tilehist, y.num_tiles, y.nb, chunk_sum);
+        DQRM_CUDA_TRY(ctx, cudaGetLastError());
+        dq_mark(ctx, st, DQ_K_SORT_SCAN);
+        sort_base_kernel<<<1, NB_MAX, 0, st>>>(chunk_sum, hist_chunks, y.nb, digit_base);
+        DQRM_CUDA_TRY(ctx, cudaGetLastError());
+        dq_mark(ctx, st, DQ_K_SORT_SCAN);
+        if (p + 1 < y.passes)
+            sort_scatter_kernel<false><<<(unsigned)y.num_tiles, ST_THREADS, 0, st>>>(
+                pin, pairs[(p + 1) & 1], nullptr, nullptr, tilehist, chunk_sum, digit_base, L, shift, y.nb, ctx->d_status);
+        else
+            sort_scatter_kernel<true><<<(unsigned)y.num_tiles, ST_THREADS, 0, st>>>(
+                pin, nullptr, keys[0], vals[0], tilehist, chunk_sum, digit_base, L, shift, y.nb, ctx->d_status);
         DQRM_CUDA_TRY(ctx, cudaGetLastError());
         dq_mark(ctx, st, DQ_K_SORT_SCATTER);
     }
-        skeys = keys[0];                         // the ping-pong starts so that the last pass lands in buffer 0
+        skeys = keys[0];
     }
     if (!sorted) {        // (the cluster sort counts the segment heads of every tile on its way out)
         seg_count_kernel<<<(unsigned)y.num_tiles, ST_THREADS, 0, st>>>(skeys, L, reinterpret_cast<u32 *>(ws + y.tile_heads));
