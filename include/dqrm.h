@@ -167,7 +167,10 @@ int dqrm_train_step(dqrm_ctx *ctx, float *tables, const int32_t *indices,
  * for the same batch.  The sorted order travels in `workspace` (dqrm_workspace_bytes): pass
  * the same workspace to both calls and to nothing in between; two workspaces used alternately
  * let batch k+1 be sorted on one stream while batch k trains on another.  The caller orders
- * the two calls (same stream, or an event).  Outputs equal those of dqrm_train_step. */
+ * the two calls (same stream, or an event).  One dqrm_sort_batch serves ONE
+ * dqrm_train_step_sorted: the step uses up counters that only the sort resets, so a second
+ * step on the same workspace without a new sort gives wrong sums (it writes nothing outside the
+ * workspace and the caller's buffers).  Outputs equal those of dqrm_train_step. */
 int dqrm_sort_batch(dqrm_ctx *ctx, const int32_t *indices, const int32_t *offsets,
                     int32_t *unique_rows, int32_t *uniq_off, int B, int64_t L,
                     void *workspace, size_t workspace_bytes, void *stream);
@@ -199,9 +202,12 @@ size_t dqrm_host_step_workspace_bytes(const dqrm_ctx *ctx, int64_t max_lookups, 
  * the pooled output back to h_out [B][T][D]; asynchronously when the host buffers are
  * pinned.  The call is ordered on `stream`: it starts behind the work already on `stream`,
  * and work put on `stream` afterwards starts once the step and both copies are complete.
- * Inside the call the upstream gradient comes in and the pooled output goes out on two
- * streams owned by the context, beside the index sort and the forward (the two transfers
- * run in opposite directions); with dqrm_set_overlap(ctx, 0) everything stays on `stream`.
+ * Inside the call the inputs come in and the pooled output goes out on two streams owned by
+ * the context, beside the index sort and the forward (the two large transfers run in opposite
+ * directions).  The workspace holds two sets of staging buffers that consecutive calls use in
+ * turn, so the inputs of a call are copied while the call before it is still computing and
+ * sending its output; a caller that issues calls back to back therefore keeps both directions
+ * of the host link busy.  With dqrm_set_overlap(ctx, 0) everything stays on `stream`.
  * tables, scales and bits stay on the device.  The sparse gradient (unique rows, codes,
  * scales) stays in the workspace.  h_grad_out and h_out must stay valid and untouched
  * until the call's work on `stream` is complete. */
@@ -298,15 +304,18 @@ int dqrm_decode_payload(dqrm_ctx *ctx, const uint8_t *payload, const float *scal
 
 /* ---- choice of the backward's sort (no counterpart in the paper) --------------------
  * dqrm_emb_bwd and dqrm_train_step order the batch's lookups by row before they sum
- * duplicates.  path 0 (default): one thread-block cluster per table sorts that table's
- * lookups in distributed shared memory.  path 1: one global least-significant-digit radix
- * sort over all tables.  Both give identical outputs; the choice only affects speed. */
+ * duplicates.  path 0 (default): one thread-block cluster per table (eight blocks, sixteen
+ * when the batch has very few tables) sorts that table's lookups in distributed shared
+ * memory; a batch with more lookups per table than such a cluster holds takes path 1 by
+ * itself.  path 1: one global least-significant-digit radix sort over all tables.  Both give
+ * identical outputs; the choice only affects speed. */
 int dqrm_set_sort_path(dqrm_ctx *ctx, int path);
 
-/* dqrm_train_step runs the index sort of its backward on a second stream owned by the
- * context (created by dqrm_create), beside the forward on the caller's stream, and joins
- * the two before the gradient is summed; the caller's stream sees one ordered step.
- * on = 0 keeps every launch on the caller's stream.  Default: 1. */
+/* dqrm_train_step and dqrm_train_step_sorted run the backward up to the summed gradient (index
+ * sort, gradient summation: neither needs the tables or the forward's output) on a second
+ * stream owned by the context (created by dqrm_create), beside the forward on the caller's
+ * stream, and join the two before the touched rows are updated; the caller's stream sees one
+ * ordered step.  on = 0 keeps every launch on the caller's stream.  Default: 1. */
 int dqrm_set_overlap(dqrm_ctx *ctx, int on);
 
 /* ---- quantiser self-check (no counterpart in the paper) ----------------------------

@@ -35,7 +35,8 @@ constexpr int SEG_CHUNK = segred::CHUNK;         // sorted entries per reduce wo
 
 struct Layout {
     int passes, digit_bits, nb;
-    int64_t num_tiles, num_chunks;
+    int ck;                                    // sorted entries per lane group of the reduce: 32, or 16
+    int64_t num_tiles, num_chunks;             // num_chunks = ceil(L / ck)
     // zeroed at call start: [0, zero_small)
     size_t absmax, counters, tile_heads, zero_small, digit_base, chunk_sum, tilehist;
     size_t keys_a, vals_a, pairs_a, pairs_b, seg_start, chunk_first, long_list, partials;
@@ -51,7 +52,16 @@ Layout make_layout(const dqrm_ctx *ctx, int64_t L)
     y.nb = 1 << y.digit_bits;
     int64_t Lc = L < 1 ? 1 : L;
     y.num_tiles = (Lc + ST_TILE - 1) / ST_TILE;
-    y.num_chunks = (Lc + SEG_CHUNK - 1) / SEG_CHUNK;
+    // A chunk is walked in order by one lane group.  A batch whose 32-entry chunks would not even give every SM
+    // one block of the reduce takes 16-entry chunks: twice the groups, each half as long (measured: 19 -> 14 us
+    // at batch 128, but 24 -> 29 us at 208 blocks, where the extra pieces cost more than the shorter walks save).
+    y.ck = SEG_CHUNK;
+    {
+        const int D = ctx->D;
+        const int rl = D <= 4 ? 4 : D <= 8 ? 8 : D <= 16 ? 4 : D <= 64 ? 16 : 32;      // lanes per row of the reduce
+        if (rl <= 16 && (Lc / SEG_CHUNK) / (256 / rl) < (int64_t)ctx->num_sms) y.ck = SEG_CHUNK / 2;
+    }
+    y.num_chunks = (Lc + y.ck - 1) / y.ck;
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
     y.absmax = take(sizeof(u32) * ctx->T);
@@ -293,7 +303,7 @@ __global__ void __launch_bounds__(ST_THREADS)
 seg_emit_kernel(const u32 *__restrict__ keys, int64_t L, const u32 *__restrict__ tile_heads,
                 const int64_t *__restrict__ row_off, int T,
                 u32 *__restrict__ seg_start, u32 *__restrict__ chunk_first,
-                int32_t *__restrict__ unique_rows, int32_t *__restrict__ uniq_off, u32 *__restrict__ counters)
+                int32_t *__restrict__ unique_rows, int32_t *__restrict__ uniq_off, u32 *__restrict__ counters, int ck)
 {
     extern __shared__ unsigned char smem_raw[];
     int64_t *s_off = reinterpret_cast<int64_t *>(smem_raw);   // [T+1]
@@ -369,7 +379,7 @@ seg_emit_kernel(const u32 *__restrict__ keys, int64_t L, const u32 *__restrict__
                 t_prev = t;
             }
             const u32 u_of_i = heads_before - 1;
-            if ((i % SEG_CHUNK) == 0) chunk_first[i / SEG_CHUNK] = u_of_i;
+            if ((i % ck) == 0) chunk_first[i / ck] = u_of_i;
             if (i == L - 1) {
                 const u32 U = u_of_i + 1;
                 seg_start[U] = (u32)L;
@@ -398,15 +408,23 @@ int launch_reduce(dqrm_ctx *ctx, const Layout &y, char *ws, const u32 *keys, con
     const u32 *seg_start = reinterpret_cast<const u32 *>(ws + y.seg_start);
     double *partials = reinterpret_cast<double *>(ws + y.partials);
     uint4 *long_list = reinterpret_cast<uint4 *>(ws + y.long_list);
-    const size_t red_smem = (size_t)(ctx->T + 1) * sizeof(u32) + (size_t)gpb * 2 * SEG_CHUNK * sizeof(u32);
-    if (ctx->D == RL * RV * RC)
-        seg_reduce_kernel<RL, RV, RC, true><<<grid, 256, red_smem, st>>>(
-            keys, vals, seg_start, reinterpret_cast<const u32 *>(ws + y.chunk_first), uniq_off, grad_out, grad_rows,
-            partials, long_list, counters, absmax, ctx->T, ctx->D, L, G, y.num_chunks, ctx->d_status);
-    else
-        seg_reduce_kernel<RL, RV, RC, false><<<grid, 256, red_smem, st>>>(
-            keys, vals, seg_start, reinterpret_cast<const u32 *>(ws + y.chunk_first), uniq_off, grad_out, grad_rows,
-            partials, long_list, counters, absmax, ctx->T, ctx->D, L, G, y.num_chunks, ctx->d_status);
+    const size_t red_smem = (size_t)(ctx->T + 1) * sizeof(u32) + (size_t)gpb * 2 * y.ck * sizeof(u32);
+    const u32 *chunk_first = reinterpret_cast<const u32 *>(ws + y.chunk_first);
+#define DQ_LAUNCH_REDUCE(EXACT, CK)                                                                                  \
+    seg_reduce_kernel<RL, RV, RC, EXACT, CK><<<grid, 256, red_smem, st>>>(                                          \
+        keys, vals, seg_start, chunk_first, uniq_off, grad_out, grad_rows, partials, long_list, counters, absmax,    \
+        ctx->T, ctx->D, L, G, y.num_chunks, ctx->d_status)
+    const bool exact = ctx->D == RL * RV * RC;
+    if constexpr (RL <= 16) {
+        if (y.ck == SEG_CHUNK / 2) {
+            if (exact) DQ_LAUNCH_REDUCE(true, SEG_CHUNK / 2); else DQ_LAUNCH_REDUCE(false, SEG_CHUNK / 2);
+        } else {
+            if (exact) DQ_LAUNCH_REDUCE(true, SEG_CHUNK); else DQ_LAUNCH_REDUCE(false, SEG_CHUNK);
+        }
+    } else {
+        if (exact) DQ_LAUNCH_REDUCE(true, SEG_CHUNK); else DQ_LAUNCH_REDUCE(false, SEG_CHUNK);
+    }
+#undef DQ_LAUNCH_REDUCE
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
     dq_mark(ctx, st, DQ_K_SEG_REDUCE);
     int64_t fblocks = (y.num_chunks + 7) / 8;                // at most one cut segment per chunk, a warp each
@@ -571,7 +589,7 @@ int dq_launch_bwd_sort(dqrm_ctx *ctx, const int32_t *indices, const int32_t *off
     seg_emit_kernel<<<(unsigned)y.num_tiles, ST_THREADS, (size_t)(ctx->T + 1) * sizeof(int64_t), st>>>(
         skeys, L, reinterpret_cast<const u32 *>(ws + y.tile_heads), ctx->d_row_off, ctx->T,
         reinterpret_cast<u32 *>(ws + y.seg_start), reinterpret_cast<u32 *>(ws + y.chunk_first), unique_rows, uniq_off,
-        reinterpret_cast<u32 *>(ws + y.counters));
+        reinterpret_cast<u32 *>(ws + y.counters), y.ck);
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
     dq_mark(ctx, st, DQ_K_SEG_EMIT);
     return DQRM_OK;

@@ -17,7 +17,7 @@
 
 namespace segred {
 
-constexpr int CHUNK = 32;            // sorted entries per warp work item
+constexpr int CHUNK = 32;            // sorted entries per lane group of the reduce (16 for a small batch of narrow rows)
 constexpr int PREFETCH_ROW_BYTES = 512;   // rows up to this size are prefetched into L2 by the reduce's head phase
 constexpr int BIG_PIECES = 32;       // cut segments with more pieces go to the block-wide fix-up
 enum { CNT_LONG = 0, CNT_U = 1, CNT_BIG = 2 };
@@ -112,9 +112,11 @@ __device__ __forceinline__ void vec_add(double (&acc)[VEC], const typename Vec<V
 // neighbouring keys once (this chunk's and the next one's); the resulting bit masks of segment heads
 // and the payloads (parked in shared memory) are all the walk needs, so an entry costs one shared
 // load, one address, one 128-bit load, a bit test and the FP64 adds.
-// (256-byte rows want four resident blocks per SM: that caps the kernel at 64 registers)
-template <int LPR, int VEC, int CH, bool EXACT, bool OWN = (LPR >= 8)>
-__global__ void __launch_bounds__(256, (LPR == 16 && VEC == 4 && CH == 1) ? 4 : 1)
+// (256-byte rows want four resident blocks per SM: that caps the kernel at 64 registers.  64-byte rows are capped
+// at three blocks' worth, 78 registers with a few spills: alone the kernel loses a microsecond, beside the sort of
+// the next batch the step gains three, because the two then fit on an SM together)
+template <int LPR, int VEC, int CH, bool EXACT, int CK = 32, bool OWN = (LPR >= 8)>
+__global__ void __launch_bounds__(256, (LPR == 16 && VEC == 4 && CH == 1) ? 4 : (LPR == 4 && VEC == 4) ? 3 : 1)
 seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
                   const u32 *__restrict__ seg_start, const u32 *__restrict__ chunk_first,
                   const int32_t *__restrict__ uniq_off,
@@ -128,13 +130,13 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
     const int D = EXACT ? LPR * VEC * CH : D_any;
     extern __shared__ unsigned char smem_raw[];
     u32 *s_uoff = reinterpret_cast<u32 *>(smem_raw);                                     // [T+1]
-    u32 *s_vals = s_uoff + (T + 1) + (size_t)(threadIdx.x / LPR) * (2 * CHUNK);          // this group's [2*CHUNK]
+    u32 *s_vals = s_uoff + (T + 1) + (size_t)(threadIdx.x / LPR) * (2 * CK);          // this group's [2*CK]
     for (int t = threadIdx.x; t <= T; t += blockDim.x) s_uoff[t] = (u32)uniq_off[t];
     __syncthreads();
 
     typedef typename Vec<VEC>::type vec_t;
     constexpr int NB = (VEC == 4 && LPR > 4) ? 4 : 8;   // rows in flight per lane
-    constexpr int EPL = CHUNK / LPR;              // chunk entries one lane looks at
+    constexpr int EPL = CK / LPR;              // chunk entries one lane looks at
     const int dv = D / VEC;                       // vectors per row
     const int lane = threadIdx.x % LPR;
     const u32 gmask = group_mask<LPR>();
@@ -147,9 +149,9 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
     const uint64_t keep = dq_policy_evict_last();
 
     for (int64_t c = group; c < num_chunks; c += n_groups) {
-        const int64_t i0 = c * CHUNK;
-        const int n = (int)(min(i0 + (int64_t)CHUNK, L) - i0);
-        const int n_next = (int)max((int64_t)0, min((int64_t)CHUNK, L - i0 - CHUNK));
+        const int64_t i0 = c * CK;
+        const int n = (int)(min(i0 + (int64_t)CK, L) - i0);
+        const int n_next = (int)max((int64_t)0, min((int64_t)CK, L - i0 - CK));
         // Heads: entry e starts a segment when its key differs from the key before it; the same for the
         // chunk behind, whose first head tells where this chunk's last segment ends.  All loads are issued
         // before the first vote so that they are in flight together.
@@ -167,16 +169,16 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
             if (OWN) {
                 kn[j] = knp[j] = vn[j] = 0u;
                 if (e < n_next) {
-                    vn[j] = vals[i + CHUNK];
-                    kn[j] = keys[i + CHUNK];
-                    knp[j] = keys[i + CHUNK - 1];
+                    vn[j] = vals[i + CK];
+                    kn[j] = keys[i + CK];
+                    knp[j] = keys[i + CK - 1];
                 }
             }
         }
         // OWN: did the run that enters this chunk begin in the chunk before?  (the keys ascend: it did unless the
         // key 33 entries back is still the same).  Otherwise: the key behind the chunk tells whether its last run ends
         u32 k_x = 0u;
-        if (OWN) { if (i0 > CHUNK) k_x = keys[i0 - CHUNK - 1]; }
+        if (OWN) { if (i0 > CK) k_x = keys[i0 - CK - 1]; }
         else if (i0 + n < L) k_x = keys[i0 + n];
         const u32 u_first = chunk_first[c];
         __syncwarp(gmask);                        // the previous chunk's payloads are no longer read
@@ -202,7 +204,7 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
                 if (e < n_next) {
                     u32 v = vn[j];
                     if ((int64_t)v >= G) { bad = true; v = 0u; }
-                    s_vals[CHUNK + e] = v;
+                    s_vals[CK + e] = v;
                 }
                 const bool head_n = (e < n_next) && (kn[j] != knp[j]);
                 heads_n |= ((__ballot_sync(gmask, head_n) >> gbase) & lm) << (j * LPR);
@@ -210,7 +212,7 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
             const bool head = (e < n) && (kc[j] != kp[j]);
             heads |= ((__ballot_sync(gmask, head) >> gbase) & lm) << (j * LPR);
         }
-        if (n_next < CHUNK) heads_n |= 1u << n_next;   // the end of the array closes a run like a head
+        if (n_next < CK) heads_n |= 1u << n_next;   // the end of the array closes a run like a head
         const u32 k_0 = __shfl_sync(gmask, kc[0], gbase);
         // the chunk's last key sits in lane (n-1) % LPR, register (n-1) / LPR
         u32 k_last = 0u;
@@ -220,7 +222,7 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
         k_last = __shfl_sync(gmask, k_last, gbase + (n - 1) % LPR);
         __syncwarp(gmask);
 
-        // ---- which entries this group sums: [ea, eb) relative to i0, eb up to 2*CHUNK.
+        // ---- which entries this group sums: [ea, eb) relative to i0, eb up to 2*CK.
         // A segment is summed where it BEGINS, together with its tail in the next chunk; a leading run that
         // began in the chunk before and ends here was summed there.  Only a segment whose tail is not over
         // within the next chunk is summed in pieces (FP64 partials, folded by the fix-up kernel).
@@ -231,12 +233,12 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
         bool lead_piece, trail_long;
         int ea, eb;
         if (OWN) {
-            const bool closes_here = any_head || n < CHUNK;
-            const bool began_prev = (i0 <= CHUNK) || (k_x != k_0);
+            const bool closes_here = any_head || n < CK;
+            const bool began_prev = (i0 <= CK) || (k_x != k_0);
             lead_piece = f > 0 && !(closes_here && began_prev);
             ea = lead_piece ? 0 : f;
             trail_long = any_head && heads_n == 0u;
-            eb = n + ((any_head && heads_n != 0u) ? __ffs(heads_n) - 1 : 0);    // (an extension only when n == CHUNK)
+            eb = n + ((any_head && heads_n != 0u) ? __ffs(heads_n) - 1 : 0);    // (an extension only when n == CK)
         } else {
             lead_piece = f > 0;
             ea = 0;
@@ -290,13 +292,13 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
                 if (begins && lane == 0) {
                     // the segment begins here: leave all the fix-up needs to know about it in one record
                     const u32 sa = seg_start[u], sb = seg_start[u + 1];
-                    const u32 npieces = (sb - 1) / CHUNK - sa / CHUNK + 1;
+                    const u32 npieces = (sb - 1) / CK - sa / CK + 1;
                     int lo = 0, hi = T;              // its table: largest t with s_uoff[t] <= u
                     while (hi - lo > 1) {
                         const int mid = (lo + hi) >> 1;
                         if (s_uoff[mid] <= u) lo = mid; else hi = mid;
                     }
-                    const uint4 rec = make_uint4(u, sa / CHUNK, npieces, (u32)lo);
+                    const uint4 rec = make_uint4(u, sa / CK, npieces, (u32)lo);
                     // (the list has a slot per chunk and every chunk begins at most one such segment; the bound only
                     // matters for a workspace that is summed twice without a sort in between, which must not write
                     // outside the list)
@@ -328,7 +330,7 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
             for (int k = 0; k < NB; ++k) {
                 const int e = e0 + k;
                 if (FULL || e < eb) {
-                    if (e > ea && e < CHUNK && ((heads >> e) & 1u)) {
+                    if (e > ea && e < CK && ((heads >> e) & 1u)) {
                         flush(run_start, e);
                         u += 1;
                         run_start = e;
@@ -352,7 +354,7 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
     if (bad) dq_report(status, DQRM_ERR_INDEX_RANGE);
 }
 
-// pieces of cut segment [a, e): chunk a/32 holds the first (slot 1), later chunks slot 0
+// pieces of a listed segment: the chunk in which it begins holds the first (slot 1), later chunks slot 0
 __device__ __forceinline__ const double *piece_ptr(const double *partials, int64_t c0, int64_t p, int D)
 {
     return partials + ((size_t)(c0 + p) * 2 + (p == 0 ? 1 : 0)) * D;
