@@ -67,6 +67,7 @@ extern "C" {
 #define DQRM_ERR_INDEX_RANGE   (-4)  /* device saw an index outside [0, R_t) or a bad offset */
 #define DQRM_ERR_TIMEOUT       (-5)  /* reserved: a bounded device-side wait ran out */
 #define DQRM_ERR_STATIC_LIMIT  (-6)  /* size exceeds the built-in scratch of a *_static call */
+#define DQRM_ERR_NOT_SORTED    (-7)  /* dqrm_train_step_sorted: the workspace holds no unconsumed sorted batch of this L, B */
 
 typedef struct dqrm_ctx dqrm_ctx;
 
@@ -168,9 +169,12 @@ int dqrm_train_step(dqrm_ctx *ctx, float *tables, const int32_t *indices,
  * the same workspace to both calls and to nothing in between; two workspaces used alternately
  * let batch k+1 be sorted on one stream while batch k trains on another.  The caller orders
  * the two calls (same stream, or an event).  One dqrm_sort_batch serves ONE
- * dqrm_train_step_sorted: the step uses up counters that only the sort resets, so a second
- * step on the same workspace without a new sort gives wrong sums (it writes nothing outside the
- * workspace and the caller's buffers).  Outputs equal those of dqrm_train_step. */
+ * dqrm_train_step_sorted: the step uses up counters that only the sort resets.  The context
+ * keeps, on the host, which workspaces hold a sorted batch that no step has taken yet;
+ * dqrm_train_step_sorted on a workspace that holds none (never sorted, already used, or sorted
+ * for another B or L) returns DQRM_ERR_NOT_SORTED and launches nothing.  A step replayed from
+ * a captured CUDA graph is outside that bookkeeping: capture each step together with its sort.
+ * Outputs equal those of dqrm_train_step. */
 int dqrm_sort_batch(dqrm_ctx *ctx, const int32_t *indices, const int32_t *offsets,
                     int32_t *unique_rows, int32_t *uniq_off, int B, int64_t L,
                     void *workspace, size_t workspace_bytes, void *stream);

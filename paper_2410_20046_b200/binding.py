@@ -15,6 +15,7 @@ ERR_CUDA = -3
 ERR_INDEX_RANGE = -4
 ERR_TIMEOUT = -5
 ERR_STATIC_LIMIT = -6
+ERR_NOT_SORTED = -7
 STATIC_MAX_TABLES = 1024
 
 _vp = ctypes.c_void_p

@@ -234,6 +234,7 @@ const char *dqrm_status_string(int status)
     case DQRM_ERR_INDEX_RANGE: return "index or offset out of range (detected on the device)";
     case DQRM_ERR_TIMEOUT: return "bounded device-side wait ran out";
     case DQRM_ERR_STATIC_LIMIT: return "size exceeds the built-in scratch of an allocation-free call";
+    case DQRM_ERR_NOT_SORTED: return "workspace holds no unconsumed sorted batch of this size (call dqrm_sort_batch first)";
     default: return "unknown status";
     }
 }
@@ -361,7 +362,13 @@ int dqrm_sort_batch(dqrm_ctx *ctx, const int32_t *indices, const int32_t *offset
     if (!ws_ok(workspace, workspace_bytes, dq_bwd_ws_bytes(ctx, L, (int64_t)ctx->T * B))) return DQRM_ERR_WORKSPACE;
     cudaStream_t st = as_stream(stream);
     if (ctx->prof_on) dq_mark(ctx, st, DQ_K_BEGIN);
-    return dq_launch_bwd_sort(ctx, indices, offsets, unique_rows, uniq_off, B, L, workspace, workspace_bytes, st, nullptr);
+    const int rc = dq_launch_bwd_sort(ctx, indices, offsets, unique_rows, uniq_off, B, L, workspace, workspace_bytes, st, nullptr);
+    {
+        std::lock_guard<std::mutex> lock(ctx->sorted_mu);
+        if (rc == DQRM_OK) ctx->sorted[workspace] = std::make_pair(L, B);
+        else ctx->sorted.erase(workspace);
+    }
+    return rc;
 }
 
 int dqrm_train_step_sorted(dqrm_ctx *ctx, float *tables, const int32_t *indices, const int32_t *offsets,
@@ -375,6 +382,13 @@ int dqrm_train_step_sorted(dqrm_ctx *ctx, float *tables, const int32_t *indices,
         return DQRM_ERR_INVALID_ARG;
     if (L > 0 && (!indices || !unique_rows || !grad_rows || !codes)) return DQRM_ERR_INVALID_ARG;
     if (!ws_ok(workspace, workspace_bytes, dq_bwd_ws_bytes(ctx, L, (int64_t)ctx->T * B))) return DQRM_ERR_WORKSPACE;
+    {   // the workspace must hold this batch, sorted by dqrm_sort_batch and not consumed yet: the summation
+        // trusts the segment lists in it and zeroes nothing itself
+        std::lock_guard<std::mutex> lock(ctx->sorted_mu);
+        auto it = ctx->sorted.find(workspace);
+        if (it == ctx->sorted.end() || it->second.first != L || it->second.second != B) return DQRM_ERR_NOT_SORTED;
+        ctx->sorted.erase(it);
+    }
     cudaStream_t st = as_stream(stream);
     if (ctx->prof_on) dq_mark(ctx, st, DQ_K_BEGIN);
     // the gradient summation (second stream of the context) runs beside the forward (caller's stream)

@@ -1,5 +1,8 @@
 // Internal declarations shared by the CUDA translation units of the DQRM library.
 #pragma once
+#include <mutex>
+#include <unordered_map>
+#include <utility>
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <stddef.h>
@@ -30,6 +33,9 @@ struct dqrm_ctx {
     cudaEvent_t ev_h_free[2] = {nullptr, nullptr}, ev_h_idx = nullptr;
     bool h_set_used[2] = {false, false};
     unsigned host_calls = 0;
+    // workspaces that hold a sorted batch nobody has consumed yet: pointer -> (L, B); host bookkeeping only
+    std::mutex sorted_mu;
+    std::unordered_map<const void *, std::pair<int64_t, int>> sorted;
     int overlap = 1;                // 0: keep everything on the caller's stream
     int payload_position = 0;       // sort payload: 0 = row of grad_out, 1 = position of the lookup (set by the merge)
     // kernels whose dynamic shared-memory limit has been raised on this context's device (the attribute is

@@ -117,6 +117,45 @@ def test_two_calls_equal_one_call():
     c.ctx.close()
 
 
+def test_step_on_a_workspace_without_a_fresh_sort_is_refused():
+    """One sort serves one step: a workspace that was never sorted, was sorted for another batch size, or whose
+    sorted batch a step has already taken is turned down on the host, before any launch."""
+    import torch
+    from paper_2410_20046_b200 import binding
+
+    wl = W.scaled_down(W.kaggle(), total_rows=50_000, B=300, name="kaggle_small")
+    c = Case(wl)
+    d_tables = c.dev(W.tables_np(wl))
+    scales = c.empty(wl.T, torch.float32)
+    c.ctx.scale_refresh(d_tables, c.bits, scales)
+    idx, off, go = c.batch(0)
+    L = len(idx)
+    out = c.empty((wl.B, wl.T, wl.D), torch.float32)
+    ur = torch.full((L,), -1, dtype=torch.int32, device="cuda")
+    uo = c.empty(wl.T + 1, torch.int32)
+    gr = torch.zeros((L, wl.D), dtype=torch.float32, device="cuda")
+    codes = torch.zeros((L, wl.D), dtype=torch.int8, device="cuda")
+    gs = c.empty(wl.T, torch.float32)
+    args = (d_tables, c.dev(idx), c.dev(off), c.dev(go), scales, c.bits, out, ur, uo, gr, codes, gs, wl.lr)
+
+    def refused(**kw):
+        with pytest.raises(binding.DqrmError) as e:
+            c.ctx.train_step_sorted(*args, **kw)
+        return e.value.status == binding.ERR_NOT_SORTED
+
+    assert refused(B=wl.B, L=L, ws=1)                       # never sorted
+    c.ctx.sort_batch(args[1], args[2], ur, uo, B=wl.B, L=L, ws=1)
+    assert refused(B=wl.B, L=L, ws=0)                       # the other workspace was
+    before = d_tables.clone()
+    c.ctx.train_step_sorted(*args, B=wl.B, L=L, ws=1)
+    c.ctx.raise_on_device_error()
+    after = d_tables.clone()
+    assert not torch.equal(before, after)
+    assert refused(B=wl.B, L=L, ws=1)                       # already taken
+    assert torch.equal(d_tables, after)                     # and nothing ran
+    c.ctx.close()
+
+
 def test_sort_held_until_the_forward_is_done_equals_one_call():
     """dqrm_stream_wait_forward: the next batch's sort starts only behind this batch's forward and runs
     beside the rest of the step; the trajectory must equal the single-call loop's bit for bit."""
