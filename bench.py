@@ -378,7 +378,7 @@ def measure(args, wl, where, primary):
             b = batches[bi]
             ctx.sort_batch(b["idx"], b["off"], urs[bi & 1], uos[bi & 1], B=wl.B, L=b["L"], ws=bi & 1)
 
-        def launch_step(bi):     # noqa: F811
+        def launch_step(bi, join=True):     # noqa: F811
             b, nb, slot = batches[bi], batches[(bi + 1) % N_BATCHES], bi & 1
             cur = torch.cuda.current_stream()
             side.wait_stream(cur)
@@ -393,7 +393,11 @@ def measure(args, wl, where, primary):
                                stream=side)
                 ctx.train_step_sorted(tables, b["idx"], b["off"], b["go"], scales, bits, out, urs[slot], uos[slot], gr,
                                       codes, gs, wl.lr, B=wl.B, L=b["L"], ws=slot, stream=cur)
-            cur.wait_stream(side)
+            # The next step's gradient summation waits for this sort by itself (an event the context keeps with the
+            # workspace); its forward does not need the sort and may start before the sort is done.  Only the last
+            # step of a captured graph joins the sort's stream (a capture must end with every stream joined).
+            if join or args.join_every_step:
+                cur.wait_stream(side)
 
         def launch_unpipelined(bi):
             b = batches[bi]
@@ -427,10 +431,15 @@ def measure(args, wl, where, primary):
             torch.cuda.synchronize()
 
             def capture(first, count):
+                if pipelined:
+                    prime(first)                     # the graph's first step takes a sort made before the graph
                 g = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g, stream=capture_stream):
                     for bi in range(first, first + count):
-                        launch_step(bi)
+                        if pipelined:
+                            launch_step(bi, join=(bi == first + count - 1))
+                        else:
+                            launch_step(bi)
                 return g
 
             n_before = ctx.launch_count()
@@ -794,6 +803,9 @@ def main():
                     help="priority of the stream the training half runs on (0: torch's current stream)")
     ap.add_argument("--sort-after-forward", type=int, default=0,
                     help="1: the next batch's sort waits for this batch's forward and runs beside the rest of the step")
+    ap.add_argument("--join-every-step", action="store_true",
+                    help="make every step wait for the next batch's sort before the following step begins "
+                         "(default: only that step's gradient summation waits; its forward starts at once)")
     ap.add_argument("--sort-path", type=int, default=0, help="0: per-table cluster sort, 1: global radix sort")
     ap.add_argument("--stub-step", action="store_true", help=argparse.SUPPRESS)
     args = ap.parse_args()

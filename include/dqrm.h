@@ -167,8 +167,14 @@ int dqrm_train_step(dqrm_ctx *ctx, float *tables, const int32_t *indices,
  * dqrm_train_step_sorted then runs forward, gradient summation, INT8 quantisation and update
  * for the same batch.  The sorted order travels in `workspace` (dqrm_workspace_bytes): pass
  * the same workspace to both calls and to nothing in between; two workspaces used alternately
- * let batch k+1 be sorted on one stream while batch k trains on another.  The caller orders
- * the two calls (same stream, or an event).  One dqrm_sort_batch serves ONE
+ * let batch k+1 be sorted on one stream while batch k trains on another.  dqrm_sort_batch
+ * records an event behind the sort and dqrm_train_step_sorted puts its gradient summation (not
+ * its forward, which does not need the sorted order) behind that event, so the step's stream
+ * need not wait for the sort's stream.  Exception: when the two calls are made inside different
+ * stream captures, or one inside a capture and one outside, the event cannot connect them and
+ * the caller orders the calls itself (join the sort's stream before the capture ends).  A
+ * workspace is written by the sort and read by the step: the next sort into the same workspace
+ * must be ordered, by the caller, behind the step that used it.  One dqrm_sort_batch serves ONE
  * dqrm_train_step_sorted: the step uses up counters that only the sort resets.  The context
  * keeps, on the host, which workspaces hold a sorted batch that no step has taken yet;
  * dqrm_train_step_sorted on a workspace that holds none (never sorted, already used, or sorted

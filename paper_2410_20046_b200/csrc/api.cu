@@ -118,6 +118,8 @@ int dqrm_destroy(dqrm_ctx *ctx)
     if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
     if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
     if (ctx->ev_fwd) cudaEventDestroy(ctx->ev_fwd);
+    for (auto &kv : ctx->sorted)
+        if (kv.second.done) cudaEventDestroy(kv.second.done);
     if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
     if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
     if (ctx->ev_h_start) cudaEventDestroy(ctx->ev_h_start);
@@ -365,8 +367,19 @@ int dqrm_sort_batch(dqrm_ctx *ctx, const int32_t *indices, const int32_t *offset
     const int rc = dq_launch_bwd_sort(ctx, indices, offsets, unique_rows, uniq_off, B, L, workspace, workspace_bytes, st, nullptr);
     {
         std::lock_guard<std::mutex> lock(ctx->sorted_mu);
-        if (rc == DQRM_OK) ctx->sorted[workspace] = std::make_pair(L, B);
-        else ctx->sorted.erase(workspace);
+        dqrm_ctx::SortedBatch &sb = ctx->sorted[workspace];
+        sb.fresh = false;
+        if (rc != DQRM_OK) return rc;
+        if (!sb.done) DQRM_CUDA_TRY(ctx, cudaEventCreateWithFlags(&sb.done, cudaEventDisableTiming));
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        unsigned long long id = 0;
+        DQRM_CUDA_TRY(ctx, cudaStreamGetCaptureInfo(st, &cs, &id));
+        DQRM_CUDA_TRY(ctx, cudaEventRecord(sb.done, st));
+        sb.captured = cs == cudaStreamCaptureStatusActive;
+        sb.capture_id = id;
+        sb.L = L;
+        sb.B = B;
+        sb.fresh = true;
     }
     return rc;
 }
@@ -382,12 +395,19 @@ int dqrm_train_step_sorted(dqrm_ctx *ctx, float *tables, const int32_t *indices,
         return DQRM_ERR_INVALID_ARG;
     if (L > 0 && (!indices || !unique_rows || !grad_rows || !codes)) return DQRM_ERR_INVALID_ARG;
     if (!ws_ok(workspace, workspace_bytes, dq_bwd_ws_bytes(ctx, L, (int64_t)ctx->T * B))) return DQRM_ERR_WORKSPACE;
+    cudaEvent_t sort_done = nullptr;
+    bool sort_captured = false;
+    unsigned long long sort_capture_id = 0;
     {   // the workspace must hold this batch, sorted by dqrm_sort_batch and not consumed yet: the summation
         // trusts the segment lists in it and zeroes nothing itself
         std::lock_guard<std::mutex> lock(ctx->sorted_mu);
         auto it = ctx->sorted.find(workspace);
-        if (it == ctx->sorted.end() || it->second.first != L || it->second.second != B) return DQRM_ERR_NOT_SORTED;
-        ctx->sorted.erase(it);
+        if (it == ctx->sorted.end() || !it->second.fresh || it->second.L != L || it->second.B != B)
+            return DQRM_ERR_NOT_SORTED;
+        it->second.fresh = false;
+        sort_done = it->second.done;
+        sort_captured = it->second.captured;
+        sort_capture_id = it->second.capture_id;
     }
     cudaStream_t st = as_stream(stream);
     if (ctx->prof_on) dq_mark(ctx, st, DQ_K_BEGIN);
@@ -397,6 +417,16 @@ int dqrm_train_step_sorted(dqrm_ctx *ctx, float *tables, const int32_t *indices,
     if (overlap) {
         DQRM_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_fork, st));
         DQRM_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
+    }
+    {   // only the summation needs the sorted order: it, not the forward, is put behind the sort's event.  An event
+        // recorded inside one stream capture cannot be waited for from another capture or from outside (and the
+        // other way round); there the caller's own ordering of the two calls is all there is.
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        unsigned long long id = 0;
+        DQRM_CUDA_TRY(ctx, cudaStreamGetCaptureInfo(st, &cs, &id));
+        const bool captured = cs == cudaStreamCaptureStatusActive;
+        if (captured == sort_captured && (!captured || id == sort_capture_id))
+            DQRM_CUDA_TRY(ctx, cudaStreamWaitEvent(ss, sort_done, 0));
     }
     int rc = dq_launch_bwd_reduce(ctx, grad_out, uniq_off, grad_rows, B, L, workspace, workspace_bytes, ss);
     int rc2 = dq_launch_fwd(ctx, tables, indices, offsets, scales, bits, out, nullptr, B, L, st);

@@ -33,9 +33,19 @@ struct dqrm_ctx {
     cudaEvent_t ev_h_free[2] = {nullptr, nullptr}, ev_h_idx = nullptr;
     bool h_set_used[2] = {false, false};
     unsigned host_calls = 0;
-    // workspaces that hold a sorted batch nobody has consumed yet: pointer -> (L, B); host bookkeeping only
+    // what the context knows, on the host, about each workspace dqrm_sort_batch has written: whether it holds a
+    // sorted batch that no step has taken yet, of which size, and the event recorded behind that sort (with the
+    // stream capture it was recorded in, if any)
+    struct SortedBatch {
+        bool fresh = false;
+        int64_t L = 0;
+        int B = 0;
+        cudaEvent_t done = nullptr;
+        bool captured = false;
+        unsigned long long capture_id = 0;
+    };
     std::mutex sorted_mu;
-    std::unordered_map<const void *, std::pair<int64_t, int>> sorted;
+    std::unordered_map<const void *, SortedBatch> sorted;
     int overlap = 1;                // 0: keep everything on the caller's stream
     int payload_position = 0;       // sort payload: 0 = row of grad_out, 1 = position of the lookup (set by the merge)
     // kernels whose dynamic shared-memory limit has been raised on this context's device (the attribute is

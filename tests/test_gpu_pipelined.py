@@ -156,6 +156,61 @@ def test_step_on_a_workspace_without_a_fresh_sort_is_refused():
     c.ctx.close()
 
 
+def test_step_waits_for_its_sort_without_the_callers_help():
+    """The gradient summation is ordered behind the sort by an event the context keeps with the workspace: the
+    sort of the next batch runs on another stream, held back there by a long wait so that it is certainly late,
+    and the step's stream never waits for that stream.  The trajectory must equal the single-call loop's."""
+    import torch
+
+    wl = W.scaled_down(W.terabyte(), total_rows=400_000, B=1500, name="terabyte_small")
+    c = Case(wl)
+    tables = W.tables_np(wl)
+    steps = 5
+    batches = [c.batch(s) for s in range(steps)]
+    Lmax = max(len(b[0]) for b in batches)
+    res = []
+    for split in (False, True):
+        d_tables = c.dev(tables)
+        scales = c.empty(wl.T, torch.float32)
+        c.ctx.scale_refresh(d_tables, c.bits, scales)
+        out = c.empty((wl.B, wl.T, wl.D), torch.float32)
+        urs = [torch.full((Lmax,), -1, dtype=torch.int32, device="cuda") for _ in range(2)]
+        uos = [c.empty(wl.T + 1, torch.int32) for _ in range(2)]
+        gr = torch.zeros((Lmax, wl.D), dtype=torch.float32, device="cuda")
+        codes = torch.zeros((Lmax, wl.D), dtype=torch.int8, device="cuda")
+        gs = c.empty(wl.T, torch.float32)
+        dev = [(c.dev(i), c.dev(o), c.dev(g), len(i)) for i, o, g in batches]
+        torch.cuda.synchronize()
+        outs = []
+        if not split:
+            for i, o, g, L in dev:
+                c.ctx.train_step(d_tables, i, o, g, scales, c.bits, out, urs[0], uos[0], gr, codes, gs, wl.lr, B=wl.B, L=L)
+                outs.append(out.cpu().numpy().copy())
+        else:
+            main, side = torch.cuda.Stream(), torch.cuda.Stream()
+            c.ctx.sort_batch(dev[0][0], dev[0][1], urs[0], uos[0], B=wl.B, L=dev[0][3], ws=0, stream=side)
+            for k, (i, o, g, L) in enumerate(dev):
+                slot = k & 1
+                if k + 1 < steps:
+                    ni, no, _, nL = dev[k + 1]
+                    side.wait_stream(main)                  # the other workspace's previous batch has trained
+                    with torch.cuda.stream(side):
+                        torch.cuda._sleep(4_000_000)        # a few milliseconds: this sort is late
+                    c.ctx.sort_batch(ni, no, urs[slot ^ 1], uos[slot ^ 1], B=wl.B, L=nL, ws=slot ^ 1, stream=side)
+                c.ctx.train_step_sorted(d_tables, i, o, g, scales, c.bits, out, urs[slot], uos[slot], gr, codes, gs,
+                                        wl.lr, B=wl.B, L=L, ws=slot, stream=main)
+                main.synchronize()
+                outs.append(out.cpu().numpy().copy())
+            side.synchronize()
+        c.ctx.raise_on_device_error()
+        res.append((d_tables.cpu().numpy(), outs, gr.cpu().numpy()[:dev[-1][3]], codes.cpu().numpy()[:dev[-1][3]]))
+    (ta, oa, ga, ca), (tb, ob, gb, cb) = res
+    assert bit_equal(ta, tb)
+    for x, y in zip(oa, ob):
+        assert bit_equal(x, y)
+    c.ctx.close()
+
+
 def test_sort_held_until_the_forward_is_done_equals_one_call():
     """dqrm_stream_wait_forward: the next batch's sort starts only behind this batch's forward and runs
     beside the rest of the step; the trajectory must equal the single-call loop's bit for bit."""
