@@ -355,6 +355,9 @@ def measure(args, wl, where, primary):
     codes = torch.empty((Lmax, wl.D), dtype=torch.int8, device="cuda")
     gs = torch.empty(wl.T, dtype=torch.float32, device="cuda")
 
+    summaries = args.refresh_mode == "summary"
+    if summaries:       # per-row (min, max) kept current by the update kernels: a refresh reads 8 bytes per row
+        ctx.row_summary_attach(tables)
     ctx.scale_refresh(tables, bits, scales)          # the steps before the first timed refresh use real scales too
 
     def launch_step(bi):
@@ -545,6 +548,11 @@ def measure(args, wl, where, primary):
 
     peak, peak_kind = measured_peak()
     ab = algorithmic_bytes(wl, Lavg, G, Uavg)
+    if summaries:       # what that refresh reads, and what the updates write on top of the rows
+        ab["refresh"] = 8 * int(wl.row_off()[-1])
+        ab["quant_update"] += 8 * Uavg
+        ab["step"] += 8 * Uavg
+        ab["step_separate_calls"] += 8 * Uavg
     dominant = max((k for k in prof if k in KERNEL_BYTES), key=lambda k: prof[k][0])
     dom_bytes = KERNEL_BYTES[dominant](ab, wl, Lavg, G, Uavg)
     dom_s = prof[dominant][0] * 1e-3 / prof[dominant][1]
@@ -614,7 +622,9 @@ def measure(args, wl, where, primary):
                           "separate_calls_frac_of_8TBps_nominal": round(step_gbs_sep / NOMINAL_HBM_GBS, 4)},
         # the same with one refresh charged every `period` steps (its own measured time and its bytes), whatever
         # --steps was
-        "refresh": {"us": None if refresh_us is None else round(refresh_us, 2), "bytes": int(ab["refresh"]),
+        "refresh": {"mode": ("per-row (min, max) summaries, 8 bytes per row, kept current by the update kernels"
+                             if summaries else "scan of the tables"),
+                    "us": None if refresh_us is None else round(refresh_us, 2), "bytes": int(ab["refresh"]),
                     "period": wl.period, "us_per_step_amortised": round(amortised_us, 3),
                     "lookups_per_s_amortised": Lavg * world / (amortised_us * 1e-6),
                     "bytes_per_step_amortised": int(amortised_bytes),
@@ -803,6 +813,9 @@ def main():
                     help="priority of the stream the training half runs on (0: torch's current stream)")
     ap.add_argument("--sort-after-forward", type=int, default=0,
                     help="1: the next batch's sort waits for this batch's forward and runs beside the rest of the step")
+    ap.add_argument("--refresh-mode", choices=("scan", "summary"), default="scan",
+                    help="scan: every refresh reads the whole tables (the paper's refresh); summary: the library keeps "
+                         "(min, max) of every row current as it updates rows and a refresh reads those, same scales")
     ap.add_argument("--join-every-step", action="store_true",
                     help="make every step wait for the next batch's sort before the following step begins "
                          "(default: only that step's gradient summation waits; its forward starts at once)")

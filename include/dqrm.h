@@ -106,6 +106,29 @@ int dqrm_scale_refresh(dqrm_ctx *ctx, const float *tables, const int32_t *bits,
                        float *scales, float *minmax,
                        void *workspace, size_t workspace_bytes, void *stream);
 
+/* Row summaries (no counterpart in the paper; Section 3.2 states the cost they remove: finding a
+ * table's range means reading the whole table, which is why the paper refreshes the scales
+ * only every P iterations).  A training step changes only the rows it touches, so the library
+ * can keep (min, max) of every row, 8 bytes per row in memory the caller provides, current as
+ * it writes rows; dqrm_scale_refresh then reads the summaries, 8 bytes per row instead of 4*D,
+ * and returns the same scales and minmax as the scan of the tables (min and max do not depend
+ * on how the elements are grouped).
+ *   dqrm_row_summary_bytes   bytes the summary needs: 8 * sum R_t
+ *   dqrm_row_summary_attach  scans `tables` once, writes every row's (min, max) to `summary`
+ *                            (device memory, 8-byte aligned, owned by the caller, kept until
+ *                            detach or dqrm_destroy); from then on dqrm_row_update,
+ *                            dqrm_train_step*, dqrm_dp_merge_update keep the entries of the rows
+ *                            they write current and dqrm_scale_refresh ignores its `tables`
+ *                            argument's contents and reads the summary.  The calls that follow
+ *                            must be ordered behind `stream` by the caller.  Rows changed by
+ *                            anyone else make the summary stale: attach again.
+ *   dqrm_row_summary_detach  dqrm_scale_refresh scans the tables again
+ * Errors: DQRM_ERR_INVALID_ARG (null or misaligned), DQRM_ERR_WORKSPACE (summary too small). */
+size_t dqrm_row_summary_bytes(const dqrm_ctx *ctx);
+int dqrm_row_summary_attach(dqrm_ctx *ctx, const float *tables, void *summary,
+                            size_t summary_bytes, void *stream);
+int dqrm_row_summary_detach(dqrm_ctx *ctx);
+
 /* Forward (Section 3.1, Figure 2(b)): for every bag, gather its rows from the FP32
  * master table, fake-quantise each gathered row with its table's stored scale and bit
  * width, and sum over the bag (in bag order, FP64 accumulator, rounded once):

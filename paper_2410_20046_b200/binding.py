@@ -43,6 +43,9 @@ SIGNATURES = {
     "dqrm_train_step": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _f, _i, _i64,
                              _vp, _sz, _vp]),
     "dqrm_stream_wait_forward": (_i, [_vp, _vp]),
+    "dqrm_row_summary_bytes": (_sz, [_vp]),
+    "dqrm_row_summary_attach": (_i, [_vp, _vp, _vp, _sz, _vp]),
+    "dqrm_row_summary_detach": (_i, [_vp]),
     "dqrm_host_step_workspace_bytes": (_sz, [_vp, _i64, _i64]),
     "dqrm_train_step_host": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _f, _i, _i64, _vp, _sz, _vp]),
     "dqrm_grad_quant_int8_static": (_i, [_i, _i, _vp, _vp, _vp, _vp, _vp]),
@@ -352,6 +355,20 @@ class Context:
 
     def stream_wait_forward(self, stream):
         self._check("dqrm_stream_wait_forward", self.lib.dqrm_stream_wait_forward(self._h, _stream(stream)))
+
+    def row_summary_attach(self, tables, stream=None):
+        """Allocates the per-row (min, max) buffer, fills it from `tables` and attaches it."""
+        import torch
+
+        n = int(self.lib.dqrm_row_summary_bytes(self._h))
+        self.row_summary = torch.empty(max(n, 8) // 4, dtype=torch.float32, device=tables.device)
+        self._check("dqrm_row_summary_attach", self.lib.dqrm_row_summary_attach(
+            self._h, _ptr(tables), _ptr(self.row_summary), n, _stream(stream)))
+        return self.row_summary
+
+    def row_summary_detach(self):
+        self._check("dqrm_row_summary_detach", self.lib.dqrm_row_summary_detach(self._h))
+        self.row_summary = None
 
     def train_step_host(self, tables, h_indices, h_offsets, h_grad_out, scales, bits, h_out, lr, *, B, L,
                         stream=None):

@@ -2,6 +2,7 @@
 // and the order of kernel launches.  No arithmetic of the method lives here.
 #include <new>
 #include <string.h>
+#include <stdint.h>
 #include "common.cuh"
 
 namespace {
@@ -439,6 +440,27 @@ int dqrm_train_step_sorted(dqrm_ctx *ctx, float *tables, const int32_t *indices,
     if (rc2 != DQRM_OK) return rc2;
     return dq_launch_quant_update(ctx, tables, unique_rows, uniq_off, grad_rows, dq_bwd_absmax_bits(ctx, L, workspace),
                                   codes, grad_scales, lr, st);
+}
+
+size_t dqrm_row_summary_bytes(const dqrm_ctx *ctx)
+{
+    return ctx ? (size_t)ctx->total_rows * sizeof(float2) : 0;
+}
+
+int dqrm_row_summary_attach(dqrm_ctx *ctx, const float *tables, void *summary, size_t summary_bytes, void *stream)
+{
+    if (!ctx || !tables || !summary || ((uintptr_t)summary & 7u)) return DQRM_ERR_INVALID_ARG;
+    if (summary_bytes < dqrm_row_summary_bytes(ctx)) return DQRM_ERR_WORKSPACE;
+    const int rc = dq_launch_row_summary(ctx, tables, reinterpret_cast<float2 *>(summary), as_stream(stream));
+    if (rc == DQRM_OK) ctx->row_summary = reinterpret_cast<float2 *>(summary);
+    return rc;
+}
+
+int dqrm_row_summary_detach(dqrm_ctx *ctx)
+{
+    if (!ctx) return DQRM_ERR_INVALID_ARG;
+    ctx->row_summary = nullptr;
+    return DQRM_OK;
 }
 
 int dqrm_stream_wait_forward(dqrm_ctx *ctx, void *stream)

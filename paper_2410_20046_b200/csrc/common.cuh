@@ -33,6 +33,7 @@ struct dqrm_ctx {
     cudaEvent_t ev_h_free[2] = {nullptr, nullptr}, ev_h_idx = nullptr;
     bool h_set_used[2] = {false, false};
     unsigned host_calls = 0;
+    float2 *row_summary = nullptr;  // [total_rows] (min, max) of every row, caller's memory; null: not kept
     // what the context knows, on the host, about each workspace dqrm_sort_batch has written: whether it holds a
     // sorted batch that no step has taken yet, of which size, and the event recorded behind that sort (with the
     // stream capture it was recorded in, if any)
@@ -231,6 +232,30 @@ __device__ __forceinline__ int dq_table_of(const int64_t *row_off, int T, int64_
 // ---------------------------------------------------------------------------------
 // host launchers (one per translation unit)
 // ---------------------------------------------------------------------------------
+// (min, max) of a row's new values, folded over the LPR lanes that hold the row (all of them call this together;
+// lane groups are aligned to LPR within the warp).  In the first exchange the even lane of a pair takes over the
+// pair's min and the odd lane its max, so that from then on every lane folds one value with one shuffle per
+// level; the group's first lane ends up with the row's min, the second with its max, and each stores its own.
+template <int LPR>
+__device__ __forceinline__ void dq_store_row_minmax(float2 *__restrict__ row_summary, int64_t arena_row, float mn, float mx)
+{
+    if (LPR == 1) {
+        row_summary[arena_row] = make_float2(mn, mx);
+        return;
+    }
+    const unsigned lane_w = threadIdx.x & 31;
+    const unsigned mask = LPR == 32 ? 0xffffffffu : (((1u << LPR) - 1u) << (lane_w / LPR * LPR));
+    const bool odd = lane_w & 1u;
+    const float other = __shfl_xor_sync(mask, odd ? mn : mx, 1);
+    float v = odd ? fmaxf(mx, other) : fminf(mn, other);
+#pragma unroll
+    for (int o = 2; o < LPR; o <<= 1) {
+        const float r = __shfl_xor_sync(mask, v, o);
+        v = odd ? fmaxf(v, r) : fminf(v, r);
+    }
+    if (lane_w % LPR < 2) reinterpret_cast<float *>(row_summary + arena_row)[odd ? 1 : 0] = v;
+}
+
 size_t dq_refresh_ws_bytes(const dqrm_ctx *ctx);
 int dq_launch_refresh(dqrm_ctx *ctx, const float *tables, const int32_t *bits, float *scales,
                       float *minmax, void *ws, size_t ws_bytes, cudaStream_t st);
@@ -276,6 +301,7 @@ int dq_launch_grad_quant(dqrm_ctx *ctx, const float *grad_rows, const int32_t *u
                          float *grad_scales, void *ws, size_t ws_bytes, cudaStream_t st);
 int dq_launch_row_update(dqrm_ctx *ctx, float *tables, const int32_t *unique_rows, const int32_t *uniq_off,
                          const int8_t *codes, const float *grad_scales, float lr, cudaStream_t st);
+int dq_launch_row_summary(dqrm_ctx *ctx, const float *tables, float2 *summary, cudaStream_t st);
 int dq_launch_quant_update(dqrm_ctx *ctx, float *tables, const int32_t *unique_rows, const int32_t *uniq_off,
                            const float *grad_rows, const u32 *absmax_bits, int8_t *codes,
                            float *grad_scales, float lr, cudaStream_t st);

@@ -93,7 +93,7 @@ dp_sum_update_kernel(float *__restrict__ tables, const int64_t *__restrict__ row
                      const int32_t *__restrict__ union_rows, const int32_t *__restrict__ union_off,
                      const u32 *__restrict__ seg_start, const u32 *__restrict__ vals, const u32 *__restrict__ src,
                      const int8_t *__restrict__ codes_cat, const float *__restrict__ grad_scales, float lr,
-                     int32_t *__restrict__ sums_out, int T, int D, int64_t n_src)
+                     int32_t *__restrict__ sums_out, int T, int D, int64_t n_src, float2 *__restrict__ row_summary)
 {
     extern __shared__ unsigned char smem_raw[];
     int32_t *s_uoff = reinterpret_cast<int32_t *>(smem_raw);
@@ -131,7 +131,9 @@ dp_sum_update_kernel(float *__restrict__ tables, const int64_t *__restrict__ row
                 }
             }
         }
-        float4 *wrow = reinterpret_cast<float4 *>(tables + (r0 + __ldg(union_rows + u)) * D);
+        const int64_t arena_row = r0 + __ldg(union_rows + u);
+        float4 *wrow = reinterpret_cast<float4 *>(tables + arena_row * D);
+        float row_mn = __int_as_float(0x7f800000), row_mx = __int_as_float(0xff800000);
 #pragma unroll
         for (int ch = 0; ch < CH; ++ch) {
             const int c4 = ch * LPR + lane;
@@ -144,8 +146,11 @@ dp_sum_update_kernel(float *__restrict__ tables, const int64_t *__restrict__ row
                 x.z = __fsub_rn(x.z, __fmul_rn(lr, __fmul_rn((float)acc[ch][2], s)));
                 x.w = __fsub_rn(x.w, __fmul_rn(lr, __fmul_rn((float)acc[ch][3], s)));
                 wrow[c4] = x;
+                row_mn = fminf(row_mn, fminf(fminf(x.x, x.y), fminf(x.z, x.w)));
+                row_mx = fmaxf(row_mx, fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w)));
             }
         }
+        if (row_summary) dq_store_row_minmax<LPR>(row_summary, arena_row, row_mn, row_mx);   // (uniform per lane group)
     }
 }
 
@@ -157,7 +162,8 @@ int launch_sum_update(dqrm_ctx *ctx, float *tables, const int32_t *union_rows, c
     const size_t smem = (size_t)(ctx->T + 1) * sizeof(int32_t);
     dp_sum_update_kernel<LPR, CH><<<ctx->num_sms * 8, 256, smem, st>>>(tables, ctx->d_row_off, union_rows, union_off,
                                                                        seg_start, vals, src, codes_cat, grad_scales, lr,
-                                                                       sums_out, ctx->T, ctx->D, n_src);
+                                                                       sums_out, ctx->T, ctx->D, n_src,
+                                                                       ctx->row_summary);
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
     dq_mark(ctx, st, DQ_K_DP_SUM_UPDATE);
     return DQRM_OK;

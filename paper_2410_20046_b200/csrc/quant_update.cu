@@ -58,17 +58,17 @@ absmax_kernel(const float *__restrict__ grad_rows, const int32_t *__restrict__ u
         if (s_max[t]) atomicMax(&absmax[t], s_max[t]);
 }
 
-template <int MODE, int LPR, int CH, bool EXACT>
+template <int MODE, int LPR, int CH, bool EXACT, bool TRACK = false>
 __global__ void __launch_bounds__(QU_THREADS)
 row_stream_kernel(float *__restrict__ tables, const int64_t *__restrict__ row_off,
                   const int32_t *__restrict__ unique_rows, const int32_t *__restrict__ uniq_off,
                   const float *__restrict__ grad_rows, const u32 *__restrict__ absmax,
                   int8_t *__restrict__ codes, float *__restrict__ grad_scales, float lr, int T, int D_any,
-                  int *__restrict__ status)
+                  int *__restrict__ status, float2 *__restrict__ row_summary)
 {
     extern __shared__ unsigned char smem_raw[];
-    row_stream_body<MODE, LPR, CH, EXACT>(smem_raw, tables, row_off, unique_rows, uniq_off, grad_rows, absmax, codes,
-                                          grad_scales, lr, T, D_any, status);
+    row_stream_body<MODE, LPR, CH, EXACT, TRACK>(smem_raw, tables, row_off, unique_rows, uniq_off, grad_rows, absmax,
+                                                 codes, grad_scales, lr, T, D_any, status, row_summary);
 }
 
 template <int MODE, int LPR, int CH>
@@ -78,14 +78,20 @@ int launch_rows(dqrm_ctx *ctx, float *tables, const int32_t *unique_rows, const 
 {
     const size_t smem = (size_t)(ctx->T + 1) * sizeof(int32_t) + (size_t)ctx->T * sizeof(float);
     int grid = ctx->num_sms * 8;      // U lives on the device: a fixed grid splits the rows evenly
-    if (ctx->D == 4 * LPR * CH)
-        row_stream_kernel<MODE, LPR, CH, true><<<grid, QU_THREADS, smem, st>>>(
-            tables, ctx->d_row_off, unique_rows, uniq_off, grad_rows, absmax, codes, grad_scales, lr, ctx->T, ctx->D,
-            ctx->d_status);
-    else
-        row_stream_kernel<MODE, LPR, CH, false><<<grid, QU_THREADS, smem, st>>>(
-            tables, ctx->d_row_off, unique_rows, uniq_off, grad_rows, absmax, codes, grad_scales, lr, ctx->T, ctx->D,
-            ctx->d_status);
+    // with a row summary attached, every kernel that writes master rows keeps the rows' (min, max) current
+    float2 *summary = MODE == MODE_QUANT ? nullptr : ctx->row_summary;
+#define DQ_ROW_STREAM(EXACT, TRACK)                                                                               \
+    row_stream_kernel<MODE, LPR, CH, EXACT, TRACK><<<grid, QU_THREADS, smem, st>>>(                                \
+        tables, ctx->d_row_off, unique_rows, uniq_off, grad_rows, absmax, codes, grad_scales, lr, ctx->T, ctx->D, \
+        ctx->d_status, summary)
+    if (ctx->D == 4 * LPR * CH) {
+        if (summary) DQ_ROW_STREAM(true, (MODE != MODE_QUANT));
+        else DQ_ROW_STREAM(true, false);
+    } else {
+        if (summary) DQ_ROW_STREAM(false, (MODE != MODE_QUANT));
+        else DQ_ROW_STREAM(false, false);
+    }
+#undef DQ_ROW_STREAM
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
     dq_mark(ctx, st, MODE == MODE_QUANT ? DQ_K_QUANT : (MODE == MODE_UPDATE ? DQ_K_UPDATE : DQ_K_QUANT_UPDATE));
     return DQRM_OK;

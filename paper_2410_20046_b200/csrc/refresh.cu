@@ -14,7 +14,14 @@ namespace {
 
 constexpr int RF_THREADS = 512;
 constexpr int RF_UNROLL = 8;
-constexpr int RF_CHUNK4 = RF_THREADS * RF_UNROLL;   // float4 per chunk (64 KB)
+constexpr int RF_CHUNK4 = RF_THREADS * RF_UNROLL;   // vectors per chunk (64 KB of float4)
+
+// What one vector contributes: a float4 of table elements its smallest and largest element, a float2 of
+// the per-row summary (min, max of one row) its two fields.
+__device__ __forceinline__ float vec_min(const float4 &v) { return fminf(fminf(v.x, v.y), fminf(v.z, v.w)); }
+__device__ __forceinline__ float vec_max(const float4 &v) { return fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)); }
+__device__ __forceinline__ float vec_min(const float2 &v) { return v.x; }
+__device__ __forceinline__ float vec_max(const float2 &v) { return v.y; }
 
 // order-preserving map float -> uint32 (so that unsigned min/max order like the floats)
 __device__ __forceinline__ u32 f2ord(float f)
@@ -28,8 +35,11 @@ __device__ __forceinline__ float ord2f(u32 o)
     return __uint_as_float(b);
 }
 
+// V = float4: arena4 is the arena of tables, d4 = D/4 vectors per row.  V = float2: arena4 is the per-row
+// summary, d4 = 1.
+template <typename V>
 __global__ void __launch_bounds__(RF_THREADS)
-refresh_kernel(const float4 *__restrict__ arena4, const int64_t *__restrict__ row_off, int T, int D,
+refresh_kernel(const V *__restrict__ arena4, const int64_t *__restrict__ row_off, int T, int d4,
                int64_t n4, const int32_t *__restrict__ bits, float *__restrict__ scales,
                float *__restrict__ minmax, u32 *__restrict__ partials /*[grid][T][2]*/,
                u32 *__restrict__ done)
@@ -40,7 +50,6 @@ refresh_kernel(const float4 *__restrict__ arena4, const int64_t *__restrict__ ro
     u32 *s_max = s_min + T;                                              // [T]
     __shared__ bool is_last;
 
-    const int d4 = D >> 2;
     for (int t = threadIdx.x; t <= T; t += RF_THREADS) v4_off[t] = row_off[t] * d4;
     for (int t = threadIdx.x; t < T; t += RF_THREADS) { s_min[t] = 0xFFFFFFFFu; s_max[t] = 0u; }
     __syncthreads();
@@ -53,20 +62,20 @@ refresh_kernel(const float4 *__restrict__ arena4, const int64_t *__restrict__ ro
         const int t0 = dq_table_of(v4_off, T, c0);
         if (c1 <= v4_off[t0 + 1]) {
             // whole chunk inside table t0
-            float4 v[RF_UNROLL];
+            V v[RF_UNROLL];
 #pragma unroll
             for (int k = 0; k < RF_UNROLL; ++k) {
                 int64_t i = c0 + k * RF_THREADS + threadIdx.x;
                 if (i < c1) v[k] = __ldcs(arena4 + i);
-                else v[k] = make_float4(__int_as_float(0x7fc00000), 0.f, 0.f, 0.f);   // marker, skipped below
+                else v[k] = V();                                                      // skipped below
             }
             float mn = __int_as_float(0x7f800000), mx = __int_as_float(0xff800000);   // +inf, -inf
 #pragma unroll
             for (int k = 0; k < RF_UNROLL; ++k) {
                 int64_t i = c0 + k * RF_THREADS + threadIdx.x;
                 if (i < c1) {
-                    mn = fminf(fminf(mn, v[k].x), fminf(v[k].y, fminf(v[k].z, v[k].w)));
-                    mx = fmaxf(fmaxf(mx, v[k].x), fmaxf(v[k].y, fmaxf(v[k].z, v[k].w)));
+                    mn = fminf(mn, vec_min(v[k]));
+                    mx = fmaxf(mx, vec_max(v[k]));
                 }
             }
 #pragma unroll
@@ -81,12 +90,13 @@ refresh_kernel(const float4 *__restrict__ arena4, const int64_t *__restrict__ ro
         } else {
             // chunk straddles a table boundary (at most T-1 such chunks in the arena)
             for (int64_t i = c0 + threadIdx.x; i < c1; i += RF_THREADS) {
-                float4 v = __ldcs(arena4 + i);
+                V v = __ldcs(arena4 + i);
                 int t = dq_table_of(v4_off, T, i);
-                float mn = fminf(fminf(v.x, v.y), fminf(v.z, v.w));
-                float mx = fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w));
-                atomicMin(&s_min[t], f2ord(mn));
-                atomicMax(&s_max[t], f2ord(mx));
+                float mn = vec_min(v), mx = vec_max(v);
+                if (mn <= mx) {
+                    atomicMin(&s_min[t], f2ord(mn));
+                    atomicMax(&s_max[t], f2ord(mx));
+                }
             }
         }
     }
@@ -140,12 +150,59 @@ int dq_launch_refresh(dqrm_ctx *ctx, const float *tables, const int32_t *bits, f
                       float *minmax, void *ws, size_t ws_bytes, cudaStream_t st)
 {
     if (ws_bytes < dq_refresh_ws_bytes(ctx)) return DQRM_ERR_WORKSPACE;
-    const int64_t n4 = ctx->total_rows * (ctx->D / 4);
     const int grid = refresh_grid(ctx);
     size_t smem = (size_t)(ctx->T + 1) * sizeof(int64_t) + (size_t)ctx->T * 2 * sizeof(u32);
-    refresh_kernel<<<grid, RF_THREADS, smem, st>>>(reinterpret_cast<const float4 *>(tables), ctx->d_row_off,
-                                                   ctx->T, ctx->D, n4, bits, scales, minmax,
-                                                   reinterpret_cast<u32 *>(ws), ctx->d_done);
+    if (ctx->row_summary) {
+        // every row's (min, max) is kept current by the update kernels: 8 bytes per row are read, not 4*D
+        refresh_kernel<float2><<<grid, RF_THREADS, smem, st>>>(ctx->row_summary, ctx->d_row_off, ctx->T, 1,
+                                                               ctx->total_rows, bits, scales, minmax,
+                                                               reinterpret_cast<u32 *>(ws), ctx->d_done);
+    } else {
+        const int64_t n4 = ctx->total_rows * (ctx->D / 4);
+        refresh_kernel<float4><<<grid, RF_THREADS, smem, st>>>(reinterpret_cast<const float4 *>(tables), ctx->d_row_off,
+                                                               ctx->T, ctx->D / 4, n4, bits, scales, minmax,
+                                                               reinterpret_cast<u32 *>(ws), ctx->d_done);
+    }
+    DQRM_CUDA_TRY(ctx, cudaGetLastError());
+    dq_mark(ctx, st, DQ_K_REFRESH);
+    return DQRM_OK;
+}
+
+namespace {
+
+// (min, max) of every row of the arena, a lane group per row
+__global__ void __launch_bounds__(256)
+row_summary_kernel(const float4 *__restrict__ arena4, int d4, int lpr, int64_t total_rows, float2 *__restrict__ summary)
+{
+    const int lane = threadIdx.x % lpr;
+    const int64_t group = ((int64_t)blockIdx.x * 256 + threadIdx.x) / lpr;
+    const int64_t n_groups = (int64_t)gridDim.x * 256 / lpr;
+    const unsigned lane_w = threadIdx.x & 31;
+    const unsigned mask = lpr == 32 ? 0xffffffffu : (((1u << lpr) - 1u) << (lane_w / lpr * lpr));
+    for (int64_t r = group; r < total_rows; r += n_groups) {
+        float mn = __int_as_float(0x7f800000), mx = __int_as_float(0xff800000);
+        for (int c = lane; c < d4; c += lpr) {
+            const float4 v = __ldcs(arena4 + r * d4 + c);
+            mn = fminf(mn, vec_min(v));
+            mx = fmaxf(mx, vec_max(v));
+        }
+        for (int o = lpr >> 1; o > 0; o >>= 1) {
+            mn = fminf(mn, __shfl_xor_sync(mask, mn, o));
+            mx = fmaxf(mx, __shfl_xor_sync(mask, mx, o));
+        }
+        if (lane == 0) summary[r] = make_float2(mn, mx);
+    }
+}
+
+}  // namespace
+
+int dq_launch_row_summary(dqrm_ctx *ctx, const float *tables, float2 *summary, cudaStream_t st)
+{
+    const int d4 = ctx->D / 4;
+    int lpr = 1;
+    while (lpr < d4 && lpr < 32) lpr <<= 1;
+    row_summary_kernel<<<ctx->num_sms * 8, 256, 0, st>>>(reinterpret_cast<const float4 *>(tables), d4, lpr,
+                                                         ctx->total_rows, summary);
     DQRM_CUDA_TRY(ctx, cudaGetLastError());
     dq_mark(ctx, st, DQ_K_REFRESH);
     return DQRM_OK;

@@ -30,13 +30,14 @@ template <int CH> struct RowsInFlight { static constexpr int v = CH >= 4 ? 1 : (
 inline size_t smem_bytes(int T) { return (size_t)(T + 1) * sizeof(int32_t) + (size_t)T * sizeof(float); }
 
 // smem_raw: smem_bytes(T) bytes of shared memory; every thread of the block calls this
-template <int MODE, int LPR, int CH, bool EXACT>
+// TRACK: the (min, max) of every row written is stored in row_summary[arena row] as well
+template <int MODE, int LPR, int CH, bool EXACT, bool TRACK = false>
 __device__ __forceinline__ void
 row_stream_body(unsigned char *smem_raw, float *__restrict__ tables, const int64_t *__restrict__ row_off,
                 const int32_t *__restrict__ unique_rows, const int32_t *__restrict__ uniq_off,
                 const float *__restrict__ grad_rows, const u32 *__restrict__ absmax,
                 int8_t *__restrict__ codes, float *__restrict__ grad_scales, float lr, int T, int D_any,
-                int *__restrict__ status)
+                int *__restrict__ status, float2 *__restrict__ row_summary = nullptr)
 {
     constexpr int NB = RowsInFlight<CH>::v;
     const int D = EXACT ? 4 * LPR * CH : D_any;
@@ -105,6 +106,7 @@ row_stream_body(unsigned char *smem_raw, float *__restrict__ tables, const int64
 #pragma unroll
         for (int b = 0; b < NB; ++b) {
             if (b < nb) {
+                float row_mn = __int_as_float(0x7f800000), row_mx = __int_as_float(0xff800000);
 #pragma unroll
                 for (int ch = 0; ch < CH; ++ch) {
                     const int c4 = ch * LPR + lane;
@@ -126,9 +128,16 @@ row_stream_body(unsigned char *smem_raw, float *__restrict__ tables, const int64
                             x.z = __fsub_rn(x.z, __fmul_rn(lr, __fmul_rn(q.z, s)));
                             x.w = __fsub_rn(x.w, __fmul_rn(lr, __fmul_rn(q.w, s)));
                             wrow[b][c4] = x;
+                            if (TRACK) {
+                                row_mn = fminf(row_mn, fminf(fminf(x.x, x.y), fminf(x.z, x.w)));
+                                row_mx = fmaxf(row_mx, fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w)));
+                            }
                         }
                     }
                 }
+                // (nb is the same in all lanes of a group, so all of them arrive here together)
+                if (TRACK && MODE != MODE_QUANT)
+                    dq_store_row_minmax<LPR>(row_summary, (reinterpret_cast<float *>(wrow[b]) - tables) / D, row_mn, row_mx);
             }
         }
         u += nb;

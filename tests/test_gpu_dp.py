@@ -82,4 +82,15 @@ def test_exchange_matches_oracle(name, ranks, oracle):
                         union_rows, union_off, None, ws)
     ctx.raise_on_device_error()
     assert d_tables2.cpu().numpy().tobytes() == o_tables.tobytes()
+    # with a row summary attached the merged update keeps every written row's (min, max) current
+    ctx.set_sort_path(0)
+    d_tables3 = dev(W.tables_np(wl))
+    summary = ctx.row_summary_attach(d_tables3)
+    ctx.dp_merge_update(d_tables3, ranks, stride, rows_cat, uoff_cat, codes_cat, scales, wl.lr, n_entries, max_table,
+                        union_rows, union_off, None, ws)
+    ctx.raise_on_device_error()
+    assert d_tables3.cpu().numpy().tobytes() == o_tables.tobytes()
+    got = summary.cpu().numpy().reshape(-1, 2)
+    assert (got[:, 0] == o_tables.min(axis=1)).all() and (got[:, 1] == o_tables.max(axis=1)).all()
+    ctx.row_summary_detach()
     ctx.close()
