@@ -311,6 +311,7 @@ seg_emit_kernel(const u32 *__restrict__ keys, int64_t L, const u32 *__restrict__
     __shared__ u32 s_prefix;
     // this thread's keys first: they depend on nothing, so they fly beside the loads of the prefix below
     const int64_t i0 = (int64_t)blockIdx.x * ST_TILE + (int64_t)threadIdx.x * ST_ITEMS;
+    const int ck_shift = 31 - __clz(ck);
     u32 k[ST_ITEMS], prev0; int n;
     load_tile_keys(keys, L, i0, k, prev0, n);
     for (int t = threadIdx.x; t <= T; t += ST_THREADS) s_off[t] = row_off[t];
@@ -379,7 +380,7 @@ seg_emit_kernel(const u32 *__restrict__ keys, int64_t L, const u32 *__restrict__
                 t_prev = t;
             }
             const u32 u_of_i = heads_before - 1;
-            if ((i % ck) == 0) chunk_first[i / ck] = u_of_i;
+            if ((i & (int64_t)(ck - 1)) == 0) chunk_first[i >> ck_shift] = u_of_i;     // ck is 16 or 32
             if (i == L - 1) {
                 const u32 U = u_of_i + 1;
                 seg_start[U] = (u32)L;
