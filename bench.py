@@ -31,7 +31,7 @@ if ROOT not in sys.path:
 
 METRIC = "QAT embedding lookups/sec (fwd+bwd+update)"
 UNIT = "lookups/s"
-N_BATCHES = 16
+N_BATCHES = 20
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
@@ -446,6 +446,9 @@ def measure(args, wl, where, primary):
     spg = args.steps_per_graph
     if spg < 1 or N_BATCHES % spg or wl.period % spg:
         spg = 1
+    # shorter groups for the head and the tail of a timed region that the long groups do not tile
+    group_sizes = [g for g in sorted({spg, 4}, reverse=True) if g > 1 and g <= spg and N_BATCHES % g == 0
+                   and wl.period % g == 0]
     if not args.no_graph and dp_step is None:
         try:
             if pipelined:
@@ -469,8 +472,8 @@ def measure(args, wl, where, primary):
             n_before = ctx.launch_count()
             graphs = [capture(bi, 1) for bi in range(N_BATCHES)]
             launches_per_step = (ctx.launch_count() - n_before) // N_BATCHES    # kernels recorded per step
-            if spg > 1:
-                group_graphs = [capture(b0, spg) for b0 in range(0, N_BATCHES, spg)]
+            if group_sizes:
+                group_graphs = {g: [capture(b0, g) for b0 in range(0, N_BATCHES, g)] for g in group_sizes}
             torch.cuda.synchronize()
         except Exception as e:                       # capture refused: plain launches
             print(f"bench: CUDA graph capture failed ({e}); launching directly", file=sys.stderr)
@@ -481,7 +484,7 @@ def measure(args, wl, where, primary):
     refreshes = {"n": 0}     # scale refreshes launched since the timed region began
 
     def step(s, end=None, direct=False):
-        """Runs step s, or steps s .. s+spg-1 from one graph when they all lie before `end`; returns how many."""
+        """Runs step s, or a group of consecutive steps from one graph when they all lie before `end`; returns how many."""
         if s % wl.period == 0:
             ctx.scale_refresh(tables, bits, scales)
             refreshes["n"] += 1
@@ -491,10 +494,12 @@ def measure(args, wl, where, primary):
             return 1
         if pipelined and last["s"] != s - 1:
             prime(s % N_BATCHES)                     # (re)start of the pipeline: this batch is not sorted yet
-        if group_graphs is not None and not direct and s % spg == 0 and end is not None and s + spg <= end:
-            group_graphs[(s % N_BATCHES) // spg].replay()      # no refresh falls inside: spg divides the period
-            last["s"] = s + spg - 1
-            return spg
+        if group_graphs is not None and not direct and end is not None:
+            for g in group_sizes:                    # the longest group that starts here and ends before `end`
+                if s % g == 0 and s + g <= end:
+                    group_graphs[g][(s % N_BATCHES) // g].replay()     # no refresh falls inside: g divides the period
+                    last["s"] = s + g - 1
+                    return g
         last["s"] = s
         if graphs is not None and not direct:
             graphs[s % N_BATCHES].replay()
@@ -615,8 +620,9 @@ def measure(args, wl, where, primary):
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": base_config(wl),
         "run": {"lookups_per_step_per_gpu": Lavg, "unique_rows_per_step": Uavg, "unique_fraction": Uavg / Lavg,
-                "launch": ((f"CUDA graph replay, {spg} consecutive steps per graph" if group_graphs is not None else
-                            "CUDA graph replay per step") if graphs is not None else "direct launches") +
+                "launch": ((f"CUDA graph replay, groups of {group_sizes} consecutive steps per graph, single steps "
+                            "for the rest" if group_graphs is not None else "CUDA graph replay per step")
+                           if graphs is not None else "direct launches") +
                           ("; the index sort of batch k+1 runs on a second stream while batch k trains "
                            "(two workspaces, every step does one sort and one training half)" if pipelined
                            else ""),
@@ -825,8 +831,8 @@ def main():
                          "instead of running independent replicas")
     ap.add_argument("--no-graph", action="store_true", help="launch every step directly instead of replaying CUDA graphs")
     ap.add_argument("--no-overlap", action="store_true", help="keep the index sort on the caller's stream")
-    ap.add_argument("--steps-per-graph", type=int, default=4,
-                    help="consecutive steps replayed from one CUDA graph (must divide 16 and the refresh period, else 1; "
+    ap.add_argument("--steps-per-graph", type=int, default=20,
+                    help="consecutive steps replayed from one CUDA graph (must divide the 20 staged batches and the refresh period, else 1; "
                          "a remainder of the timed region runs from single-step graphs)")
     ap.add_argument("--sort-priority", type=int, default=0,
                     help="priority of the second stream that sorts the next batch (-1 high, 0 default)")

@@ -38,8 +38,8 @@
 #include <stdlib.h>
 #include <string.h>
 
-/* ---- quantiser (Section 4.1: per-table scale; Appendix A: uniform mapping,
- *      static min-max range) ------------------------------------------------ */
+/* ---- quantiser (Section 4.1: one scale per table; Appendix A: evenly spaced
+ *      levels, the clipping range fixed by the table's min and max) --------- */
 
 static int32_t q_max(int bits) { return (int32_t)((1u << (bits - 1)) - 1u); }
 static int32_t q_min(int bits) { return -(int32_t)(1u << (bits - 1)); }
