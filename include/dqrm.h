@@ -186,9 +186,11 @@ int dqrm_train_step(dqrm_ctx *ctx, float *tables, const int32_t *indices,
 /* dqrm_train_step in two calls, for a training loop that knows the next batch's indices
  * while the current batch trains (no counterpart in the paper; Section 4.3 only fixes what the
  * sparse gradient holds).  dqrm_sort_batch does the part of the backward that needs the
- * indices alone: it orders the lookups by row and writes unique_rows and uniq_off.
+ * indices alone: it orders the lookups by row and finds where every row's run begins.
  * dqrm_train_step_sorted then runs forward, gradient summation, INT8 quantisation and update
- * for the same batch.  The sorted order travels in `workspace` (dqrm_workspace_bytes): pass
+ * for the same batch.  unique_rows and uniq_off are outputs of the PAIR of calls: pass the same
+ * buffers to both; they are complete when dqrm_train_step_sorted is (the sort numbers each
+ * table's rows by itself, and the tables' bases are added where the gradients are summed).  The sorted order travels in `workspace` (dqrm_workspace_bytes): pass
  * the same workspace to both calls and to nothing in between; two workspaces used alternately
  * let batch k+1 be sorted on one stream while batch k trains on another.  dqrm_sort_batch
  * records an event behind the sort and dqrm_train_step_sorted puts its gradient summation (not
@@ -210,7 +212,7 @@ int dqrm_sort_batch(dqrm_ctx *ctx, const int32_t *indices, const int32_t *offset
 int dqrm_train_step_sorted(dqrm_ctx *ctx, float *tables, const int32_t *indices,
                            const int32_t *offsets, const float *grad_out,
                            const float *scales, const int32_t *bits, float *out,
-                           const int32_t *unique_rows, const int32_t *uniq_off, float *grad_rows,
+                           int32_t *unique_rows, int32_t *uniq_off, float *grad_rows,
                            int8_t *codes, float *grad_scales, float lr, int B, int64_t L,
                            void *workspace, size_t workspace_bytes, void *stream);
 

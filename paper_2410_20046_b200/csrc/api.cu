@@ -308,9 +308,9 @@ int dqrm_train_step(dqrm_ctx *ctx, float *tables, const int32_t *indices, const 
         DQRM_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_fork, st));
         DQRM_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
     }
-    int rc = dq_launch_bwd_sort(ctx, indices, offsets, unique_rows, uniq_off, B, L, workspace, workspace_bytes, ss, nullptr);
+    int rc = dq_launch_bwd_sort(ctx, indices, offsets, unique_rows, uniq_off, B, L, workspace, workspace_bytes, ss, nullptr, true);
     if (rc == DQRM_OK)
-        rc = dq_launch_bwd_reduce(ctx, grad_out, uniq_off, grad_rows, B, L, workspace, workspace_bytes, ss);
+        rc = dq_launch_bwd_reduce(ctx, grad_out, unique_rows, uniq_off, grad_rows, B, L, workspace, workspace_bytes, ss);
     int rc2 = dq_launch_fwd(ctx, tables, indices, offsets, scales, bits, out, nullptr, B, L, st);
     if (overlap) {   // join even after an error so that the caller's stream stays ordered behind the side stream
         cudaEventRecord(ctx->ev_join, ctx->side);
@@ -365,7 +365,7 @@ int dqrm_sort_batch(dqrm_ctx *ctx, const int32_t *indices, const int32_t *offset
     if (!ws_ok(workspace, workspace_bytes, dq_bwd_ws_bytes(ctx, L, (int64_t)ctx->T * B))) return DQRM_ERR_WORKSPACE;
     cudaStream_t st = as_stream(stream);
     if (ctx->prof_on) dq_mark(ctx, st, DQ_K_BEGIN);
-    const int rc = dq_launch_bwd_sort(ctx, indices, offsets, unique_rows, uniq_off, B, L, workspace, workspace_bytes, st, nullptr);
+    const int rc = dq_launch_bwd_sort(ctx, indices, offsets, unique_rows, uniq_off, B, L, workspace, workspace_bytes, st, nullptr, true);
     {
         std::lock_guard<std::mutex> lock(ctx->sorted_mu);
         dqrm_ctx::SortedBatch &sb = ctx->sorted[workspace];
@@ -387,7 +387,7 @@ int dqrm_sort_batch(dqrm_ctx *ctx, const int32_t *indices, const int32_t *offset
 
 int dqrm_train_step_sorted(dqrm_ctx *ctx, float *tables, const int32_t *indices, const int32_t *offsets,
                            const float *grad_out, const float *scales, const int32_t *bits, float *out,
-                           const int32_t *unique_rows, const int32_t *uniq_off, float *grad_rows, int8_t *codes,
+                           int32_t *unique_rows, int32_t *uniq_off, float *grad_rows, int8_t *codes,
                            float *grad_scales, float lr, int B, int64_t L, void *workspace, size_t workspace_bytes,
                            void *stream)
 {
@@ -429,7 +429,7 @@ int dqrm_train_step_sorted(dqrm_ctx *ctx, float *tables, const int32_t *indices,
         if (captured == sort_captured && (!captured || id == sort_capture_id))
             DQRM_CUDA_TRY(ctx, cudaStreamWaitEvent(ss, sort_done, 0));
     }
-    int rc = dq_launch_bwd_reduce(ctx, grad_out, uniq_off, grad_rows, B, L, workspace, workspace_bytes, ss);
+    int rc = dq_launch_bwd_reduce(ctx, grad_out, unique_rows, uniq_off, grad_rows, B, L, workspace, workspace_bytes, ss);
     int rc2 = dq_launch_fwd(ctx, tables, indices, offsets, scales, bits, out, nullptr, B, L, st);
     cudaEventRecord(ctx->ev_fwd, st);                           // for dqrm_stream_wait_forward
     if (overlap) {
@@ -570,7 +570,7 @@ int dqrm_train_step_host(dqrm_ctx *ctx, float *tables, const int32_t *h_indices,
     DQRM_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
     char *step_ws = ws + y.step_ws;
     const size_t step_ws_bytes = workspace_bytes - y.step_ws;
-    int rc = dq_launch_bwd_sort(ctx, d_idx, d_off, d_ur, d_uo, B, L, step_ws, step_ws_bytes, ctx->side, nullptr);
+    int rc = dq_launch_bwd_sort(ctx, d_idx, d_off, d_ur, d_uo, B, L, step_ws, step_ws_bytes, ctx->side, nullptr, true);
     if (rc == DQRM_OK) rc = dq_launch_fwd(ctx, tables, d_idx, d_off, scales, bits, d_out, nullptr, B, L, st);
     // join every stream even after an error, so that the caller's stream stays ordered behind them
     cudaEventRecord(ctx->ev_h_fwd, st);
@@ -579,7 +579,7 @@ int dqrm_train_step_host(dqrm_ctx *ctx, float *tables, const int32_t *h_indices,
     cudaEventRecord(ctx->ev_h_out, ctx->copy_out);
     // the gradient summation follows the sort on the second stream as soon as the upstream gradient has arrived
     cudaStreamWaitEvent(ctx->side, ctx->ev_h_go, 0);
-    if (rc == DQRM_OK) rc = dq_launch_bwd_reduce(ctx, d_go, d_uo, d_gr, B, L, step_ws, step_ws_bytes, ctx->side);
+    if (rc == DQRM_OK) rc = dq_launch_bwd_reduce(ctx, d_go, d_ur, d_uo, d_gr, B, L, step_ws, step_ws_bytes, ctx->side);
     cudaEventRecord(ctx->ev_join, ctx->side);
     cudaStreamWaitEvent(st, ctx->ev_join, 0);
     if (rc == DQRM_OK)

@@ -39,7 +39,7 @@ struct Layout {
     int64_t num_tiles, num_chunks;             // num_chunks = ceil(L / ck)
     // zeroed at call start: [0, zero_small)
     size_t absmax, counters, tile_heads, zero_small, digit_base, chunk_sum, tilehist;
-    size_t keys_a, vals_a, pairs_a, pairs_b, seg_start, chunk_first, long_list, partials;
+    size_t keys_a, vals_a, pairs_a, pairs_b, seg_start, chunk_first, long_list, partials, table_cnt, tb;
     size_t total;
 };
 
@@ -75,7 +75,9 @@ Layout make_layout(const dqrm_ctx *ctx, int64_t L)
     y.vals_a = take(sizeof(u32) * Lc);
     y.pairs_a = take(sizeof(uint2) * Lc);
     y.pairs_b = take(sizeof(uint2) * Lc);
-    y.seg_start = take(sizeof(u32) * (Lc + 1));
+    y.seg_start = take(sizeof(u32) * (Lc + ctx->T + 1));     // (lists by table: one slot more per table)
+    y.table_cnt = take(sizeof(u32) * ctx->T);
+    y.tb = take(sizeof(u32) * (ctx->T + 1));
     y.chunk_first = take(sizeof(u32) * y.num_chunks);
     y.long_list = take(sizeof(uint4) * y.num_chunks);
     y.partials = take(sizeof(double) * y.num_chunks * 2 * ctx->D);
@@ -396,8 +398,8 @@ seg_emit_kernel(const u32 *__restrict__ keys, int64_t L, const u32 *__restrict__
 // RL/RV/RC: lanes per row, floats per lane vector and vectors per lane of the reduce kernel;
 // LPR/CH: the same for the fix-up kernels (always 128-bit vectors)
 template <int RL, int RV, int RC, int LPR, int CH>
-int launch_reduce(dqrm_ctx *ctx, const Layout &y, char *ws, const u32 *keys, const u32 *vals, const int32_t *uniq_off,
-                  const float *grad_out, float *grad_rows, int64_t L, int64_t G, cudaStream_t st)
+int launch_reduce(dqrm_ctx *ctx, const Layout &y, char *ws, const u32 *keys, const u32 *vals, int32_t *unique_rows,
+                  int32_t *uniq_off, const float *grad_out, float *grad_rows, int64_t L, int64_t G, cudaStream_t st)
 {
     using namespace segred;
     const int64_t cap = (int64_t)ctx->num_sms * 8;
@@ -409,12 +411,18 @@ int launch_reduce(dqrm_ctx *ctx, const Layout &y, char *ws, const u32 *keys, con
     const u32 *seg_start = reinterpret_cast<const u32 *>(ws + y.seg_start);
     double *partials = reinterpret_cast<double *>(ws + y.partials);
     uint4 *long_list = reinterpret_cast<uint4 *>(ws + y.long_list);
-    const size_t red_smem = (size_t)(ctx->T + 1) * sizeof(u32) + (size_t)gpb * 2 * y.ck * sizeof(u32);
+    const size_t red_smem = (size_t)(ctx->T + 1) * 2 * sizeof(u32) + (size_t)gpb * 2 * y.ck * sizeof(u32);
+    ByTable bt;
+    bt.table_cnt = reinterpret_cast<const u32 *>(ws + y.table_cnt);
+    bt.tb = reinterpret_cast<const u32 *>(ws + y.tb);
+    bt.row_off = ctx->d_row_off;
+    bt.unique_rows = unique_rows;
+    bt.uniq_off = uniq_off;
     const u32 *chunk_first = reinterpret_cast<const u32 *>(ws + y.chunk_first);
 #define DQ_LAUNCH_REDUCE(EXACT, CK)                                                                                  \
     seg_reduce_kernel<RL, RV, RC, EXACT, CK><<<grid, 256, red_smem, st>>>(                                          \
         keys, vals, seg_start, chunk_first, uniq_off, grad_out, grad_rows, partials, long_list, counters, absmax,    \
-        ctx->T, ctx->D, L, G, y.num_chunks, ctx->d_status)
+        ctx->T, ctx->D, L, G, y.num_chunks, ctx->d_status, bt)
     const bool exact = ctx->D == RL * RV * RC;
     if constexpr (RL <= 16) {
         if (y.ck == SEG_CHUNK / 2) {
@@ -499,7 +507,7 @@ size_t dq_bwd_ws_bytes(const dqrm_ctx *ctx, int64_t L, int64_t G)
 // segment starts).  It needs no upstream gradient, so a training step runs it beside the forward.
 int dq_launch_bwd_sort(dqrm_ctx *ctx, const int32_t *indices, const int32_t *offsets,
                        int32_t *unique_rows, int32_t *uniq_off, int B, int64_t L,
-                       void *ws_, size_t ws_bytes, cudaStream_t st, const u32 **absmax_bits_out)
+                       void *ws_, size_t ws_bytes, cudaStream_t st, const u32 **absmax_bits_out, bool lists_by_table)
 {
     const Layout y = make_layout(ctx, L);
     if (ws_bytes < y.total) return DQRM_ERR_WORKSPACE;
@@ -535,6 +543,15 @@ int dq_launch_bwd_sort(dqrm_ctx *ctx, const int32_t *indices, const int32_t *off
         ca.status = ctx->d_status;
         ca.payload_position = ctx->payload_position;
         ca.tile_heads = reinterpret_cast<u32 *>(ws + y.tile_heads);
+        // when dq_launch_bwd_reduce follows, the clusters number their own tables' segments and seg_emit is not run
+        ca.lists_by_table = lists_by_table ? 1 : 0;
+        ca.seg_start = reinterpret_cast<u32 *>(ws + y.seg_start);
+        ca.chunk_first = reinterpret_cast<u32 *>(ws + y.chunk_first);
+        ca.table_cnt = reinterpret_cast<u32 *>(ws + y.table_cnt);
+        ca.tb = reinterpret_cast<u32 *>(ws + y.tb);
+        ca.counters = reinterpret_cast<u32 *>(ws + y.counters);
+        ca.ck_shift = y.ck == SEG_CHUNK ? 5 : 4;
+        ca.fmt_slot = segred::CNT_FMT; ca.fmt_by_table = segred::LISTS_BY_TABLE; ca.fmt_broken = segred::LISTS_BROKEN;
         const int64_t per_table = (L + ctx->T - 1) / ctx->T;
         const bool wide = ctx->T * csort::CLUSTER_WIDE * 2 <= ctx->num_sms && per_table >= csort::CLUSTER_WIDE * 1024;
         cudaError_t e = cudaErrorUnknown;
@@ -582,7 +599,8 @@ int dq_launch_bwd_sort(dqrm_ctx *ctx, const int32_t *indices, const int32_t *off
     }
         skeys = keys[0];
     }
-    if (!sorted) {        // (the cluster sort counts the segment heads of every tile on its way out)
+    if (sorted && lists_by_table) return DQRM_OK;      // the lists are there; unique_rows and uniq_off come with the sums
+    if (!sorted) {        // (a cluster sort that did not number the segments itself has counted the segment heads of every tile)
         seg_count_kernel<<<(unsigned)y.num_tiles, ST_THREADS, 0, st>>>(skeys, L, reinterpret_cast<u32 *>(ws + y.tile_heads));
         DQRM_CUDA_TRY(ctx, cudaGetLastError());
         dq_mark(ctx, st, DQ_K_SEG_COUNT);
@@ -597,8 +615,8 @@ int dq_launch_bwd_sort(dqrm_ctx *ctx, const int32_t *indices, const int32_t *off
 }
 
 // second half: segmented sum of the upstream gradient over the sorted lookups
-int dq_launch_bwd_reduce(dqrm_ctx *ctx, const float *grad_out, const int32_t *uniq_off, float *grad_rows, int B, int64_t L,
-                         void *ws_, size_t ws_bytes, cudaStream_t st)
+int dq_launch_bwd_reduce(dqrm_ctx *ctx, const float *grad_out, int32_t *unique_rows, int32_t *uniq_off, float *grad_rows,
+                         int B, int64_t L, void *ws_, size_t ws_bytes, cudaStream_t st)
 {
     const Layout y = make_layout(ctx, L);
     if (ws_bytes < y.total) return DQRM_ERR_WORKSPACE;
@@ -609,7 +627,7 @@ int dq_launch_bwd_reduce(dqrm_ctx *ctx, const float *grad_out, const int32_t *un
     const u32 *skeys = reinterpret_cast<const u32 *>(ws + y.keys_a), *svals = reinterpret_cast<const u32 *>(ws + y.vals_a);
     const int D = ctx->D, d4 = D / 4;
 #define DQ_RED(RL, RV, RC, LPR, CH) \
-    return launch_reduce<RL, RV, RC, LPR, CH>(ctx, y, ws, skeys, svals, uniq_off, grad_out, grad_rows, L, G, st)
+    return launch_reduce<RL, RV, RC, LPR, CH>(ctx, y, ws, skeys, svals, unique_rows, uniq_off, grad_out, grad_rows, L, G, st)
     if (D <= 4) DQ_RED(4, 1, 1, 1, 1);
     if (D <= 8) DQ_RED(8, 1, 1, 2, 1);
     if (D <= 16) DQ_RED(4, 4, 1, 4, 1);
@@ -626,7 +644,7 @@ int dq_launch_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, 
                   int32_t *unique_rows, int32_t *uniq_off, float *grad_rows, int B, int64_t L,
                   void *ws, size_t ws_bytes, cudaStream_t st, const u32 **absmax_bits_out)
 {
-    int rc = dq_launch_bwd_sort(ctx, indices, offsets, unique_rows, uniq_off, B, L, ws, ws_bytes, st, absmax_bits_out);
+    int rc = dq_launch_bwd_sort(ctx, indices, offsets, unique_rows, uniq_off, B, L, ws, ws_bytes, st, absmax_bits_out, true);
     if (rc != DQRM_OK) return rc;
-    return dq_launch_bwd_reduce(ctx, grad_out, uniq_off, grad_rows, B, L, ws, ws_bytes, st);
+    return dq_launch_bwd_reduce(ctx, grad_out, unique_rows, uniq_off, grad_rows, B, L, ws, ws_bytes, st);
 }

@@ -12,7 +12,10 @@
 // Tables whose lookups do not fit the shared-memory slices use the same algorithm on
 // global staging buffers.  The result - keys (arena rows) ascending, payloads (rows of
 // grad_out) in the original order within equal keys - is written table-major, which is
-// the globally sorted order the segmented reduction expects.
+// the globally sorted order the segmented reduction expects.  On the way out the cluster
+// also finds where every row's run begins: either it numbers its table's segments itself
+// (the kernel that sums them adds the tables' bases), or it counts the segment starts per
+// 2048-entry tile for a kernel that numbers them over the whole batch.
 #pragma once
 #include <cooperative_groups.h>
 #include "common.cuh"
@@ -40,6 +43,15 @@ struct Args {
     int payload_position;           // 0: payload = row of grad_out [B][T][D]; 1: payload = position of the lookup in indices
     int *status;
     u32 *tile_heads;                // [ceil(L / 2048)] zeroed by the caller: segment heads per tile of the sorted order
+    // lists_by_table: instead of the per-tile head counts (from which a later kernel numbers the segments over the
+    // whole batch), every cluster numbers its own table's segments from 0 and leaves
+    //   seg_start[tb0 + t + u] = sorted position where the table's segment u begins, [.. + count] = the table's end
+    //   chunk_first[c]         = the table's segment that holds sorted entry c << ck_shift (for c inside the table)
+    //   table_cnt[t], tb[t]    = segments and first sorted position of table t (tb[T] = L)
+    // and counters[fmt_slot] says so; the kernel that sums the segments adds the tables' bases
+    int lists_by_table;
+    u32 *seg_start, *chunk_first, *table_cnt, *tb, *counters;
+    int ck_shift, fmt_slot, fmt_by_table, fmt_broken;
 };
 
 __device__ __forceinline__ u32 *remote(cg::cluster_group &cluster, u32 *p, unsigned rank)
@@ -65,6 +77,9 @@ cluster_sort_kernel(const Args a)
     __shared__ u32 s_cnt[WARPS][BINS];
     __shared__ u32 s_hist[BINS];
     __shared__ u32 s_scan[BINS / 32];
+    __shared__ u32 s_wheads[WARPS];                // write-out: segment starts in each warp's part of the slice
+    __shared__ u32 s_btotal;                       // ... and in the block's slice
+    __shared__ u32 s_cbase, s_ctotal;              // ... in the blocks before this one, and in the whole table
 
     cg::cluster_group cluster = cg::this_cluster();
     const unsigned c = cluster.block_rank();
@@ -74,10 +89,19 @@ cluster_sort_kernel(const Args a)
 
     int64_t tb0 = __ldg(a.offsets + (int64_t)t * a.B), tb1 = __ldg(a.offsets + (int64_t)(t + 1) * a.B);
     if (tb0 < 0 || tb1 < tb0 || tb1 > a.L) {
-        if (threadIdx.x == 0 && c == 0) dq_report(a.status, DQRM_ERR_INDEX_RANGE);
+        if (threadIdx.x == 0 && c == 0) {
+            dq_report(a.status, DQRM_ERR_INDEX_RANGE);
+            if (a.lists_by_table) atomicMax(&a.counters[a.fmt_slot], (u32)a.fmt_broken);   // nothing downstream runs
+        }
         return;                                    // uniform over the cluster
     }
     const int64_t n = tb1 - tb0;
+    if (a.lists_by_table && c == 0 && threadIdx.x == 0) {
+        a.tb[t] = (u32)tb0;
+        if (t == a.T - 1) a.tb[a.T] = (u32)tb1;
+        if (t == 0) atomicMax(&a.counters[a.fmt_slot], (u32)a.fmt_by_table);
+        if (n == 0) a.table_cnt[t] = 0u;
+    }
     if (n == 0) return;
     const int64_t r0 = __ldg(a.row_off + t);
     const int64_t nrows = __ldg(a.row_off + t + 1) - r0;
@@ -227,7 +251,8 @@ cluster_sort_kernel(const Args a)
         s ^= 1;
     }
     // ---- write the sorted slice: arena row keys ----
-    // and count, per 2048-entry tile of the sorted order, the entries that start a new row
+    // and either count, per 2048-entry tile of the sorted order, the entries that start a new row, or number the
+    // table's segments right here
     {
         const uint2 *fin = s ? pb1 : pb0;
         u32 prev_last = 0xFFFFFFFFu;               // last row of the previous block's slice (full by construction)
@@ -236,25 +261,104 @@ cluster_sort_kernel(const Args a)
                                       : (s ? a.gp[1] : a.gp[0]) + tb0 + (int64_t)(c - 1) * npc;
             prev_last = pf[npc - 1].x;
         }
-        for (int i0 = warp * 32; i0 < my_n; i0 += THREADS) {
-            const int i = i0 + lane;
-            const bool valid = i < my_n;
-            const int64_t j = tb0 + (int64_t)c * npc + i;
-            bool head = false;
-            if (valid) {
-                const uint2 pr = fin[i];
-                a.keys_out[j] = (u32)(r0 + pr.x);
-                a.vals_out[j] = pr.y;
-                const u32 before = i > 0 ? fin[i - 1].x : prev_last;
-                head = (c == 0 && i == 0) || before != pr.x;
+        if (!a.lists_by_table) {
+            for (int i0 = warp * 32; i0 < my_n; i0 += THREADS) {
+                const int i = i0 + lane;
+                const bool valid = i < my_n;
+                const int64_t j = tb0 + (int64_t)c * npc + i;
+                bool head = false;
+                if (valid) {
+                    const uint2 pr = fin[i];
+                    a.keys_out[j] = (u32)(r0 + pr.x);
+                    a.vals_out[j] = pr.y;
+                    const u32 before = i > 0 ? fin[i - 1].x : prev_last;
+                    head = (c == 0 && i == 0) || before != pr.x;
+                }
+                const int64_t tile = j >> 11;
+                const int64_t tile0 = __shfl_sync(0xffffffffu, tile, 0);
+                const u32 m0 = __ballot_sync(0xffffffffu, head && tile == tile0);
+                const u32 m1 = __ballot_sync(0xffffffffu, head && tile != tile0);
+                if (lane == 0) {
+                    if (m0) atomicAdd(&a.tile_heads[tile0], __popc(m0));
+                    if (m1) atomicAdd(&a.tile_heads[tile0 + 1], __popc(m1));
+                }
             }
-            const int64_t tile = j >> 11;
-            const int64_t tile0 = __shfl_sync(0xffffffffu, tile, 0);
-            const u32 m0 = __ballot_sync(0xffffffffu, head && tile == tile0);
-            const u32 m1 = __ballot_sync(0xffffffffu, head && tile != tile0);
-            if (lane == 0) {
-                if (m0) atomicAdd(&a.tile_heads[tile0], __popc(m0));
-                if (m1) atomicAdd(&a.tile_heads[tile0 + 1], __popc(m1));
+        } else {
+            // every warp takes a contiguous part [w0, w1) of the slice, so that the segment starts before an entry
+            // are those of the blocks before, of the warps before, and a count the warp carries along
+            // (a part of up to 1024 entries: lane k keeps the 32 head bits of the part's k-th round, so that the
+            // second walk need not read the pairs again)
+            const bool few = wsz <= 1024;
+            u32 mine = 0, kept = 0;
+            for (int i0 = w0, it = 0; i0 < w1; i0 += 32, ++it) {
+                const int i = i0 + lane;
+                bool head = false;
+                if (i < w1) {
+                    const int64_t j = tb0 + (int64_t)c * npc + i;
+                    const uint2 pr = fin[i];
+                    a.keys_out[j] = (u32)(r0 + pr.x);
+                    a.vals_out[j] = pr.y;
+                    const u32 before = i > 0 ? fin[i - 1].x : prev_last;
+                    head = (c == 0 && i == 0) || before != pr.x;
+                }
+                const u32 m = __ballot_sync(0xffffffffu, head);
+                if (lane == it) kept = m;
+                mine += __popc(m);
+            }
+            if (lane == 0) s_wheads[warp] = mine;
+            __syncthreads();
+            if (warp == 0) {                       // the warps' bases within the block, and the block's total
+                const u32 v = lane < WARPS ? s_wheads[lane] : 0u;
+                u32 incl = v;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const u32 x = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += x;
+                }
+                if (lane < WARPS) s_wheads[lane] = incl - v;
+                if (lane == WARPS - 1) s_btotal = incl;
+            }
+            cluster.sync();                        // every block's total can be read (and the warps' bases here)
+            if (warp == 0) {                       // one warp fetches the blocks' totals: a lane per block
+                const u32 v = lane < CL ? *cluster.map_shared_rank(&s_btotal, (unsigned)lane) : 0u;
+                u32 before = lane < (int)c ? v : 0u, all = v;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    before += __shfl_xor_sync(0xffffffffu, before, o);
+                    all += __shfl_xor_sync(0xffffffffu, all, o);
+                }
+                if (lane == 0) { s_cbase = before; s_ctotal = all; }
+            }
+            __syncthreads();
+            const u32 base = s_cbase, total = s_ctotal;
+            u32 *segs = a.seg_start + tb0 + t;
+            if (c == 0 && threadIdx.x == 0) {
+                a.table_cnt[t] = total;
+                segs[total] = (u32)tb1;            // the slot behind the last segment holds the table's end
+            }
+            const u32 ck_mask = (1u << a.ck_shift) - 1u;
+            u32 before_me = base + s_wheads[warp];
+            for (int i0 = w0, it = 0; i0 < w1; i0 += 32, ++it) {
+                const int i = i0 + lane;
+                const int64_t j = tb0 + (int64_t)c * npc + i;
+                u32 m;
+                if (few) {
+                    m = __shfl_sync(0xffffffffu, kept, it);
+                } else {
+                    bool again = false;
+                    if (i < w1) {
+                        const u32 before = i > 0 ? fin[i - 1].x : prev_last;
+                        again = (c == 0 && i == 0) || before != fin[i].x;
+                    }
+                    m = __ballot_sync(0xffffffffu, again);
+                }
+                const bool head = (m >> lane) & 1u;
+                if (i < w1) {
+                    const u32 upto = before_me + __popc(m & (lt | (1u << lane)));     // segment starts in [0, i]
+                    if (head) segs[upto - 1] = (u32)j;
+                    if (((u32)j & ck_mask) == 0u) a.chunk_first[j >> a.ck_shift] = upto - 1;
+                }
+                before_me += __popc(m);
             }
         }
     }

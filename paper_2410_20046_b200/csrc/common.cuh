@@ -273,12 +273,14 @@ int dq_launch_bwd(dqrm_ctx *ctx, const float *grad_out, const int32_t *indices, 
                   int32_t *unique_rows, int32_t *uniq_off, float *grad_rows, int B, int64_t L,
                   void *ws, size_t ws_bytes, cudaStream_t st, const u32 **absmax_bits_out);
 
+// lists_by_table: dq_launch_bwd_reduce follows on the same workspace; the cluster sort then numbers each table's
+// segments itself, no separate kernel numbers them over the batch, and unique_rows / uniq_off are written by
+// dq_launch_bwd_reduce.  Without it they are complete when the sort is.
 int dq_launch_bwd_sort(dqrm_ctx *ctx, const int32_t *indices, const int32_t *offsets, int32_t *unique_rows,
                        int32_t *uniq_off, int B, int64_t L, void *ws, size_t ws_bytes, cudaStream_t st,
-                       const u32 **absmax_bits_out);
-int dq_launch_bwd_reduce(dqrm_ctx *ctx, const float *grad_out, const int32_t *uniq_off, float *grad_rows, int B,
-                         int64_t L, void *ws,
-                         size_t ws_bytes, cudaStream_t st);
+                       const u32 **absmax_bits_out, bool lists_by_table = false);
+int dq_launch_bwd_reduce(dqrm_ctx *ctx, const float *grad_out, int32_t *unique_rows, int32_t *uniq_off,
+                         float *grad_rows, int B, int64_t L, void *ws, size_t ws_bytes, cudaStream_t st);
 
 size_t dq_quant_ws_bytes(const dqrm_ctx *ctx);
 int dq_launch_grad_absmax(dqrm_ctx *ctx, const float *grad_rows, const int32_t *uniq_off, float *absmax,

@@ -3,7 +3,9 @@
 //
 // Input: keys[L] (arena rows, ascending), vals[L] (row of grad_out for each lookup, in
 // stable order), chunk_first[c] = index of the segment that holds sorted entry 32*c,
-// seg_start[U+1].  Work is dealt in chunks of 32 sorted entries, one lane group per chunk,
+// seg_start[] = sorted position where every segment begins; the segments are numbered over
+// the whole batch or per table (see LISTS_* below), and in the second case this kernel also
+// writes unique_rows and uniq_off.  Work is dealt in chunks of 32 sorted entries, one lane group per chunk,
 // but a segment is summed by the group in whose chunk it BEGINS, tail in the next chunk
 // included; the group sees where that tail ends from the next chunk's keys, which it loads
 // with its own.  All sums are FP64 and have a shape fixed by the entry positions, so results
@@ -20,7 +22,23 @@ namespace segred {
 constexpr int CHUNK = 32;            // sorted entries per lane group of the reduce (16 for a small batch of narrow rows)
 constexpr int PREFETCH_ROW_BYTES = 512;   // rows up to this size are prefetched into L2 by the reduce's head phase
 constexpr int BIG_PIECES = 32;       // cut segments with more pieces go to the block-wide fix-up
-enum { CNT_LONG = 0, CNT_U = 1, CNT_BIG = 2 };
+enum { CNT_LONG = 0, CNT_U = 1, CNT_BIG = 2, CNT_FMT = 3 };
+// counters[CNT_FMT]: how the segment lists that the sort left are laid out.
+//   LISTS_GLOBAL    seg_start[u], chunk_first[c] and uniq_off[] number the segments over the whole batch (seg_emit)
+//   LISTS_BY_TABLE  the cluster sort numbered each table's segments from 0: table t's starts sit at
+//                   seg_start[tb[t] + t + .] (tb[t] = first sorted position of the table, one slot more than it
+//                   has segments: the last holds the table's end), chunk_first[c] counts within the table that
+//                   holds entry c*CK, table_cnt[t] says how many segments the table has; unique_rows and
+//                   uniq_off are then written by the reduce, which adds the tables' bases
+//   LISTS_BROKEN    a table's boundary offsets were unusable (reported): nothing is summed, no row is updated
+enum { LISTS_GLOBAL = 0, LISTS_BY_TABLE = 1, LISTS_BROKEN = 2 };
+struct ByTable {
+    const u32 *table_cnt;       // [T]
+    const u32 *tb;              // [T+1]
+    const int64_t *row_off;     // [T+1]
+    int32_t *unique_rows;       // [U] out
+    int32_t *uniq_off;          // [T+1] out
+};
 
 template <int LPR>
 __device__ __forceinline__ u32 group_mask()
@@ -123,16 +141,58 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
                   const float *__restrict__ grad_out, float *__restrict__ grad_rows,
                   double *__restrict__ partials, uint4 *__restrict__ long_list, u32 *__restrict__ counters,
                   u32 *__restrict__ absmax, int T, int D_any,
-                  int64_t L, int64_t G, int64_t num_chunks, int *__restrict__ status)
+                  int64_t L, int64_t G, int64_t num_chunks, int *__restrict__ status, const ByTable bt)
 {
     // EXACT: the feature size fills the lanes exactly, so it is a compile-time constant and the
     // per-vector range checks fall away
     const int D = EXACT ? LPR * VEC * CH : D_any;
     extern __shared__ unsigned char smem_raw[];
     u32 *s_uoff = reinterpret_cast<u32 *>(smem_raw);                                     // [T+1]
-    u32 *s_vals = s_uoff + (T + 1) + (size_t)(threadIdx.x / LPR) * (2 * CK);          // this group's [2*CK]
-    for (int t = threadIdx.x; t <= T; t += blockDim.x) s_uoff[t] = (u32)uniq_off[t];
-    __syncthreads();
+    u32 *s_tb = s_uoff + (T + 1);                                                        // [T+1] (lists by table)
+    u32 *s_vals = s_tb + (T + 1) + (size_t)(threadIdx.x / LPR) * (2 * CK);            // this group's [2*CK]
+    // (the first T+1 threads fetch what either layout of the lists needs before the layout is known, so that the
+    // kernel starts with one round trip to memory, not two)
+    u32 r_tb = 0u, r_cnt = 0u, r_uo = 0u;
+    if ((int)threadIdx.x <= T) { r_tb = bt.tb[threadIdx.x]; r_uo = (u32)uniq_off[threadIdx.x]; }
+    if ((int)threadIdx.x < T) r_cnt = bt.table_cnt[threadIdx.x];
+    const u32 fmt = counters[CNT_FMT];
+    if (fmt == LISTS_BROKEN) {                    // (block-uniform)
+        if (blockIdx.x == 0) {
+            for (int t = threadIdx.x; t <= T; t += blockDim.x) bt.uniq_off[t] = 0;
+            if (threadIdx.x == 0) counters[CNT_U] = 0u;
+        }
+        return;
+    }
+    const bool by_table = fmt == LISTS_BY_TABLE;
+    if (by_table) {
+        // the tables' first segments: a running sum over their segment counts (T is small against the batch; one
+        // warp adds them up 32 at a time)
+        if (threadIdx.x < 32) {
+            u32 run = 0;
+            for (int t0 = 0; t0 < T; t0 += 32) {
+                const int t = t0 + (int)threadIdx.x;
+                const u32 cnt = t0 == 0 ? r_cnt : (t < T ? bt.table_cnt[t] : 0u);
+                u32 incl = cnt;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const u32 v = __shfl_up_sync(0xffffffffu, incl, o);
+                    if ((int)threadIdx.x >= o) incl += v;
+                }
+                if (t < T) s_uoff[t] = run + incl - cnt;
+                run += __shfl_sync(0xffffffffu, incl, 31);
+            }
+            if (threadIdx.x == 0) s_uoff[T] = run;
+        }
+        for (int t = threadIdx.x; t <= T; t += blockDim.x) s_tb[t] = t == (int)threadIdx.x ? r_tb : bt.tb[t];
+        __syncthreads();
+        if (blockIdx.x == 0) {
+            for (int t = threadIdx.x; t <= T; t += blockDim.x) bt.uniq_off[t] = (int32_t)s_uoff[t];
+            if (threadIdx.x == 0) counters[CNT_U] = s_uoff[T];
+        }
+    } else {
+        for (int t = threadIdx.x; t <= T; t += blockDim.x) s_uoff[t] = t == (int)threadIdx.x ? r_uo : (u32)uniq_off[t];
+        __syncthreads();
+    }
 
     typedef typename Vec<VEC>::type vec_t;
     constexpr int NB = (VEC == 4 && LPR > 4) ? 4 : 8;   // rows in flight per lane
@@ -180,7 +240,17 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
         u32 k_x = 0u;
         if (OWN) { if (i0 > CK) k_x = keys[i0 - CK - 1]; }
         else if (i0 + n < L) k_x = keys[i0 + n];
-        const u32 u_first = chunk_first[c];
+        u32 u_first = chunk_first[c];
+        int t_first = 0;                          // lists by table: the table that holds the chunk's first entry
+        if (by_table) {
+            int lo = 0, hi = T;                   // largest t with s_tb[t] <= i0 (empty tables share a start: the last)
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if ((int64_t)s_tb[mid] <= i0) lo = mid; else hi = mid;
+            }
+            t_first = lo;
+            u_first += s_uoff[lo];
+        }
         __syncwarp(gmask);                        // the previous chunk's payloads are no longer read
         u32 heads = 0, heads_n = 0;
 #pragma unroll
@@ -211,6 +281,27 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
             }
             const bool head = (e < n) && (kc[j] != kp[j]);
             heads |= ((__ballot_sync(gmask, head) >> gbase) & lm) << (j * LPR);
+        }
+        if (by_table) {
+            // every entry that starts a segment names the segment's row: segment of entry e = u_first + heads in (0, e]
+            int64_t base = __ldg(bt.row_off + t_first);
+            const bool one_table = (int64_t)s_tb[min(t_first + 1, T)] >= i0 + n;     // (group-uniform)
+#pragma unroll
+            for (int j = 0; j < EPL; ++j) {
+                const int e = j * LPR + lane;
+                if (e < n && kc[j] != kp[j]) {
+                    if (!one_table) {             // the chunk straddles tables: this key's own table
+                        int lo = t_first, hi = T;
+                        while (hi - lo > 1) {
+                            const int mid = (lo + hi) >> 1;
+                            if (__ldg(bt.row_off + mid) <= (int64_t)kc[j]) lo = mid; else hi = mid;
+                        }
+                        base = __ldg(bt.row_off + lo);
+                    }
+                    const u32 ue = u_first + __popc(heads & ~1u & (0xffffffffu >> (31 - e)));
+                    bt.unique_rows[ue] = (int32_t)((int64_t)kc[j] - base);
+                }
+            }
         }
         if (n_next < CK) heads_n |= 1u << n_next;   // the end of the array closes a run like a head
         const u32 k_0 = __shfl_sync(gmask, kc[0], gbase);
@@ -291,13 +382,16 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
                 }
                 if (begins && lane == 0) {
                     // the segment begins here: leave all the fix-up needs to know about it in one record
-                    const u32 sa = seg_start[u], sb = seg_start[u + 1];
-                    const u32 npieces = (sb - 1) / CK - sa / CK + 1;
                     int lo = 0, hi = T;              // its table: largest t with s_uoff[t] <= u
                     while (hi - lo > 1) {
                         const int mid = (lo + hi) >> 1;
                         if (s_uoff[mid] <= u) lo = mid; else hi = mid;
                     }
+                    // (lists by table: the table's starts sit at seg_start[tb[t] + t + .], the slot behind its last
+                    // segment holds its end)
+                    const int64_t at = by_table ? (int64_t)s_tb[lo] + lo + (u - s_uoff[lo]) : (int64_t)u;
+                    const u32 sa = seg_start[at], sb = seg_start[at + 1];
+                    const u32 npieces = (sb - 1) / CK - sa / CK + 1;
                     const uint4 rec = make_uint4(u, sa / CK, npieces, (u32)lo);
                     // (the list has a slot per chunk and every chunk begins at most one such segment; the bound only
                     // matters for a workspace that is summed twice without a sort in between, which must not write

@@ -326,6 +326,35 @@ def test_decreasing_offsets_are_reported_not_followed(oracle, sort_path):
     c.ctx.close()
 
 
+def test_table_boundary_beyond_the_lookups_is_reported_and_nothing_is_summed(oracle):
+    """A table whose first offset points past the batch's lookups cannot be sorted at all: its cluster says so,
+    the summation then touches nothing and reports zero unique rows, and the context stays usable."""
+    import paper_2410_20046_b200 as dq
+
+    wl = W.Workload("mini_bags", (50, 7, 300), D=16, B=64, alpha=1.1, bits=4, bag_mean=3.0, bag_max=6)
+    c = Case(wl)
+    idx, off, go = c.batch(0)
+    bad = off.copy()
+    bad[wl.B] = len(idx) + 3                      # where table 1 begins
+    c.ctx.set_sort_path(0)
+    L = len(idx)
+    ur = c.torch.full((L,), -1, dtype=c.torch.int32, device="cuda")
+    uo = c.torch.full((wl.T + 1,), -1, dtype=c.torch.int32, device="cuda")
+    gr = c.torch.full((L, wl.D), 7.0, dtype=c.torch.float32, device="cuda")
+    c.ctx.emb_bwd(c.dev(go), c.dev(idx), c.dev(bad), ur, uo, gr, B=wl.B, L=L)
+    with pytest.raises(dq.DqrmError) as e:
+        c.ctx.raise_on_device_error()
+    assert e.value.status == dq.ERR_INDEX_RANGE
+    assert (uo.cpu().numpy() == 0).all()
+    assert (gr.cpu().numpy() == 7.0).all() and (ur.cpu().numpy() == -1).all()
+    assert c.ctx.check_status() == dq.OK
+    g_ur, g_uo, g_gr = c.gpu_bwd(idx, off, go)    # still usable and correct
+    o_ur, o_uo, o_gr = oracle.emb_bwd(go, wl.T, wl.D, wl.B, idx, off)
+    assert bit_equal(g_ur, o_ur) and bit_equal(g_uo, o_uo)
+    assert_close_fp32(g_gr, o_gr)
+    c.ctx.close()
+
+
 def test_bad_arguments_are_refused_on_the_host():
     import ctypes
     import torch
