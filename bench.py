@@ -135,16 +135,16 @@ def base_config(wl):
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (set an entry to None when its kernel has changed since the capture)
 NCU_TRAFFIC = {
-    ("kaggle_b16384", "seg_reduce_kernel"): 31.12e6,
-    ("kaggle_b16384", "fwd_kernel"): 26.27e6,
-    ("kaggle_b16384", "row_stream_kernel<fused>"): 25.26e6,
+    ("kaggle_b16384", "seg_reduce_kernel"): 31.13e6,
+    ("kaggle_b16384", "fwd_kernel"): 26.33e6,
+    ("kaggle_b16384", "row_stream_kernel<fused>"): 25.25e6,
     # the Terabyte-shaped step captured over 2 GB of tables (the full tables are too large for a counter capture)
-    ("terabyte_2gb_b32768", "seg_reduce_kernel"): 237.87e6,
-    ("terabyte_2gb_b32768", "fwd_kernel"): 210.98e6,
-    ("terabyte_2gb_b32768", "row_stream_kernel<fused>"): 80.34e6,
+    ("terabyte_2gb_b32768", "seg_reduce_kernel"): 238.30e6,
+    ("terabyte_2gb_b32768", "fwd_kernel"): 212.28e6,
+    ("terabyte_2gb_b32768", "row_stream_kernel<fused>"): 79.73e6,
     # ... and scaled to the full tables by the reduce's algorithmic bytes (265.79 MB against 254.88 MB per launch):
     # its traffic is the upstream-gradient rows (the same) plus the unique rows it writes
-    ("terabyte_b32768", "seg_reduce_kernel"): 248.05e6,
+    ("terabyte_b32768", "seg_reduce_kernel"): 248.50e6,
 }
 
 KERNEL_BYTES = {
