@@ -411,7 +411,7 @@ int launch_reduce(dqrm_ctx *ctx, const Layout &y, char *ws, const u32 *keys, con
     const u32 *seg_start = reinterpret_cast<const u32 *>(ws + y.seg_start);
     double *partials = reinterpret_cast<double *>(ws + y.partials);
     uint4 *long_list = reinterpret_cast<uint4 *>(ws + y.long_list);
-    const size_t red_smem = (size_t)(ctx->T + 1) * 2 * sizeof(u32) + (size_t)gpb * 2 * y.ck * sizeof(u32);
+    const size_t red_smem = (size_t)(ctx->T + 1) * 3 * sizeof(u32) + (size_t)gpb * 2 * y.ck * sizeof(u32);
     ByTable bt;
     bt.table_cnt = reinterpret_cast<const u32 *>(ws + y.table_cnt);
     bt.tb = reinterpret_cast<const u32 *>(ws + y.tb);

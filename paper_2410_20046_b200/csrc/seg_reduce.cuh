@@ -149,11 +149,16 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
     extern __shared__ unsigned char smem_raw[];
     u32 *s_uoff = reinterpret_cast<u32 *>(smem_raw);                                     // [T+1]
     u32 *s_tb = s_uoff + (T + 1);                                                        // [T+1] (lists by table)
-    u32 *s_vals = s_tb + (T + 1) + (size_t)(threadIdx.x / LPR) * (2 * CK);            // this group's [2*CK]
+    u32 *s_row = s_tb + (T + 1);                                                         // [T+1] (lists by table)
+    u32 *s_vals = s_row + (T + 1) + (size_t)(threadIdx.x / LPR) * (2 * CK);           // this group's [2*CK]
     // (the first T+1 threads fetch what either layout of the lists needs before the layout is known, so that the
     // kernel starts with one round trip to memory, not two)
-    u32 r_tb = 0u, r_cnt = 0u, r_uo = 0u;
-    if ((int)threadIdx.x <= T) { r_tb = bt.tb[threadIdx.x]; r_uo = (u32)uniq_off[threadIdx.x]; }
+    u32 r_tb = 0u, r_cnt = 0u, r_uo = 0u, r_row = 0u;
+    if ((int)threadIdx.x <= T) {
+        r_tb = bt.tb[threadIdx.x];
+        r_uo = (u32)uniq_off[threadIdx.x];
+        r_row = (u32)bt.row_off[threadIdx.x];      // (arena rows are 32-bit keys throughout)
+    }
     if ((int)threadIdx.x < T) r_cnt = bt.table_cnt[threadIdx.x];
     const u32 fmt = counters[CNT_FMT];
     if (fmt == LISTS_BROKEN) {                    // (block-uniform)
@@ -183,7 +188,10 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
             }
             if (threadIdx.x == 0) s_uoff[T] = run;
         }
-        for (int t = threadIdx.x; t <= T; t += blockDim.x) s_tb[t] = t == (int)threadIdx.x ? r_tb : bt.tb[t];
+        for (int t = threadIdx.x; t <= T; t += blockDim.x) {
+            s_tb[t] = t == (int)threadIdx.x ? r_tb : bt.tb[t];
+            s_row[t] = t == (int)threadIdx.x ? r_row : (u32)bt.row_off[t];
+        }
         __syncthreads();
         if (blockIdx.x == 0) {
             for (int t = threadIdx.x; t <= T; t += blockDim.x) bt.uniq_off[t] = (int32_t)s_uoff[t];
@@ -284,7 +292,7 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
         }
         if (by_table) {
             // every entry that starts a segment names the segment's row: segment of entry e = u_first + heads in (0, e]
-            int64_t base = __ldg(bt.row_off + t_first);
+            u32 base = s_row[t_first];
             const bool one_table = (int64_t)s_tb[min(t_first + 1, T)] >= i0 + n;     // (group-uniform)
 #pragma unroll
             for (int j = 0; j < EPL; ++j) {
@@ -294,12 +302,12 @@ seg_reduce_kernel(const u32 *__restrict__ keys, const u32 *__restrict__ vals,
                         int lo = t_first, hi = T;
                         while (hi - lo > 1) {
                             const int mid = (lo + hi) >> 1;
-                            if (__ldg(bt.row_off + mid) <= (int64_t)kc[j]) lo = mid; else hi = mid;
+                            if (s_row[mid] <= kc[j]) lo = mid; else hi = mid;
                         }
-                        base = __ldg(bt.row_off + lo);
+                        base = s_row[lo];
                     }
                     const u32 ue = u_first + __popc(heads & ~1u & (0xffffffffu >> (31 - e)));
-                    bt.unique_rows[ue] = (int32_t)((int64_t)kc[j] - base);
+                    bt.unique_rows[ue] = (int32_t)(kc[j] - base);
                 }
             }
         }
