@@ -78,7 +78,7 @@ cluster_sort_kernel(const Args a)
     __shared__ u32 s_hist[BINS];
     __shared__ u32 s_scan[BINS / 32];
     __shared__ u32 s_wheads[WARPS];                // write-out: segment starts in each warp's part of the slice
-    __shared__ u32 s_btotal;                       // ... and in the block's slice
+    __shared__ u32 s_totals[16];                   // ... and in every block's slice (each block sends its own)
     __shared__ u32 s_cbase, s_ctotal;              // ... in the blocks before this one, and in the whole table
 
     cg::cluster_group cluster = cg::this_cluster();
@@ -316,11 +316,14 @@ cluster_sort_kernel(const Args a)
                     if (lane >= o) incl += x;
                 }
                 if (lane < WARPS) s_wheads[lane] = incl - v;
-                if (lane == WARPS - 1) s_btotal = incl;
+                // the block's total goes into every block's shared memory, under cover of the barrier below
+                // (sending or fetching made no measurable difference, here or for the passes' digit counts)
+                const u32 mine_all = __shfl_sync(0xffffffffu, incl, WARPS - 1);
+                if (lane < CL) *cluster.map_shared_rank(&s_totals[c], (unsigned)lane) = mine_all;
             }
-            cluster.sync();                        // every block's total can be read (and the warps' bases here)
-            if (warp == 0) {                       // one warp fetches the blocks' totals: a lane per block
-                const u32 v = lane < CL ? *cluster.map_shared_rank(&s_btotal, (unsigned)lane) : 0u;
+            cluster.sync();                        // every block's total has arrived (and the warps' bases are here)
+            if (warp == 0) {
+                const u32 v = lane < CL ? s_totals[lane] : 0u;
                 u32 before = lane < (int)c ? v : 0u, all = v;
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) {
