@@ -25,6 +25,8 @@ struct dqrm_ctx {
     int sort_path = 0;              // 0: per-table cluster sort, 1: global radix sort
     cudaStream_t side = nullptr;    // second stream: a training step sorts the indices and sums the gradient beside its forward
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    cudaStream_t low = nullptr;     // lowest priority: the forward of a step whose next batch is being sorted elsewhere
+    cudaEvent_t ev_low_fork = nullptr, ev_low_join = nullptr;
     cudaEvent_t ev_fwd = nullptr;   // recorded behind the forward of the last training step enqueued
     // host-buffer step: the upstream gradient comes in and the pooled output goes out on streams of their own
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
