@@ -350,7 +350,10 @@ int dqrm_set_sort_path(dqrm_ctx *ctx, int path);
  * sort, gradient summation: neither needs the tables or the forward's output) on a second
  * stream owned by the context (created by dqrm_create), beside the forward on the caller's
  * stream, and join the two before the touched rows are updated; the caller's stream sees one
- * ordered step.  on = 0 keeps every launch on the caller's stream.  Default: 1. */
+ * ordered step.  dqrm_train_step_sorted also moves its forward to a third, lowest-priority
+ * stream of the context (forked from and joined to the caller's stream), so that the forward's
+ * many blocks do not keep a sort of the next batch, running elsewhere, off the SMs.
+ * on = 0 keeps every launch on the caller's stream.  Default: 1. */
 int dqrm_set_overlap(dqrm_ctx *ctx, int on);
 
 /* ---- quantiser self-check (no counterpart in the paper) ----------------------------
